@@ -1,0 +1,178 @@
+/*
+ * gem_nlr.h -- C ABI of the B200 (sm_100a) library for the spectrally normalized
+ * nonnegative low-rank (NLR) K-means iteration ("GEM iteration").
+ *
+ * The library runs Algorithm 1 of the paper (restated call by call in its
+ * Algorithm 2) on one GPU:
+ *
+ *   setup      X_c = X - 1 xbar^T,  a = ||X_c||_2,  X-hat = X_c / a        (Section 3)
+ *   iteration  Theta = X-hat^T U;  ybar = y/sqrt(n) + (beta/n) q;  s = U^T ybar;
+ *              W = [U + 2 alpha X-hat Theta - alpha (ybar p^T + 1 s^T)]_+   (Eq. "gpu-positive-update")
+ *              a = ||W||_F^2, b = ||U||_F^2, h = <W, U> in FP64            (Eq. "fused-statistics")
+ *              c = FP32(sqrt(K)/sqrt(a));  U <- c W;
+ *              delta-hat = sqrt(max{c^2 a + b - 2 c h, 0} / K)             (Eq. "movement-estimate")
+ *              p = U^T 1;  q = U p - 1;  dual step if gated;  rho = ||q||_2 / sqrt(n); stop test.
+ *
+ * Conventions
+ *  - All matrices are row-major FP32.  X is n x d, U is n x r (r >= K), Theta is d x r.
+ *  - Every pointer named *_dev is DEVICE memory owned by the caller; it must stay valid
+ *    until gem_nlr_destroy.  Pointers named *_host are host memory.  The handle itself
+ *    owns only host memory (a pinned read-back record); it never calls a device allocator.
+ *  - U_dev is the single n x r factor buffer.  It is updated in place.  Between the
+ *    kernels of an iteration it holds the unnormalized W together with a pending FP32
+ *    multiplier kept on the device; whenever a call of this header returns, U_dev holds the
+ *    normalized factor (the multiplier has been applied), except after a normalization
+ *    breakdown, where it holds W as the paper's loop leaves it.
+ *  - Work is enqueued on the CUDA stream given at creation (a cudaStream_t passed as
+ *    void*; NULL is the legacy default stream).  Calls that return host-visible numbers
+ *    synchronize that stream before returning.  One handle = one stream; a handle is not
+ *    thread-safe.
+ *  - Return values: >= 0 success (GEM_NLR_OK, GEM_NLR_CONVERGED, GEM_NLR_ITER_CAP),
+ *    < 0 error.  No exception crosses this boundary and no kernel traps.
+ */
+#ifndef GEM_NLR_H
+#define GEM_NLR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GEM_NLR_OK            0   /* call succeeded; iteration neither stopped nor capped        */
+#define GEM_NLR_CONVERGED     1   /* the stopping test of Algorithm 1 fired                      */
+#define GEM_NLR_ITER_CAP      2   /* gem_nlr_run reached T iterations                            */
+#define GEM_NLR_E_INVALID    -1   /* bad argument, NULL or misaligned pointer                    */
+#define GEM_NLR_E_CUDA       -2   /* a CUDA call failed; see gem_nlr_last_error                  */
+#define GEM_NLR_E_WORKSPACE  -3   /* workspace smaller than gem_nlr_workspace_bytes              */
+#define GEM_NLR_E_BREAKDOWN  -4   /* sqrt(a) <= 1e-20: W vanished (Algorithm 1, breakdown line)   */
+#define GEM_NLR_E_NONFINITE  -5   /* a, b or h is not finite                                     */
+#define GEM_NLR_E_NOT_READY  -6   /* iteration requested before X was normalized                 */
+
+typedef struct gem_nlr gem_nlr_t;   /* opaque handle */
+
+/* Problem statement of Algorithm 1 plus the controls the paper leaves open. */
+typedef struct {
+    int64_t  n;             /* rows of X (data points)                                           */
+    int32_t  d;             /* columns of X (features)                                           */
+    int32_t  K;             /* number of clusters: radius ||U||_F^2 = K and divisor of delta-hat */
+    int32_t  r;             /* columns of U, r >= K                                              */
+    float    alpha;         /* primal step size                                                  */
+    float    beta;          /* penalty on h = g/sqrt(n); the stored penalty is beta/n            */
+    int32_t  T;             /* iteration cap                                                     */
+    int32_t  T_min;         /* no stop before this many iterations                               */
+    double   eps_d;         /* dual gate:  max{c^2 a + b - 2 c h, 0} < eps_d^2 K                 */
+    double   eps_c;         /* stop: gate and delta-hat < eps_c and rho < eps_c                  */
+    int32_t  center;        /* 1: subtract the column mean before the spectral norm (paper)      */
+    int32_t  x_inplace;     /* 1: X_dev is overwritten by X-hat; 0: X-hat lives in the workspace */
+    int32_t  pi_max_iters;  /* power-iteration cap for ||X_c||_2 (<=0: 100)                      */
+    double   pi_tol;        /* stop when |sigma_k - sigma_{k-1}| <= pi_tol * sigma_k (<=0: 1e-7) */
+    uint64_t pi_seed;       /* seed of the starting vector                                       */
+    int32_t  precision;     /* contraction arithmetic: 0 FP32 FFMA, 1 3xTF32 tensor cores,       */
+                            /* -1 let the library choose by shape                                */
+    int32_t  history;       /* 1: keep one gem_nlr_iter_info per iteration in the workspace      */
+} gem_nlr_params;
+
+/* What one iteration of Algorithm 1 produced (all FP64 as on the paper's host side). */
+typedef struct {
+    int32_t t;              /* index of the iteration (0-based)                                  */
+    int32_t dual_applied;   /* 1 if the dual-ascent gate fired                                   */
+    int32_t stop;           /* 1 if the stopping test fired at this iteration                    */
+    int32_t status;         /* GEM_NLR_OK or a negative GEM_NLR_E_* raised by this iteration     */
+    double  a, b, h;        /* ||W||_F^2, ||U_prev||_F^2, <W, U_prev>                            */
+    double  c;              /* FP64 value of the FP32 multiplier sqrt(K)/sqrt(a)                 */
+    double  delta_hat;      /* relative primal movement estimate                                 */
+    double  rho;            /* ||q||_2 / sqrt(n) for the new iterate                             */
+    double  fhat;           /* objective f-hat_y(U) at the iterate this iteration started from   */
+} gem_nlr_iter_info;
+
+/* Bytes of caller-provided device workspace needed for these parameters (0 if invalid).
+ * Includes the y/sqrt(n) and ybar vectors, Theta, p, s, the reduction partials, the
+ * optional history and, when x_inplace == 0, a copy of X.                                      */
+size_t gem_nlr_workspace_bytes(const gem_nlr_params *params);
+
+/* Device bytes the paper's own buffer table would use for the same problem:
+ * 4 (nd + nr + dr + 4n + 2r) + 24 (ceil(n/128) ceil(r/64) + 1)   (Eq. "gpu-storage").          */
+size_t gem_nlr_paper_storage_bytes(const gem_nlr_params *params);
+
+/* Create a solver.  X_dev: n x d data (16-byte aligned).  U_dev: n x r starting factor in the
+ * feasible set (nonnegative, ||U||_F^2 = K), 16-byte aligned.  workspace_dev: 256-byte aligned,
+ * at least gem_nlr_workspace_bytes.  The dual variable starts at zero.  Nothing is launched.   */
+int gem_nlr_create(gem_nlr_t **out, const gem_nlr_params *params, float *X_dev, float *U_dev,
+                   void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/* Setup of Section 3: column mean (if center), a = ||X_c||_2 by power iteration on X_c^T X_c
+ * applied implicitly (one pass over X per iteration), then X-hat = X_c / a written over X_dev
+ * (x_inplace) or into the workspace.  *a_out receives a.  Synchronizes.                        */
+int gem_nlr_spectral_norm(gem_nlr_t *h, double *a_out);
+
+/* Declare that X_dev already holds X-hat (normalized elsewhere); a is recorded only.           */
+int gem_nlr_set_normalized(gem_nlr_t *h, double a);
+
+/* Exactly one iteration of Algorithm 1 from the current (U, y).  On return U_dev holds the new
+ * normalized U and *info (may be NULL) the iteration's numbers.  Returns GEM_NLR_OK,
+ * GEM_NLR_CONVERGED if the stop test fired, or an error.  Synchronizes.                        */
+int gem_nlr_step(gem_nlr_t *h, gem_nlr_iter_info *info);
+
+/* Iterate until the stop test fires or T iterations have been taken in total.  No host round
+ * trip per iteration: the gate, the multiplier and the stop flag stay on the device.
+ * *last (may be NULL) describes the final iteration, *iters_done the total count.
+ * Returns GEM_NLR_CONVERGED, GEM_NLR_ITER_CAP or an error.  Synchronizes once at the end.      */
+int gem_nlr_run(gem_nlr_t *h, gem_nlr_iter_info *last, int32_t *iters_done);
+
+/* label_i = smallest j with U_ij = max_j U_ij (an all-zero row gets 0).  labels_dev: n int32.
+ * Enqueued on the handle's stream; does not synchronize.                                       */
+int gem_nlr_labels(gem_nlr_t *h, int32_t *labels_dev);
+
+/* f-hat_y(U) of Eq. "normalized" at the current (U, y).  Synchronizes.                         */
+int gem_nlr_objective(gem_nlr_t *h, double *fhat_out);
+
+/* Checkpoint helpers.  get: copies y/sqrt(n) (n floats, device to device) and the iteration
+ * counter; U is already in the caller's buffer.  set: the caller has written a new U into
+ * U_dev; ytilde_dev (n floats, may be NULL for zeros) and t replace the dual and the counter.  */
+int gem_nlr_get_state(gem_nlr_t *h, float *ytilde_dev, int32_t *t_out);
+int gem_nlr_set_state(gem_nlr_t *h, const float *ytilde_dev, int32_t t);
+
+/* Copies up to max_records per-iteration records (oldest first) to host memory; returns the
+ * number copied, or a negative error.  Needs params.history == 1.  Synchronizes.               */
+int gem_nlr_history(gem_nlr_t *h, gem_nlr_iter_info *records_host, int32_t max_records);
+
+/* Device pointers into the workspace, for inspection by tests (valid until destroy):
+ * which: 0 Theta (d*r floats), 1 p (r), 2 s (r), 3 ytilde (n), 4 ybar (n), 5 X-hat (n*d).      */
+int gem_nlr_buffer(gem_nlr_t *h, int32_t which, void **ptr_dev);
+
+/* Name of the kernel family chosen for the two contractions ("generic", "ffma", "tf32x3").     */
+const char *gem_nlr_path(gem_nlr_t *h);
+
+/* Text of the last CUDA error seen by this handle ("" if none).                                */
+const char *gem_nlr_last_error(gem_nlr_t *h);
+
+int gem_nlr_destroy(gem_nlr_t *h);
+
+/* Measurement helpers (no counterpart in the paper's algorithm).
+ * gem_nlr_profile(h, 1) makes every following iteration record CUDA events on the handle's
+ * stream around its two phases: (1) vector pass + first product Theta = X-hat^T U with its
+ * reductions, (2) the fused second-product kernel.  gem_nlr_profile_read returns the device
+ * milliseconds accumulated per phase and the number of iterations they cover (at most 1024
+ * iterations between two read-backs of the control block are recorded).
+ * gem_nlr_launch_count: kernels this handle has launched since creation.                       */
+int gem_nlr_profile(gem_nlr_t *h, int32_t enable);
+int gem_nlr_profile_read(gem_nlr_t *h, double *ms_first_phase, double *ms_second_product,
+                         int64_t *iterations);
+int64_t gem_nlr_launch_count(gem_nlr_t *h);
+
+/* Whole job with HOST buffers: copies X_host and U_host to device_buffer_dev, runs setup, up to
+ * T iterations and the label read-out, and copies U (into U_host) and the labels back.
+ * device_buffer_dev must hold gem_nlr_host_job_device_bytes(params) bytes (256-byte aligned).
+ * a_out, last, iters_done may be NULL.  Returns as gem_nlr_run.                                */
+size_t gem_nlr_host_job_device_bytes(const gem_nlr_params *params);
+int gem_nlr_run_host(const gem_nlr_params *params, const float *X_host, float *U_host,
+                     int32_t *labels_host, void *device_buffer_dev, size_t device_bytes,
+                     void *cuda_stream, double *a_out, gem_nlr_iter_info *last,
+                     int32_t *iters_done);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GEM_NLR_H */

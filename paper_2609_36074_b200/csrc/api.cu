@@ -1,0 +1,487 @@
+// C ABI of the NLR iteration library: argument checks, workspace layout, the host control loop.
+// Every arithmetic step of the method runs in the kernels; this file only orders launches and
+// reads back the small control block.
+#include "nlr_common.cuh"
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+#include <new>
+
+namespace gemnlr {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static int clampi(int64_t v, int64_t lo, int64_t hi) { return (int)(v < lo ? lo : (v > hi ? hi : v)); }
+
+static bool valid_params(const gem_nlr_params& P)
+{
+    if (P.n < 1 || P.d < 1 || P.K < 1 || P.r < P.K) return false;
+    if (P.r > 7168 || P.d > 2816) return false;       // shared-memory accumulators of the vector / setup passes
+    if (!(P.alpha > 0.f) || !(P.beta > 0.f)) return false;
+    if (P.T < 0 || P.T_min < 0 || P.eps_d < 0.0 || P.eps_c < 0.0) return false;
+    if (P.precision < -1 || P.precision > 1) return false;
+    return true;
+}
+
+Layout make_layout(const gem_nlr_params& P)
+{
+    Layout L;
+    memset(&L, 0, sizeof(L));
+    const int64_t n = P.n;
+    const int d = P.d, r = P.r;
+    L.g1y_d = (int)ceil_div(d, G_DT);
+    L.g1y_r = (int)ceil_div(r, G_RT);
+    const int tiles1 = L.g1y_d * L.g1y_r;
+    L.g1x = clampi(ceil_div(kSMs * 4, tiles1), 1, ceil_div(n, G_TM));
+    L.gv = clampi(ceil_div(n, 4), 1, kSMs * 8);
+    L.g2y = (int)ceil_div(r, G2_RT);
+    L.g2x = clampi(ceil_div(kSMs * 4, L.g2y), 1, ceil_div(n, G2_TM));
+    L.gs = clampi(ceil_div(n, 8), 1, kSMs * 4);
+    L.nred1 = (int)ceil_div((int64_t)d * r, 64);
+
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.ctl = take(1024);
+    L.p = take(sizeof(float) * r);
+    L.s = take(sizeof(float) * r);
+    L.alpha_s = take(sizeof(float) * r);
+    L.theta = take(sizeof(float) * (size_t)d * r);
+    L.ytilde = take(sizeof(float) * (size_t)n);
+    L.ybar = take(sizeof(float) * (size_t)n);
+    // partial areas are sized for the largest user among the kernel families
+    size_t p1 = sizeof(double) * (size_t)L.g1x * d * r;
+    size_t p1_fast = ((size_t)d * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)d * r + r + 4) : 0;
+    L.part1 = take(p1 > p1_fast ? p1 : p1_fast);
+    L.part1v = take(sizeof(double) * (size_t)L.gv * (r + 2));
+    size_t p2 = sizeof(double) * (size_t)L.g2x * L.g2y * (3 + G2_RT);
+    size_t p2_fast = sizeof(double) * (size_t)kSMs * 4 * (4 + (size_t)r);
+    L.part2 = take(p2 > p2_fast ? p2 : p2_fast);
+    L.red1 = take(sizeof(double) * (size_t)L.nred1);
+    L.setup = take(sizeof(double) * (2 * (size_t)d + 4 + (size_t)L.gs * d));
+    L.hist = take(P.history ? sizeof(gem_nlr_iter_info) * (size_t)(P.T > 0 ? P.T : 1) : 0);
+    L.xhat = take(P.x_inplace ? 0 : sizeof(float) * (size_t)n * d);
+    L.total = off;
+    return L;
+}
+
+}  // namespace gemnlr
+
+using namespace gemnlr;
+
+struct gem_nlr {
+    Problem pb;
+    float* X_in;
+    bool normalized;
+    bool loaded;           // p = U^T 1 is on the device for the current U
+    double a;
+    int32_t t_host;        // iterations completed as of the last read-back
+    int32_t sticky_error;
+    Ctl* host_ctl;         // pinned read-back record
+    double* host_scratch;  // pinned
+    const char* path;
+    char err[256];
+    int64_t launches;      // kernels launched by this handle
+    int pi_iters;          // power iterations taken by the last setup
+    // optional per-phase timing: events recorded around the two passes of every iteration
+    bool profile;
+    cudaEvent_t* ev;       // 3 per iteration: start, after the first-product phase, after the second product
+    int ev_cap, ev_used;
+    double prof_ms[3];     // accumulated: first-product phase, second-product kernel, (unused)
+    int64_t prof_iters;
+};
+
+static int cuda_fail(gem_nlr_t* h, cudaError_t e, const char* where)
+{
+    snprintf(h->err, sizeof(h->err), "%s: %s", where, cudaGetErrorString(e));
+    h->sticky_error = GEM_NLR_E_CUDA;
+    return GEM_NLR_E_CUDA;
+}
+
+#define CK(h, call)                                                   \
+    do {                                                              \
+        cudaError_t e__ = (call);                                     \
+        if (e__ != cudaSuccess) return cuda_fail((h), e__, #call);    \
+    } while (0)
+
+static int reset_ctl(gem_nlr_t* h, int32_t t)
+{
+    Ctl c;
+    memset(&c, 0, sizeof(c));
+    c.c_f = 1.0f;
+    c.t = t;
+    c.hist_cap = h->pb.P.history ? (h->pb.P.T > 0 ? h->pb.P.T : 1) : 0;
+    *h->host_ctl = c;
+    CK(h, cudaMemcpyAsync(h->pb.ctl(), h->host_ctl, sizeof(Ctl), cudaMemcpyHostToDevice, h->pb.stream));
+    CK(h, cudaStreamSynchronize(h->pb.stream));   // host_ctl is reused for read-backs
+    h->t_host = t;
+    h->loaded = false;
+    return GEM_NLR_OK;
+}
+
+static int read_ctl(gem_nlr_t* h)
+{
+    CK(h, cudaMemcpyAsync(h->host_ctl, h->pb.ctl(), sizeof(Ctl), cudaMemcpyDeviceToHost, h->pb.stream));
+    CK(h, cudaStreamSynchronize(h->pb.stream));
+    CK(h, cudaGetLastError());
+    h->t_host = h->host_ctl->t;
+    return GEM_NLR_OK;
+}
+
+static int ensure_loaded(gem_nlr_t* h)
+{
+    if (!h->loaded) {
+        launch_init_colsum(h->pb);
+        h->loaded = true;
+    }
+    return GEM_NLR_OK;
+}
+
+// One iteration = vector pass + first product (+ reductions), then the fused second product
+// and its scalar reduction.  With profiling on, events bracket the two phases.
+static void launch_iteration(gem_nlr_t* h)
+{
+    const bool prof = h->profile && h->ev_used + 3 <= h->ev_cap;
+    cudaEvent_t* e = prof ? h->ev + h->ev_used : nullptr;
+    if (prof) cudaEventRecord(e[0], h->pb.stream);
+    launch_vector_pass(h->pb);
+    launch_generic_pass1(h->pb, 0);
+    launch_fin1(h->pb, 0);
+    if (prof) cudaEventRecord(e[1], h->pb.stream);
+    launch_generic_pass2_kernel(h->pb);
+    if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
+    launch_fin2(h->pb, h->pb.L.g2x, h->pb.L.g2y, G2_RT);
+}
+
+static void drain_profile(gem_nlr_t* h)
+{
+    for (int i = 0; i + 2 < h->ev_used; i += 3) {
+        float a = 0.f, b = 0.f;
+        if (cudaEventElapsedTime(&a, h->ev[i], h->ev[i + 1]) == cudaSuccess &&
+            cudaEventElapsedTime(&b, h->ev[i + 1], h->ev[i + 2]) == cudaSuccess) {
+            h->prof_ms[0] += a;
+            h->prof_ms[1] += b;
+            h->prof_iters += 1;
+        }
+    }
+    h->ev_used = 0;
+}
+
+static int clear_stop(gem_nlr_t* h)
+{
+    // a previous "converged" stop does not forbid further iterations; errors are sticky
+    CK(h, cudaMemsetAsync(&h->pb.ctl()->stopped, 0, 2 * sizeof(int32_t), h->pb.stream));
+    return GEM_NLR_OK;
+}
+
+extern "C" {
+
+size_t gem_nlr_workspace_bytes(const gem_nlr_params* params)
+{
+    if (!params || !valid_params(*params)) return 0;
+    return make_layout(*params).total;
+}
+
+size_t gem_nlr_paper_storage_bytes(const gem_nlr_params* params)
+{
+    if (!params || !valid_params(*params)) return 0;
+    const size_t n = (size_t)params->n, d = (size_t)params->d, r = (size_t)params->r;
+    const size_t n_tile = ((n + 127) / 128) * ((r + 63) / 64);
+    return 4 * (n * d + n * r + d * r + 4 * n + 2 * r) + 24 * (n_tile + 1);
+}
+
+int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, float* U_dev,
+                   void* workspace_dev, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!out) return GEM_NLR_E_INVALID;
+    *out = nullptr;
+    if (!params || !X_dev || !U_dev || !workspace_dev) return GEM_NLR_E_INVALID;
+    if (!valid_params(*params)) return GEM_NLR_E_INVALID;
+    if (((uintptr_t)X_dev & 15) || ((uintptr_t)U_dev & 15) || ((uintptr_t)workspace_dev & 255))
+        return GEM_NLR_E_INVALID;
+    Layout L = make_layout(*params);
+    if (workspace_bytes < L.total) return GEM_NLR_E_WORKSPACE;
+    gem_nlr_t* h = new (std::nothrow) gem_nlr_t;
+    if (!h) return GEM_NLR_E_INVALID;
+    memset(h, 0, sizeof(*h));
+    h->pb.P = *params;
+    h->pb.L = L;
+    h->pb.ws = (char*)workspace_dev;
+    h->pb.U = U_dev;
+    h->X_in = X_dev;
+    h->pb.X = params->x_inplace ? X_dev : (float*)((char*)workspace_dev + L.xhat);
+    h->pb.stream = (cudaStream_t)cuda_stream;
+    h->pb.gamma = (double)params->beta / (double)params->n;
+    h->pb.gamma_f = (float)h->pb.gamma;
+    h->path = "generic";
+    h->err[0] = 0;
+    h->pb.launches = &h->launches;
+    if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||
+        cudaMallocHost((void**)&h->host_scratch, 64) != cudaSuccess) {
+        if (h->host_ctl) cudaFreeHost(h->host_ctl);
+        delete h;
+        return GEM_NLR_E_CUDA;
+    }
+    int rc = reset_ctl(h, 0);
+    if (rc == GEM_NLR_OK &&
+        cudaMemsetAsync(h->pb.ytilde(), 0, sizeof(float) * (size_t)params->n, h->pb.stream) != cudaSuccess)
+        rc = GEM_NLR_E_CUDA;
+    if (rc != GEM_NLR_OK) {
+        cudaFreeHost(h->host_ctl);
+        cudaFreeHost(h->host_scratch);
+        delete h;
+        return rc;
+    }
+    *out = h;
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_spectral_norm(gem_nlr_t* h, double* a_out)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (h->sticky_error) return h->sticky_error;
+    if (h->normalized) return GEM_NLR_E_INVALID;     // X_dev already holds X-hat
+    double a = 0.0;
+    int rc = run_spectral_norm(h->pb, h->X_in, h->pb.X, &a, h->host_scratch);
+    if (rc != GEM_NLR_OK) {
+        if (rc == GEM_NLR_E_CUDA) return cuda_fail(h, cudaGetLastError(), "spectral_norm");
+        return rc;
+    }
+    CK(h, cudaStreamSynchronize(h->pb.stream));
+    h->a = a;
+    h->normalized = true;
+    if (a_out) *a_out = a;
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_set_normalized(gem_nlr_t* h, double a)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (!h->pb.P.x_inplace) return GEM_NLR_E_INVALID;  // X-hat must be in the caller's buffer
+    h->a = a;
+    h->normalized = true;
+    return GEM_NLR_OK;
+}
+
+static int result_code(gem_nlr_t* h, bool capped)
+{
+    const Ctl& c = *h->host_ctl;
+    if (c.status < 0) { h->sticky_error = c.status; return c.status; }
+    if (c.last.stop) return GEM_NLR_CONVERGED;
+    return capped ? GEM_NLR_ITER_CAP : GEM_NLR_OK;
+}
+
+int gem_nlr_step(gem_nlr_t* h, gem_nlr_iter_info* info)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (h->sticky_error) return h->sticky_error;
+    if (!h->normalized) return GEM_NLR_E_NOT_READY;
+    int rc = clear_stop(h);
+    if (rc) return rc;
+    ensure_loaded(h);
+    launch_iteration(h);
+    launch_tail(h->pb);
+    rc = read_ctl(h);
+    if (rc) return rc;
+    if (info) *info = h->host_ctl->last;
+    return result_code(h, false);
+}
+
+int gem_nlr_run(gem_nlr_t* h, gem_nlr_iter_info* last, int32_t* iters_done)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (h->sticky_error) return h->sticky_error;
+    if (!h->normalized) return GEM_NLR_E_NOT_READY;
+    int rc = clear_stop(h);
+    if (rc) return rc;
+    ensure_loaded(h);
+    const int32_t T = h->pb.P.T, T_min = h->pb.P.T_min;
+    const int32_t t0 = h->t_host;
+    int since_check = 0;
+    for (int32_t t = t0; t < T; ++t) {
+        launch_iteration(h);
+        ++since_check;
+        // The stop test of iteration t is evaluated by the first kernels of iteration t + 1, so a
+        // flag seen here is at most one iteration old; kernels launched after a stop return at once.
+        if (t + 1 >= T_min && since_check >= 16 && t + 1 < T) {
+            rc = read_ctl(h);
+            if (rc) return rc;
+            if (h->profile) drain_profile(h);
+            since_check = 0;
+            if (h->host_ctl->stopped) break;
+        }
+    }
+    launch_tail(h->pb);
+    rc = read_ctl(h);
+    if (rc) return rc;
+    if (h->profile) drain_profile(h);
+    if (last) *last = h->host_ctl->last;
+    if (iters_done) *iters_done = h->host_ctl->t;
+    return result_code(h, true);
+}
+
+int gem_nlr_labels(gem_nlr_t* h, int32_t* labels_dev)
+{
+    if (!h || !labels_dev) return GEM_NLR_E_INVALID;
+    launch_labels(h->pb, labels_dev);
+    CK(h, cudaGetLastError());
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_objective(gem_nlr_t* h, double* fhat_out)
+{
+    if (!h || !fhat_out) return GEM_NLR_E_INVALID;
+    if (!h->normalized) return GEM_NLR_E_NOT_READY;
+    ensure_loaded(h);
+    launch_objective(h->pb);
+    int rc = read_ctl(h);
+    if (rc) return rc;
+    *fhat_out = h->host_ctl->f_final;
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_get_state(gem_nlr_t* h, float* ytilde_dev, int32_t* t_out)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (ytilde_dev)
+        CK(h, cudaMemcpyAsync(ytilde_dev, h->pb.ytilde(), sizeof(float) * (size_t)h->pb.P.n,
+                              cudaMemcpyDeviceToDevice, h->pb.stream));
+    CK(h, cudaStreamSynchronize(h->pb.stream));
+    if (t_out) *t_out = h->t_host;
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_set_state(gem_nlr_t* h, const float* ytilde_dev, int32_t t)
+{
+    if (!h || t < 0) return GEM_NLR_E_INVALID;
+    if (ytilde_dev)
+        CK(h, cudaMemcpyAsync(h->pb.ytilde(), ytilde_dev, sizeof(float) * (size_t)h->pb.P.n,
+                              cudaMemcpyDeviceToDevice, h->pb.stream));
+    else
+        CK(h, cudaMemsetAsync(h->pb.ytilde(), 0, sizeof(float) * (size_t)h->pb.P.n, h->pb.stream));
+    h->sticky_error = 0;
+    return reset_ctl(h, t);
+}
+
+int gem_nlr_history(gem_nlr_t* h, gem_nlr_iter_info* records_host, int32_t max_records)
+{
+    if (!h || !records_host || max_records < 0) return GEM_NLR_E_INVALID;
+    if (!h->pb.P.history) return GEM_NLR_E_INVALID;
+    int rc = read_ctl(h);
+    if (rc) return rc;
+    int n = h->host_ctl->hist_len < max_records ? h->host_ctl->hist_len : max_records;
+    if (n > 0) CK(h, cudaMemcpy(records_host, h->pb.hist(), sizeof(gem_nlr_iter_info) * (size_t)n,
+                                cudaMemcpyDeviceToHost));
+    return n;
+}
+
+int gem_nlr_buffer(gem_nlr_t* h, int32_t which, void** ptr_dev)
+{
+    if (!h || !ptr_dev) return GEM_NLR_E_INVALID;
+    switch (which) {
+        case 0: *ptr_dev = h->pb.theta(); break;
+        case 1: *ptr_dev = h->pb.p(); break;
+        case 2: *ptr_dev = h->pb.s(); break;
+        case 3: *ptr_dev = h->pb.ytilde(); break;
+        case 4: *ptr_dev = h->pb.ybar(); break;
+        case 5: *ptr_dev = h->pb.X; break;
+        default: return GEM_NLR_E_INVALID;
+    }
+    return GEM_NLR_OK;
+}
+
+const char* gem_nlr_path(gem_nlr_t* h) { return h ? h->path : ""; }
+
+const char* gem_nlr_last_error(gem_nlr_t* h) { return h ? h->err : ""; }
+
+int gem_nlr_destroy(gem_nlr_t* h)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    cudaStreamSynchronize(h->pb.stream);
+    if (h->host_ctl) cudaFreeHost(h->host_ctl);
+    if (h->host_scratch) cudaFreeHost(h->host_scratch);
+    if (h->ev) {
+        for (int i = 0; i < h->ev_cap; ++i) cudaEventDestroy(h->ev[i]);
+        delete[] h->ev;
+    }
+    delete h;
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_profile(gem_nlr_t* h, int32_t enable)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (enable && !h->ev) {
+        h->ev_cap = 3 * 1024;
+        h->ev = new (std::nothrow) cudaEvent_t[h->ev_cap];
+        if (!h->ev) return GEM_NLR_E_INVALID;
+        for (int i = 0; i < h->ev_cap; ++i) CK(h, cudaEventCreate(&h->ev[i]));
+    }
+    h->profile = enable != 0;
+    h->ev_used = 0;
+    h->prof_ms[0] = h->prof_ms[1] = h->prof_ms[2] = 0.0;
+    h->prof_iters = 0;
+    return GEM_NLR_OK;
+}
+
+int gem_nlr_profile_read(gem_nlr_t* h, double* ms_first_phase, double* ms_second_product,
+                         int64_t* iterations)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (ms_first_phase) *ms_first_phase = h->prof_ms[0];
+    if (ms_second_product) *ms_second_product = h->prof_ms[1];
+    if (iterations) *iterations = h->prof_iters;
+    return GEM_NLR_OK;
+}
+
+int64_t gem_nlr_launch_count(gem_nlr_t* h) { return h ? h->launches : 0; }
+
+size_t gem_nlr_host_job_device_bytes(const gem_nlr_params* params)
+{
+    if (!params || !valid_params(*params)) return 0;
+    gem_nlr_params P = *params;
+    P.x_inplace = 1;
+    const size_t n = (size_t)P.n;
+    return align_up(4 * n * P.d, 256) + align_up(4 * n * P.r, 256) + align_up(4 * n, 256) +
+           make_layout(P).total;
+}
+
+int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U_host,
+                     int32_t* labels_host, void* device_buffer_dev, size_t device_bytes,
+                     void* cuda_stream, double* a_out, gem_nlr_iter_info* last, int32_t* iters_done)
+{
+    if (!params || !X_host || !U_host || !device_buffer_dev) return GEM_NLR_E_INVALID;
+    if (!valid_params(*params) || ((uintptr_t)device_buffer_dev & 255)) return GEM_NLR_E_INVALID;
+    if (device_bytes < gem_nlr_host_job_device_bytes(params)) return GEM_NLR_E_WORKSPACE;
+    gem_nlr_params P = *params;
+    P.x_inplace = 1;
+    const size_t n = (size_t)P.n;
+    char* base = (char*)device_buffer_dev;
+    float* Xd = (float*)base;
+    float* Ud = (float*)(base + align_up(4 * n * P.d, 256));
+    int32_t* Ld = (int32_t*)((char*)Ud + align_up(4 * n * P.r, 256));
+    char* ws = (char*)Ld + align_up(4 * n, 256);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(Xd, X_host, 4 * n * P.d, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(Ud, U_host, 4 * n * P.r, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return GEM_NLR_E_CUDA;
+    gem_nlr_t* h = nullptr;
+    int rc = gem_nlr_create(&h, &P, Xd, Ud, ws, make_layout(P).total, cuda_stream);
+    if (rc < 0) return rc;
+    rc = gem_nlr_spectral_norm(h, a_out);
+    int run_rc = rc;
+    if (rc >= 0) run_rc = gem_nlr_run(h, last, iters_done);
+    if (run_rc >= 0 || run_rc == GEM_NLR_E_BREAKDOWN) {
+        if (labels_host) {
+            gem_nlr_labels(h, Ld);
+            if (cudaMemcpyAsync(labels_host, Ld, 4 * n, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+                run_rc = GEM_NLR_E_CUDA;
+        }
+        if (cudaMemcpyAsync(U_host, Ud, 4 * n * P.r, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            run_rc = GEM_NLR_E_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) run_rc = GEM_NLR_E_CUDA;
+    }
+    gem_nlr_destroy(h);
+    return run_rc;
+}
+
+}  // extern "C"

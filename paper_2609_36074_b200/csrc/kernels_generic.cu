@@ -1,0 +1,593 @@
+// Generic kernel family of the NLR iteration: works for every (n, d, r), plain global loads,
+// shared-memory tiles and FP32 FFMA.  It is the fallback for shapes the specialised families
+// do not cover and the reference the specialised families are cross-checked against on the GPU.
+//
+// Reductions are deterministic: every partial sum has a fixed owner and partials are combined
+// in a fixed order (FP64), so two runs on the same inputs give the same bits.
+#include "nlr_common.cuh"
+#include "device_utils.cuh"
+
+namespace gemnlr {
+
+// ------------------------------------------------------------------------------------------
+// Vector pass (Algorithm 2, call sites 2, 3, 8-11 in one sweep over U): one warp per row.
+//   u_i = c_f * w_i ; q_i = u_i . p - 1 ; if gate pending: ytilde_i += gamma q_i ;
+//   ybar_i = ytilde_i + gamma q_i ; s += u_i ybar_i ; sum q_i^2 ; sum ytilde_i q_i.
+// MATERIALIZE additionally writes u_i back (the scaling call U <- c W).
+// Output: part[blockIdx][0..r-1] = s partial, [r] = sum q^2, [r+1] = sum ytilde q.
+// ------------------------------------------------------------------------------------------
+constexpr int RV_WARPS = 4;
+
+template <bool MATERIALIZE>
+__global__ void __launch_bounds__(RV_WARPS * 32)
+k_rowvec(float* __restrict__ U, float* __restrict__ ytilde, float* __restrict__ ybar,
+         const Ctl* __restrict__ ctl, const float* __restrict__ p, int64_t n, int r, double gamma,
+         double* __restrict__ part, int ignore_stop)
+{
+    if (!ignore_stop && ctl->stopped) return;
+    extern __shared__ double sm_s[];              // [RV_WARPS][r]
+    __shared__ double sm_red[2][RV_WARPS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float cf = ctl->c_f;
+    const int dual = ctl->dual_pending;
+    double* my_s = sm_s + (size_t)warp * r;
+    for (int j = lane; j < r; j += 32) my_s[j] = 0.0;
+    double qq = 0.0, yq = 0.0;
+    const int64_t stride = (int64_t)gridDim.x * RV_WARPS;
+    for (int64_t row = (int64_t)blockIdx.x * RV_WARPS + warp; row < n; row += stride) {
+        float* urow = U + row * r;
+        float acc = 0.f;
+        for (int j = lane; j < r; j += 32) {
+            float u = cf * urow[j];
+            acc = fmaf(u, p[j], acc);
+        }
+        acc = warp_sum(acc);
+        const float q = acc - 1.0f;
+        float yt = ytilde[row];
+        if (dual) yt = (float)((double)yt + gamma * (double)q);
+        const float yb = (float)((double)yt + gamma * (double)q);
+        if (lane == 0) {
+            if (dual) ytilde[row] = yt;
+            ybar[row] = yb;
+            qq += (double)q * (double)q;
+            yq += (double)yt * (double)q;
+        }
+        for (int j = lane; j < r; j += 32) {
+            float u = cf * urow[j];
+            my_s[j] += (double)u * (double)yb;
+            if (MATERIALIZE) urow[j] = u;
+        }
+    }
+    if (lane == 0) { sm_red[0][warp] = qq; sm_red[1][warp] = yq; }
+    __syncthreads();
+    double* out = part + (size_t)blockIdx.x * (r + 2);
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+        double v = 0.0;
+        for (int w = 0; w < RV_WARPS; ++w) v += sm_s[(size_t)w * r + j];
+        out[j] = v;
+    }
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < RV_WARPS; ++w) { a += sm_red[0][w]; b += sm_red[1][w]; }
+        out[r] = a;
+        out[r + 1] = b;
+    }
+}
+
+// Column sums of c_f * U (p = U^T 1 for a freshly loaded factor): part[blockIdx][0..r-1].
+__global__ void __launch_bounds__(RV_WARPS * 32)
+k_colsum(const float* __restrict__ U, const Ctl* __restrict__ ctl, int64_t n, int r,
+         double* __restrict__ part)
+{
+    extern __shared__ double sm_s[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float cf = ctl->c_f;
+    double* my_s = sm_s + (size_t)warp * r;
+    for (int j = lane; j < r; j += 32) my_s[j] = 0.0;
+    const int64_t stride = (int64_t)gridDim.x * RV_WARPS;
+    for (int64_t row = (int64_t)blockIdx.x * RV_WARPS + warp; row < n; row += stride) {
+        const float* urow = U + row * r;
+        for (int j = lane; j < r; j += 32) my_s[j] += (double)(cf * urow[j]);
+    }
+    __syncthreads();
+    double* out = part + (size_t)blockIdx.x * (r + 2);
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+        double v = 0.0;
+        for (int w = 0; w < RV_WARPS; ++w) v += sm_s[(size_t)w * r + j];
+        out[j] = v;
+    }
+}
+
+__global__ void k_fin_colsum(const double* __restrict__ part, int g, int r, float* __restrict__ p)
+{
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+        double v = 0.0;
+        for (int b = 0; b < g; ++b) v += part[(size_t)b * (r + 2) + j];
+        p[j] = (float)v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// First product, Theta = X-hat^T U, as split-K partials: CTA (gx, tile) accumulates the
+// G_DT x G_RT tile of Theta over its contiguous row chunk.  Per row tile the sums run in FP32
+// registers and are then folded into FP64 running sums, so the FP32 chains stay G_TM long.
+// part[gx][j * r + k] (FP64).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_pass1_generic(const float* __restrict__ X, const float* __restrict__ U,
+                const Ctl* __restrict__ ctl, int64_t n, int d, int r, int tiles_r,
+                double* __restrict__ part, int ignore_stop)
+{
+    if (!ignore_stop && ctl->stopped) return;
+    __shared__ __align__(16) float Xs[G_TM][G_DT];
+    __shared__ __align__(16) float Us[G_TM][G_RT];
+    const float cf = ctl->c_f;
+    const int tile = blockIdx.y;
+    const int j0 = (tile / tiles_r) * G_DT, k0 = (tile % tiles_r) * G_RT;
+    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+    const int64_t rows_per = (n + gridDim.x - 1) / gridDim.x;
+    const int64_t r_lo = (int64_t)blockIdx.x * rows_per;
+    const int64_t r_hi = (r_lo + rows_per < n) ? r_lo + rows_per : n;
+    double acc64[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc64[a][b] = 0.0;
+    for (int64_t m0 = r_lo; m0 < r_hi; m0 += G_TM) {
+        for (int idx = threadIdx.x; idx < G_TM * G_DT; idx += 256) {
+            int m = idx / G_DT, jj = idx % G_DT;
+            int64_t row = m0 + m;
+            int col = j0 + jj;
+            Xs[m][jj] = (row < r_hi && col < d) ? X[row * d + col] : 0.f;
+        }
+        for (int idx = threadIdx.x; idx < G_TM * G_RT; idx += 256) {
+            int m = idx / G_RT, kk = idx % G_RT;
+            int64_t row = m0 + m;
+            int col = k0 + kk;
+            Us[m][kk] = (row < r_hi && col < r) ? cf * U[row * r + col] : 0.f;
+        }
+        __syncthreads();
+        float acc[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+#pragma unroll 8
+        for (int m = 0; m < G_TM; ++m) {
+            const float4 xv = *reinterpret_cast<const float4*>(&Xs[m][ty * 4]);
+            const float4 uv = *reinterpret_cast<const float4*>(&Us[m][tx * 4]);
+            const float xa[4] = {xv.x, xv.y, xv.z, xv.w};
+            const float ua[4] = {uv.x, uv.y, uv.z, uv.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xa[a], ua[b], acc[a][b]);
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc64[a][b] += (double)acc[a][b];
+        __syncthreads();
+    }
+    double* out = part + (size_t)blockIdx.x * ((size_t)d * r);
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        int j = j0 + ty * 4 + a;
+        if (j >= d) continue;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            int k = k0 + tx * 4 + b;
+            if (k < r) out[(size_t)j * r + k] = acc64[a][b];
+        }
+    }
+}
+
+// Theta[e] = FP32(sum_g part[g][e]) in ascending g (four interleaved slices combined in order);
+// red[blockIdx] = this block's share of ||Theta||_F^2 (from the unrounded sums).
+__global__ void __launch_bounds__(256)
+k_red1(const double* __restrict__ part, int g, int64_t dr, const Ctl* __restrict__ ctl,
+       float* __restrict__ theta, double* __restrict__ red, int ignore_stop)
+{
+    if (!ignore_stop && ctl->stopped) return;
+    __shared__ double sl[4][64];
+    __shared__ double sred[32];
+    const int e_local = threadIdx.x & 63, slice = threadIdx.x >> 6;
+    const int64_t e = (int64_t)blockIdx.x * 64 + e_local;
+    double v = 0.0;
+    if (e < dr)
+        for (int b = slice; b < g; b += 4) v += part[(size_t)b * dr + e];
+    sl[slice][e_local] = v;
+    __syncthreads();
+    double t2 = 0.0;
+    if (slice == 0 && e < dr) {
+        double tot = ((sl[0][e_local] + sl[1][e_local]) + sl[2][e_local]) + sl[3][e_local];
+        theta[e] = (float)tot;
+        t2 = tot * tot;
+    }
+    t2 = block_sum<256>(t2, sred);
+    if (threadIdx.x == 0) red[blockIdx.x] = t2;
+}
+
+// Scalars after the vector pass (and the Theta reduction): s, alpha*s, sum q^2, sum ytilde q,
+// ||Theta||^2; finishes the previous iteration (rho, stop test, history record).
+// mode 0: start of an iteration, 1: tail (also resets the multiplier after the U buffer was
+// rescaled), 2: objective evaluation only.
+__global__ void __launch_bounds__(256)
+k_fin1(Ctl* __restrict__ ctl, const double* __restrict__ part1v, int gv, const double* __restrict__ red,
+       int nred, int r, int64_t n, float alpha, double gamma, double eps_c, int T_min,
+       float* __restrict__ s, float* __restrict__ alpha_s, gem_nlr_iter_info* __restrict__ hist, int mode)
+{
+    if (mode == 0 && ctl->stopped) return;
+    __shared__ double sred[32];
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+        double v = 0.0;
+        for (int b = 0; b < gv; ++b) v += part1v[(size_t)b * (r + 2) + j];
+        float sf = (float)v;
+        s[j] = sf;
+        alpha_s[j] = alpha * sf;
+    }
+    double qq = 0.0, yq = 0.0, t2 = 0.0;
+    for (int b = threadIdx.x; b < gv; b += blockDim.x) {
+        qq += part1v[(size_t)b * (r + 2) + r];
+        yq += part1v[(size_t)b * (r + 2) + r + 1];
+    }
+    if (mode != 1)
+        for (int b = threadIdx.x; b < nred; b += blockDim.x) t2 += red[b];
+    qq = block_sum<256>(qq, sred);
+    yq = block_sum<256>(yq, sred);
+    t2 = block_sum<256>(t2, sred);
+    if (threadIdx.x == 0) {
+        ctl->qq = qq;
+        ctl->yq = yq;
+        if (mode != 1) ctl->theta2 = t2;
+        if (ctl->tail_pending) {
+            gem_nlr_iter_info rec = ctl->last;
+            rec.rho = sqrt(qq / (double)n);
+            rec.stop = (rec.dual_applied && rec.delta_hat < eps_c && rec.rho < eps_c &&
+                        rec.t + 1 >= T_min) ? 1 : 0;
+            ctl->last = rec;
+            if (ctl->hist_cap > 0 && rec.t < ctl->hist_cap) {
+                hist[rec.t] = rec;
+                ctl->hist_len = rec.t + 1;
+            }
+            ctl->tail_pending = 0;
+            ctl->dual_pending = 0;
+            if (rec.stop) { ctl->stopped = 1; ctl->status = GEM_NLR_CONVERGED; }
+        }
+        if (mode != 1) {
+            double f = -t2 + yq + 0.5 * gamma * qq;
+            if (mode == 0) ctl->fhat_cur = f;
+            if (mode == 2 || ctl->stopped) ctl->f_final = f;
+        } else {
+            ctl->c_f = 1.0f;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Second product with the fused epilogue (Eq. "entrywise-fusion"): for a G2_TM x G2_RT output
+// tile, acc = (X-hat Theta)_ij, u = c_f * U_ij,
+//   w = max{ u + 2 alpha acc - alpha ybar_i p_j - alpha s_j, 0 },  U_ij <- w,
+// with FP64 sums of w^2, u^2, w u and of the columns of w.  CTAs walk row tiles with a grid
+// stride; part[(gx * tiles_r + ty)][0..2] = a, b, h partials, [3..3+G2_RT) = column sums.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_pass2_generic(const float* __restrict__ X, const float* __restrict__ theta, float* __restrict__ U,
+                const float* __restrict__ ybar, const float* __restrict__ p,
+                const float* __restrict__ alpha_s, const Ctl* __restrict__ ctl, int64_t n, int d,
+                int r, float alpha, double* __restrict__ part)
+{
+    if (ctl->stopped) return;
+    __shared__ __align__(16) float Xs[G2_TM][G2_DT + 1];
+    __shared__ __align__(16) float Ts[G2_DT][G2_RT];
+    __shared__ double sred[32];
+    __shared__ double scol[16][G2_RT];
+    const float cf = ctl->c_f;
+    const float two_alpha = 2.0f * alpha;
+    const int k0 = blockIdx.y * G2_RT;
+    const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+    const int64_t n_tiles = (n + G2_TM - 1) / G2_TM;
+    double sa = 0.0, sb = 0.0, sh = 0.0;
+    double csum[4] = {0.0, 0.0, 0.0, 0.0};
+    float pk[4], ask[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+        int k = k0 + tx * 4 + b;
+        pk[b] = (k < r) ? p[k] : 0.f;
+        ask[b] = (k < r) ? alpha_s[k] : 0.f;
+    }
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int64_t m0 = tile * G2_TM;
+        float acc[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+        for (int j0 = 0; j0 < d; j0 += G2_DT) {
+            for (int idx = threadIdx.x; idx < G2_TM * G2_DT; idx += 256) {
+                int m = idx / G2_DT, jj = idx % G2_DT;
+                int64_t row = m0 + m;
+                int col = j0 + jj;
+                Xs[m][jj] = (row < n && col < d) ? X[row * d + col] : 0.f;
+            }
+            for (int idx = threadIdx.x; idx < G2_DT * G2_RT; idx += 256) {
+                int jj = idx / G2_RT, kk = idx % G2_RT;
+                int j = j0 + jj, k = k0 + kk;
+                Ts[jj][kk] = (j < d && k < r) ? theta[(size_t)j * r + k] : 0.f;
+            }
+            __syncthreads();
+#pragma unroll 8
+            for (int jj = 0; jj < G2_DT; ++jj) {
+                const float4 tv = *reinterpret_cast<const float4*>(&Ts[jj][tx * 4]);
+                const float ta[4] = {tv.x, tv.y, tv.z, tv.w};
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    const float x = Xs[ty * 4 + a][jj];
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(x, ta[b], acc[a][b]);
+                }
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const int64_t row = m0 + ty * 4 + a;
+            if (row >= n) continue;
+            const float nay = -alpha * ybar[row];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int k = k0 + tx * 4 + b;
+                if (k >= r) continue;
+                const float u = cf * U[row * r + k];
+                float v = fmaf(two_alpha, acc[a][b], u);
+                v = fmaf(nay, pk[b], v);
+                v -= ask[b];
+                const float w = fmaxf(v, 0.f);
+                const double wd = (double)w, ud = (double)u;
+                sa = fma(wd, wd, sa);
+                sb = fma(ud, ud, sb);
+                sh = fma(wd, ud, sh);
+                csum[b] += wd;
+                U[row * r + k] = w;
+            }
+        }
+    }
+    sa = block_sum<256>(sa, sred);
+    sb = block_sum<256>(sb, sred);
+    sh = block_sum<256>(sh, sred);
+#pragma unroll
+    for (int b = 0; b < 4; ++b) scol[ty][tx * 4 + b] = csum[b];
+    __syncthreads();
+    double* out = part + ((size_t)blockIdx.x * gridDim.y + blockIdx.y) * (3 + G2_RT);
+    if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; out[2] = sh; }
+    if (threadIdx.x < G2_RT) {
+        double v = 0.0;
+        for (int y = 0; y < 16; ++y) v += scol[y][threadIdx.x];
+        out[3 + threadIdx.x] = v;
+    }
+}
+
+// Scalars after the second product (Algorithm 2, steps (d)-(e)): a, b, h, the multiplier,
+// the movement estimate, the dual gate, and p = U^T 1 of the new iterate as c * (column sums
+// of W).  nparts = gx * gy records of stride (3 + cols_per); column j lives in record
+// (gx, j / cols_per) at 3 + j % cols_per.
+__global__ void __launch_bounds__(256)
+k_fin2(Ctl* __restrict__ ctl, const double* __restrict__ part, int gx, int gy, int cols_per, int r,
+       int K, double eps_d, float* __restrict__ p)
+{
+    if (ctl->stopped) return;
+    __shared__ double sred[32];
+    __shared__ double sc;
+    __shared__ int sbad;
+    const int stride = 3 + cols_per;
+    const int nparts = gx * gy;
+    double a = 0.0, b = 0.0, h = 0.0;
+    for (int i = threadIdx.x; i < nparts; i += blockDim.x) {
+        a += part[(size_t)i * stride + 0];
+        b += part[(size_t)i * stride + 1];
+        h += part[(size_t)i * stride + 2];
+    }
+    a = block_sum<256>(a, sred);
+    b = block_sum<256>(b, sred);
+    h = block_sum<256>(h, sred);
+    if (threadIdx.x == 0) {
+        gem_nlr_iter_info rec;
+        rec.t = ctl->t;
+        rec.dual_applied = 0;
+        rec.stop = 0;
+        rec.status = GEM_NLR_OK;
+        rec.a = a; rec.b = b; rec.h = h;
+        rec.c = 0.0; rec.delta_hat = 0.0; rec.rho = 0.0;
+        rec.fhat = ctl->fhat_cur;
+        int bad = 0;
+        double c = 1.0;
+        if (!isfinite(a) || !isfinite(b) || !isfinite(h)) {
+            rec.status = GEM_NLR_E_NONFINITE; bad = 1;
+        } else {
+            const double nu = sqrt(a);
+            if (nu <= 1e-20) {
+                rec.status = GEM_NLR_E_BREAKDOWN; bad = 1;
+            } else {
+                const float cf = (float)(sqrt((double)K) / nu);
+                c = (double)cf;
+                double Delta = c * c * a + b - 2.0 * c * h;
+                if (Delta < 0.0) Delta = 0.0;
+                rec.c = c;
+                rec.delta_hat = sqrt(Delta) / sqrt((double)K);
+                rec.dual_applied = (Delta < eps_d * eps_d * (double)K) ? 1 : 0;
+                ctl->c_f = cf;
+                ctl->dual_pending = rec.dual_applied;
+                ctl->tail_pending = 1;
+                ctl->t = rec.t + 1;
+            }
+        }
+        if (bad) {
+            ctl->c_f = 1.0f;          // the buffer holds W as the paper's loop leaves it
+            ctl->stopped = 1;
+            ctl->status = rec.status;
+            ctl->dual_pending = 0;
+            ctl->tail_pending = 0;
+        }
+        ctl->last = rec;
+        sc = c;
+        sbad = bad;
+    }
+    __syncthreads();
+    if (sbad) return;
+    const double c = sc;
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+        const int yy = j / cols_per, jj = j % cols_per;
+        double v = 0.0;
+        for (int x = 0; x < gx; ++x) v += part[((size_t)x * gy + yy) * stride + 3 + jj];
+        p[j] = (float)(c * v);
+    }
+}
+
+// Row-argmax read-out: smallest index among maxima of c_f * U_i (c_f > 0 does not change it).
+__global__ void k_labels(const float* __restrict__ U, int64_t n, int r, int32_t* __restrict__ labels)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    if (r <= 32) {
+        // one thread per row
+        for (int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; row < n;
+             row += (int64_t)gridDim.x * blockDim.x) {
+            const float* u = U + row * r;
+            float bv = u[0];
+            int best = 0;
+            for (int j = 1; j < r; ++j) {
+                float v = u[j];
+                if (v > bv) { bv = v; best = j; }
+            }
+            labels[row] = best;
+        }
+        return;
+    }
+    for (int64_t row = warp; row < n; row += nwarps) {
+        const float* u = U + row * r;
+        float bv = -INFINITY;
+        int best = 0x7fffffff;
+        for (int j = lane; j < r; j += 32) {
+            float v = u[j];
+            if (v > bv) { bv = v; best = j; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            int ob = __shfl_xor_sync(0xffffffffu, best, o);
+            if (ov > bv || (ov == bv && ob < best)) { bv = ov; best = ob; }
+        }
+        if (lane == 0) labels[row] = best;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host-side launchers
+// ------------------------------------------------------------------------------------------
+static size_t rv_smem(int r) { return (size_t)RV_WARPS * r * sizeof(double); }
+
+static void set_rv_attr(int r)
+{
+    static int done_r = -1;
+    if (rv_smem(r) > 48 * 1024 && done_r < r) {
+        cudaFuncSetAttribute(k_rowvec<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rv_smem(r));
+        cudaFuncSetAttribute(k_rowvec<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rv_smem(r));
+        cudaFuncSetAttribute(k_colsum, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rv_smem(r));
+        done_r = r;
+    }
+}
+
+void launch_init_colsum(const Problem& pb)
+{
+    const auto& P = pb.P;
+    set_rv_attr(P.r);
+    k_colsum<<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(pb.U, pb.ctl(), P.n, P.r, pb.part1v());
+    k_fin_colsum<<<1, 256, 0, pb.stream>>>(pb.part1v(), pb.L.gv, P.r, pb.p());
+    pb.count(2);
+}
+
+void launch_vector_pass(const Problem& pb)
+{
+    const auto& P = pb.P;
+    set_rv_attr(P.r);
+    k_rowvec<false><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
+        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), 0);
+    pb.count();
+}
+
+void launch_fin1(const Problem& pb, int mode)
+{
+    const auto& P = pb.P;
+    k_fin1<<<1, 256, 0, pb.stream>>>(pb.ctl(), pb.part1v(), pb.L.gv, pb.red1(), pb.L.nred1, P.r, P.n,
+                                     P.alpha, pb.gamma, P.eps_c, P.T_min, pb.s(), pb.alpha_s(),
+                                     pb.hist(), mode);
+    pb.count();
+}
+
+void launch_fin2(const Problem& pb, int gx, int gy, int cols_per)
+{
+    const auto& P = pb.P;
+    k_fin2<<<1, 256, 0, pb.stream>>>(pb.ctl(), pb.part2(), gx, gy, cols_per, P.r, P.K, P.eps_d, pb.p());
+    pb.count();
+}
+
+void launch_generic_pass1(const Problem& pb, int ignore_stop)
+{
+    const auto& P = pb.P;
+    const auto& L = pb.L;
+    dim3 g1(L.g1x, L.g1y_d * L.g1y_r);
+    k_pass1_generic<<<g1, 256, 0, pb.stream>>>(pb.X, pb.U, pb.ctl(), P.n, P.d, P.r, L.g1y_r, pb.part1(),
+                                               ignore_stop);
+    k_red1<<<L.nred1, 256, 0, pb.stream>>>(pb.part1(), L.g1x, (int64_t)P.d * P.r, pb.ctl(), pb.theta(),
+                                            pb.red1(), ignore_stop);
+    pb.count(2);
+}
+
+void launch_generic_pass2_kernel(const Problem& pb)
+{
+    const auto& P = pb.P;
+    const auto& L = pb.L;
+    dim3 g2(L.g2x, L.g2y);
+    k_pass2_generic<<<g2, 256, 0, pb.stream>>>(pb.X, pb.theta(), pb.U, pb.ybar(), pb.p(), pb.alpha_s(),
+                                               pb.ctl(), P.n, P.d, P.r, P.alpha, pb.part2());
+    pb.count();
+}
+
+
+void launch_tail(const Problem& pb)
+{
+    const auto& P = pb.P;
+    set_rv_attr(P.r);
+    k_rowvec<true><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
+        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), 1);
+    pb.count();
+    launch_fin1(pb, 1);
+}
+
+void launch_objective(const Problem& pb)
+{
+    const auto& P = pb.P;
+    set_rv_attr(P.r);
+    // Called after the tail: no gate is pending and the multiplier is 1, so the vector pass has
+    // no side effect on the dual.  The objective is also wanted after a stop, so the stop flag
+    // is ignored.
+    k_rowvec<false><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
+        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), 1);
+    pb.count();
+    launch_generic_pass1(pb, 1);
+    launch_fin1(pb, 2);
+}
+
+void launch_labels(const Problem& pb, int32_t* labels)
+{
+    const auto& P = pb.P;
+    int blocks = (int)((P.n + 255) / 256);
+    if (P.r > 32) blocks = (int)((P.n + 7) / 8);
+    if (blocks > kSMs * 16) blocks = kSMs * 16;
+    if (blocks < 1) blocks = 1;
+    k_labels<<<blocks, 256, 0, pb.stream>>>(pb.U, P.n, P.r, labels);
+    pb.count();
+}
+
+}  // namespace gemnlr

@@ -1,0 +1,90 @@
+// Shared declarations of the NLR iteration library: the device-resident control block,
+// the workspace layout and the launch entry points of each kernel family.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/gem_nlr.h"
+
+namespace gemnlr {
+
+// Device-resident control block.  The gate, the pending multiplier and the stop flag never
+// leave the GPU between iterations; every iteration kernel reads them from here.
+struct Ctl {
+    float   c_f;            // pending multiplier: logical U = c_f * (contents of the U buffer)
+    int32_t t;              // iterations completed
+    int32_t dual_pending;   // gate of the last completed iteration fired, ytilde not yet updated
+    int32_t tail_pending;   // rho / stop test of the last completed iteration not yet evaluated
+    int32_t stopped;        // stop test fired or an error was raised: iteration kernels return at once
+    int32_t status;         // GEM_NLR_OK / GEM_NLR_CONVERGED / negative error
+    int32_t hist_cap;       // capacity of the history array (0: none)
+    int32_t hist_len;       // records written
+    double  fhat_cur;       // objective at the iterate the iteration in flight started from
+    double  theta2;         // ||Theta||_F^2 of the latest Theta
+    double  qq, yq;         // sum q_i^2, sum ytilde_i q_i of the latest vector pass
+    double  f_final;        // objective at the current iterate when the stop test fired
+    gem_nlr_iter_info last; // latest iteration (rho/stop filled in when its tail has run)
+    uint32_t counter[4];    // arrival counters for last-block reductions (always left at zero)
+};
+
+struct Layout {
+    size_t ctl, p, s, alpha_s, theta, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
+    int g1x, g1y_d, g1y_r;   // generic pass-1 grid: row chunks, d tiles, r tiles
+    int gv;                  // vector kernel CTAs
+    int g2x, g2y;            // generic pass-2 grid: row-tile CTAs, column tiles
+    int gs;                  // setup kernels' CTAs
+    int nred1;               // CTAs of the Theta reduction
+};
+
+constexpr int kSMs = 148;
+constexpr int G_TM = 64, G_DT = 64, G_RT = 64;       // generic pass-1 tile
+constexpr int G2_TM = 64, G2_RT = 64, G2_DT = 32;    // generic pass-2 tile
+
+Layout make_layout(const gem_nlr_params& P);
+
+struct Problem {
+    gem_nlr_params P;
+    float* X;        // X-hat once normalized
+    float* U;
+    char*  ws;
+    Layout L;
+    cudaStream_t stream;
+    float gamma_f;   // beta / n
+    double gamma;
+    int64_t* launches;       // host counter of kernel launches (owned by the handle)
+    void count(int k = 1) const { if (launches) *launches += k; }
+    Ctl* ctl() const { return reinterpret_cast<Ctl*>(ws + L.ctl); }
+    float* p() const { return reinterpret_cast<float*>(ws + L.p); }
+    float* s() const { return reinterpret_cast<float*>(ws + L.s); }
+    float* alpha_s() const { return reinterpret_cast<float*>(ws + L.alpha_s); }
+    float* theta() const { return reinterpret_cast<float*>(ws + L.theta); }
+    float* ytilde() const { return reinterpret_cast<float*>(ws + L.ytilde); }
+    float* ybar() const { return reinterpret_cast<float*>(ws + L.ybar); }
+    double* part1() const { return reinterpret_cast<double*>(ws + L.part1); }
+    double* part1v() const { return reinterpret_cast<double*>(ws + L.part1v); }
+    double* part2() const { return reinterpret_cast<double*>(ws + L.part2); }
+    double* red1() const { return reinterpret_cast<double*>(ws + L.red1); }
+    double* setup() const { return reinterpret_cast<double*>(ws + L.setup); }
+    gem_nlr_iter_info* hist() const { return reinterpret_cast<gem_nlr_iter_info*>(ws + L.hist); }
+};
+
+// ---- generic family (any n, d, r) -------------------------------------------------------
+// One iteration = vector pass, Theta partials, Theta reduction + scalars, fused second product,
+// statistics reduction + scalars.  tail: finish the last iteration (dual step, rho, stop) and
+// apply the pending multiplier to the U buffer.
+void launch_init_colsum(const Problem& pb);                 // p = U^T 1 for a freshly loaded U
+void launch_vector_pass(const Problem& pb);
+void launch_generic_pass1(const Problem& pb, int ignore_stop);
+void launch_fin1(const Problem& pb, int mode);
+void launch_generic_pass2_kernel(const Problem& pb);   // the fused second product alone
+void launch_fin2(const Problem& pb, int gx, int gy, int cols_per);
+void launch_tail(const Problem& pb);
+void launch_objective(const Problem& pb);                   // fills ctl->f_final for the current (U, y)
+void launch_labels(const Problem& pb, int32_t* labels);
+
+// ---- setup (Section 3) -------------------------------------------------------------------
+// Returns a negative GEM_NLR_E_* or 0; writes a to *a_out.  Synchronizes the stream.
+int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, double* a_out,
+                      double* host_scratch /* pinned, >= 4 doubles */);
+
+}  // namespace gemnlr
