@@ -49,6 +49,7 @@ extern "C" {
 #define GEM_NLR_E_BREAKDOWN  -4   /* sqrt(a) <= 1e-20: W vanished (Algorithm 1, breakdown line)   */
 #define GEM_NLR_E_NONFINITE  -5   /* a, b or h is not finite                                     */
 #define GEM_NLR_E_NOT_READY  -6   /* iteration requested before X was normalized                 */
+#define GEM_NLR_E_TIMEOUT    -7   /* a bounded device-side wait (copy pipeline) ran out          */
 
 typedef struct gem_nlr gem_nlr_t;   /* opaque handle */
 
@@ -70,6 +71,7 @@ typedef struct {
     double   pi_tol;        /* stop when |sigma_k - sigma_{k-1}| <= pi_tol * sigma_k (<=0: 1e-7) */
     uint64_t pi_seed;       /* seed of the starting vector                                       */
     int32_t  precision;     /* contraction arithmetic: 0 FP32 FFMA, 1 3xTF32 tensor cores,       */
+                            /* 2 the generic FFMA kernels whatever the shape (cross-checks),     */
                             /* -1 let the library choose by shape                                */
     int32_t  history;       /* 1: keep one gem_nlr_iter_info per iteration in the workspace      */
 } gem_nlr_params;

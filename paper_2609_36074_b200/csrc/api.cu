@@ -2,6 +2,7 @@
 // Every arithmetic step of the method runs in the kernels; this file only orders launches and
 // reads back the small control block.
 #include "nlr_common.cuh"
+#include "ffma_family.cuh"
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
@@ -19,7 +20,7 @@ static bool valid_params(const gem_nlr_params& P)
     if (P.r > 7168 || P.d > 2816) return false;       // shared-memory accumulators of the vector / setup passes
     if (!(P.alpha > 0.f) || !(P.beta > 0.f)) return false;
     if (P.T < 0 || P.T_min < 0 || P.eps_d < 0.0 || P.eps_c < 0.0) return false;
-    if (P.precision < -1 || P.precision > 1) return false;
+    if (P.precision < -1 || P.precision > 2) return false;
     return true;
 }
 
@@ -79,6 +80,8 @@ struct gem_nlr {
     Ctl* host_ctl;         // pinned read-back record
     double* host_scratch;  // pinned
     const char* path;
+    bool use_ffma;
+    FfmaPlan ffma;
     char err[256];
     int64_t launches;      // kernels launched by this handle
     int pi_iters;          // power iterations taken by the last setup
@@ -143,6 +146,13 @@ static void launch_iteration(gem_nlr_t* h)
     const bool prof = h->profile && h->ev_used + 3 <= h->ev_cap;
     cudaEvent_t* e = prof ? h->ev + h->ev_used : nullptr;
     if (prof) cudaEventRecord(e[0], h->pb.stream);
+    if (h->use_ffma) {
+        ffma_launch_first(h->pb, h->ffma, 0);
+        if (prof) cudaEventRecord(e[1], h->pb.stream);
+        ffma_launch_second(h->pb, h->ffma);
+        if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
+        return;
+    }
     launch_vector_pass(h->pb);
     launch_generic_pass1(h->pb, 0);
     launch_fin1(h->pb, 0);
@@ -215,6 +225,10 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     h->path = "generic";
     h->err[0] = 0;
     h->pb.launches = &h->launches;
+    if (params->precision <= 0 && ffma_plan(h->pb, &h->ffma)) {
+        h->use_ffma = true;
+        h->path = "ffma";
+    }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||
         cudaMallocHost((void**)&h->host_scratch, 64) != cudaSuccess) {
         if (h->host_ctl) cudaFreeHost(h->host_ctl);

@@ -1,0 +1,22 @@
+// Launch interface of the TMA-staged FP32-FFMA kernel family (kernels_ffma.cu).
+#pragma once
+#include <cuda.h>
+#include "nlr_common.cuh"
+
+namespace gemnlr {
+
+struct FfmaPlan {
+    alignas(64) CUtensorMap tm1;   // X-hat tiles of the first product
+    alignas(64) CUtensorMap tm2;   // X-hat tiles of the second product
+    int shape_id;
+    int g1, g2;                    // persistent grids
+};
+
+// True if (d, r, n) is covered by an instantiated shape and the tensor maps could be encoded.
+bool ffma_plan(const Problem& pb, FfmaPlan* plan);
+// Vector pass + Theta = X-hat^T U + reductions + the scalar step finishing the previous iteration.
+void ffma_launch_first(const Problem& pb, const FfmaPlan& plan, int mode);
+// Fused second product, statistics, scalar step (multiplier, movement, gate, p).
+void ffma_launch_second(const Problem& pb, const FfmaPlan& plan);
+
+}  // namespace gemnlr

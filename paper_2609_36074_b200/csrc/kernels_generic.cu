@@ -6,6 +6,7 @@
 // in a fixed order (FP64), so two runs on the same inputs give the same bits.
 #include "nlr_common.cuh"
 #include "device_utils.cuh"
+#include "fin_logic.cuh"
 
 namespace gemnlr {
 
@@ -236,32 +237,7 @@ k_fin1(Ctl* __restrict__ ctl, const double* __restrict__ part1v, int gv, const d
     qq = block_sum<256>(qq, sred);
     yq = block_sum<256>(yq, sred);
     t2 = block_sum<256>(t2, sred);
-    if (threadIdx.x == 0) {
-        ctl->qq = qq;
-        ctl->yq = yq;
-        if (mode != 1) ctl->theta2 = t2;
-        if (ctl->tail_pending) {
-            gem_nlr_iter_info rec = ctl->last;
-            rec.rho = sqrt(qq / (double)n);
-            rec.stop = (rec.dual_applied && rec.delta_hat < eps_c && rec.rho < eps_c &&
-                        rec.t + 1 >= T_min) ? 1 : 0;
-            ctl->last = rec;
-            if (ctl->hist_cap > 0 && rec.t < ctl->hist_cap) {
-                hist[rec.t] = rec;
-                ctl->hist_len = rec.t + 1;
-            }
-            ctl->tail_pending = 0;
-            ctl->dual_pending = 0;
-            if (rec.stop) { ctl->stopped = 1; ctl->status = GEM_NLR_CONVERGED; }
-        }
-        if (mode != 1) {
-            double f = -t2 + yq + 0.5 * gamma * qq;
-            if (mode == 0) ctl->fhat_cur = f;
-            if (mode == 2 || ctl->stopped) ctl->f_final = f;
-        } else {
-            ctl->c_f = 1.0f;
-        }
-    }
+    if (threadIdx.x == 0) fin1_scalars(ctl, qq, yq, t2, n, gamma, eps_c, T_min, hist, mode);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -391,46 +367,9 @@ k_fin2(Ctl* __restrict__ ctl, const double* __restrict__ part, int gx, int gy, i
     b = block_sum<256>(b, sred);
     h = block_sum<256>(h, sred);
     if (threadIdx.x == 0) {
-        gem_nlr_iter_info rec;
-        rec.t = ctl->t;
-        rec.dual_applied = 0;
-        rec.stop = 0;
-        rec.status = GEM_NLR_OK;
-        rec.a = a; rec.b = b; rec.h = h;
-        rec.c = 0.0; rec.delta_hat = 0.0; rec.rho = 0.0;
-        rec.fhat = ctl->fhat_cur;
-        int bad = 0;
-        double c = 1.0;
-        if (!isfinite(a) || !isfinite(b) || !isfinite(h)) {
-            rec.status = GEM_NLR_E_NONFINITE; bad = 1;
-        } else {
-            const double nu = sqrt(a);
-            if (nu <= 1e-20) {
-                rec.status = GEM_NLR_E_BREAKDOWN; bad = 1;
-            } else {
-                const float cf = (float)(sqrt((double)K) / nu);
-                c = (double)cf;
-                double Delta = c * c * a + b - 2.0 * c * h;
-                if (Delta < 0.0) Delta = 0.0;
-                rec.c = c;
-                rec.delta_hat = sqrt(Delta) / sqrt((double)K);
-                rec.dual_applied = (Delta < eps_d * eps_d * (double)K) ? 1 : 0;
-                ctl->c_f = cf;
-                ctl->dual_pending = rec.dual_applied;
-                ctl->tail_pending = 1;
-                ctl->t = rec.t + 1;
-            }
-        }
-        if (bad) {
-            ctl->c_f = 1.0f;          // the buffer holds W as the paper's loop leaves it
-            ctl->stopped = 1;
-            ctl->status = rec.status;
-            ctl->dual_pending = 0;
-            ctl->tail_pending = 0;
-        }
-        ctl->last = rec;
+        double c;
+        sbad = fin2_scalars(ctl, a, b, h, K, eps_d, &c) ? 0 : 1;
         sc = c;
-        sbad = bad;
     }
     __syncthreads();
     if (sbad) return;
