@@ -50,6 +50,7 @@ extern "C" {
 #define GEM_NLR_E_NONFINITE  -5   /* a, b or h is not finite                                     */
 #define GEM_NLR_E_NOT_READY  -6   /* iteration requested before X was normalized                 */
 #define GEM_NLR_E_TIMEOUT    -7   /* a bounded device-side wait (copy pipeline) ran out          */
+#define GEM_NLR_E_TOO_LARGE  -8   /* size beyond the fixed capacity of a *_static entry point    */
 
 typedef struct gem_nlr gem_nlr_t;   /* opaque handle */
 
@@ -173,6 +174,34 @@ int gem_nlr_run_host(const gem_nlr_params *params, const float *X_host, float *U
                      int32_t *labels_host, void *device_buffer_dev, size_t device_bytes,
                      void *cuda_stream, double *a_out, gem_nlr_iter_info *last,
                      int32_t *iters_done);
+
+/* Column sums without any allocation: p_dev[j] = sum_i U_dev[i * r + j], j < r (FP64 sums in a
+ * fixed order, rounded once to FP32) -- the p = U^T 1 of the iteration, for a factor the caller
+ * holds.  The paper has no counterpart of this entry point; it exists for callers that cannot
+ * allocate device memory at the time of the call: code living inside a host application that
+ * distributes all device memory at start-up and forbids cudaMalloc afterwards, latency-critical
+ * loops where an allocation's device-wide synchronization is not acceptable, or processes whose
+ * memory already belongs to a pool they do not control.  Such callers have no workspace to hand
+ * to gem_nlr_create either.
+ *
+ * U_dev: n x r row-major FP32 device memory (input, not modified).  p_dev: r floats of device
+ * memory (output).  Both are the caller's.  The scratch for the per-block partial sums is a
+ * fixed array inside the library (about 300 KB per GPU that loads the library, held until the
+ * process exits); this call never calls cudaMalloc, cudaFree or any allocating routine.
+ * Limit: r <= GEM_NLR_STATIC_MAX_R; a wider factor is refused with GEM_NLR_E_TOO_LARGE and
+ * nothing is launched.  n is not limited.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before any stream capture begins.  All calls share
+ * the one array and it keeps the previous call's partial sums: every call overwrites what it
+ * reads, so nothing needs clearing, but two calls whose kernels overlap on the GPU (different
+ * streams without an ordering between them) race on it -- order them.
+ * The work is enqueued on cuda_stream (a cudaStream_t; NULL = legacy default stream) and the
+ * call does not synchronize.  Returns GEM_NLR_OK, GEM_NLR_E_INVALID (NULL pointer, n < 1 or
+ * r < 1), GEM_NLR_E_TOO_LARGE, or GEM_NLR_E_CUDA.                                               */
+#define GEM_NLR_STATIC_MAX_R 128
+int gem_nlr_column_sums_static(const float *U_dev, int64_t n, int32_t r, float *p_dev,
+                               void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -14,5 +14,7 @@ from .binding import (  # noqa: F401
     workspace_bytes,
     paper_storage_bytes,
     host_job_device_bytes,
+    column_sums_static,
+    E_TIMEOUT, E_TOO_LARGE, STATIC_MAX_R,
     OK, CONVERGED, ITER_CAP, E_INVALID, E_CUDA, E_WORKSPACE, E_BREAKDOWN, E_NONFINITE, E_NOT_READY,
 )

@@ -9,6 +9,8 @@ _LIB_PATH = os.path.join(_HERE, "libgemnlr.so")
 
 OK, CONVERGED, ITER_CAP = 0, 1, 2
 E_INVALID, E_CUDA, E_WORKSPACE, E_BREAKDOWN, E_NONFINITE, E_NOT_READY = -1, -2, -3, -4, -5, -6
+E_TIMEOUT, E_TOO_LARGE = -7, -8
+STATIC_MAX_R = 128
 
 
 class Params(C.Structure):
@@ -77,6 +79,8 @@ def lib():
         L.gem_nlr_profile_read.restype = C.c_int
         L.gem_nlr_launch_count.argtypes = [vp]
         L.gem_nlr_launch_count.restype = C.c_int64
+        L.gem_nlr_column_sums_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp]
+        L.gem_nlr_column_sums_static.restype = C.c_int
         for name in ("create", "spectral_norm", "set_normalized", "step", "run", "labels", "objective",
                      "get_state", "set_state", "history", "buffer", "destroy", "run_host"):
             getattr(L, "gem_nlr_" + name).restype = C.c_int
@@ -240,3 +244,18 @@ def run_host(X_host, U_host, K, device_buffer, stream=None, want_labels=True, **
                                 device_buffer.data_ptr(), device_buffer.numel() * device_buffer.element_size(),
                                 st.cuda_stream, C.byref(a), C.byref(info), C.byref(iters))
     return rc, labels, a.value, info.as_dict(), iters.value
+
+
+def column_sums_static(U, out=None, stream=None):
+    """gem_nlr_column_sums_static: p = U^T 1 for a CUDA float32 matrix U, using only the scratch
+    array built into the library -- for callers that cannot allocate device memory when they call
+    (here `out` is allocated by torch only if the caller did not pass one).  Returns (rc, out);
+    rc is E_TOO_LARGE when U has more than STATIC_MAX_R columns.  Does not synchronize."""
+    import torch
+    assert U.is_cuda and U.dtype == torch.float32 and U.is_contiguous() and U.dim() == 2
+    n, r = U.shape
+    if out is None:
+        out = torch.empty(r, dtype=torch.float32, device=U.device)
+    st = stream if stream is not None else torch.cuda.current_stream(U.device)
+    rc = lib().gem_nlr_column_sums_static(U.data_ptr(), int(n), int(r), out.data_ptr(), st.cuda_stream)
+    return rc, out
