@@ -3,6 +3,7 @@
 // reads back the small control block.
 #include "nlr_common.cuh"
 #include "ffma_family.cuh"
+#include "tc_family.cuh"
 #include <math.h>
 #include <stdio.h>
 #include <string.h>
@@ -47,6 +48,7 @@ Layout make_layout(const gem_nlr_params& P)
     L.s = take(sizeof(float) * r);
     L.alpha_s = take(sizeof(float) * r);
     L.theta = take(sizeof(float) * (size_t)d * r);
+    L.thimg = take(sizeof(float) * 2 * (size_t)((d + 31) / 32 * 32) * ((r + 15) / 16 * 16));
     L.ytilde = take(sizeof(float) * (size_t)n);
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families
@@ -80,8 +82,10 @@ struct gem_nlr {
     Ctl* host_ctl;         // pinned read-back record
     double* host_scratch;  // pinned
     const char* path;
-    bool use_ffma;
+    bool use_ffma;         // first (and, unless use_tc, second) product by the FFMA family
+    bool use_tc;           // second product by the tcgen05 family
     FfmaPlan ffma;
+    TcPlan tc;
     char err[256];
     int64_t launches;      // kernels launched by this handle
     int pi_iters;          // power iterations taken by the last setup
@@ -148,15 +152,18 @@ static void launch_iteration(gem_nlr_t* h)
     if (prof) cudaEventRecord(e[0], h->pb.stream);
     if (h->use_ffma) {
         ffma_launch_first(h->pb, h->ffma, 0);
-        if (prof) cudaEventRecord(e[1], h->pb.stream);
-        ffma_launch_second(h->pb, h->ffma);
+    } else {
+        launch_vector_pass(h->pb);
+        launch_generic_pass1(h->pb, 0);
+        launch_fin1(h->pb, 0);
+    }
+    if (prof) cudaEventRecord(e[1], h->pb.stream);
+    if (h->use_tc || h->use_ffma) {
+        if (h->use_tc) tc_launch_second(h->pb, h->tc);
+        else ffma_launch_second(h->pb, h->ffma);
         if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
         return;
     }
-    launch_vector_pass(h->pb);
-    launch_generic_pass1(h->pb, 0);
-    launch_fin1(h->pb, 0);
-    if (prof) cudaEventRecord(e[1], h->pb.stream);
     launch_generic_pass2_kernel(h->pb);
     if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
     launch_fin2(h->pb, h->pb.L.g2x, h->pb.L.g2y, G2_RT);
@@ -225,9 +232,14 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     h->path = "generic";
     h->err[0] = 0;
     h->pb.launches = &h->launches;
-    if (params->precision <= 0 && ffma_plan(h->pb, &h->ffma)) {
+    if (params->precision != 2 && ffma_plan(h->pb, &h->ffma)) {
         h->use_ffma = true;
         h->path = "ffma";
+    }
+    if (params->precision == 1 &&
+        tc_plan(h->pb, &h->tc, reinterpret_cast<float*>((char*)workspace_dev + L.thimg))) {
+        h->use_tc = true;
+        h->path = h->use_ffma ? "ffma+tf32x3" : "generic+tf32x3";
     }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||
         cudaMallocHost((void**)&h->host_scratch, 64) != cudaSuccess) {

@@ -1,0 +1,385 @@
+// 3xTF32 tensor-core family (tcgen05 + TMEM): the fused second product of the iteration,
+//   acc = X-hat Theta ;  W = [U + 2 alpha acc - alpha (ybar p^T + 1 s^T)]_+ in place ;  FP64 a, b, h ;
+//   column sums of W,
+// for shapes where FP32 FFMA cannot keep up with HBM (d >= 64 with r >= 16).
+//
+// FP32 accuracy from TF32 tensor cores: each operand is split as x = hi + lo with hi exactly
+// representable in TF32, and the product is accumulated as hi*hi' + lo*hi' + hi*lo' (three MMAs
+// into the same TMEM accumulator); the dropped lo*lo' term is below 2^-22 relative.
+//
+// One persistent CTA per SM, ten warps:
+//   warp 0      producer: TMA loads of X-hat boxes (128 rows x 32 features, 128-byte swizzle = the
+//               K-major UMMA operand layout) and of U panels (128 rows x 32 columns); the pre-split
+//               Theta^T images are brought in once per CTA.
+//   warps 6-9   split: rewrite each box as hi (in place) and lo (second buffer).
+//   warp 1      MMA issuer: per box 4 k-steps x 3 tcgen05.mma (M = 128 rows, N = padded r);
+//               tcgen05.commit frees the stage and publishes the accumulator (two TMEM buffers).
+//   warps 2-5   epilogue: thread = row; tcgen05.ld of 32 columns at a time, entrywise update
+//               against the U panel in shared memory, FP64 statistics, W written back into the
+//               panel and stored with a TMA tile store; column sums by a transposed second sweep.
+// The last CTA reduces the per-CTA partials in CTA order and runs the scalar step.
+// Every mbarrier wait is bounded; on expiry the kernel flags GEM_NLR_E_TIMEOUT, stops waiting,
+// runs to its end and frees its TMEM.
+#include "nlr_common.cuh"
+#include "device_utils.cuh"
+#include "fin_logic.cuh"
+#include "pipeline.cuh"
+#include "tc_common.cuh"
+#include "tc_family.cuh"
+
+namespace gemnlr {
+namespace tc {
+
+constexpr int TILE_M = 128;
+constexpr int BOX_BYTES = TILE_M * 128;       // 128 rows x 32 floats
+constexpr int NTHREADS = 320;
+constexpr int MAX_RING = 8;
+
+// Theta (d x r, FP32 row-major) -> two images of Theta^T in the K-major 128-byte-swizzled UMMA
+// layout: box b (features 32b..32b+31) holds NP rows (columns of Theta, zero beyond r) of 128 bytes.
+__global__ void k_theta_images(const float* __restrict__ theta, int d, int r, int NP, const Ctl* __restrict__ ctl,
+                               float* __restrict__ img_hi, float* __restrict__ img_lo)
+{
+    if (ctl->stopped) return;
+    const int NB = d / 32;
+    const int total = NB * 32 * NP;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const int j = e / NP, k = e % NP;             // feature, column
+        const float v = (k < r) ? theta[(size_t)j * r + k] : 0.f;
+        const float hi = tf32_hi(v);
+        const int b = j >> 5, jj = j & 31, c = jj >> 2, w = jj & 3;
+        const size_t off = (size_t)b * NP * 32 + (size_t)k * 32 + (((c ^ (k & 7)) << 2) + w);
+        img_hi[off] = hi;
+        img_lo[off] = v - hi;
+    }
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU,
+           const float* __restrict__ img_hi, const float* __restrict__ img_lo,
+           const float* __restrict__ ybar, const float* __restrict__ p, const float* __restrict__ alpha_s,
+           Ctl* __restrict__ ctl, int64_t n, int d, int r, int NP, int NSB, int NUP, float alpha, int K,
+           double eps_d, double* __restrict__ part, float* __restrict__ p_out)
+{
+    if (ctl->stopped) return;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t bars[5 * MAX_RING + 5];
+    __shared__ uint32_t abort_flag;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ double sred[32];
+    __shared__ int is_last;
+    __shared__ double sc;
+    __shared__ int sok;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NB = d / 32;                         // boxes (k blocks) per tile
+    const int NPAN = (r + 31) / 32;                // 32-column panels of U per tile
+    const int ACC_COLS = NPAN * 32;                // TMEM columns per accumulator buffer
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * ACC_COLS) tmem_cols <<= 1;
+    const uint32_t th_bytes = (uint32_t)NB * NP * 128;
+
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t stage0 = smem_base;                                   // NSB x (hi, lo)
+    const uint32_t th_hi_s = stage0 + (uint32_t)NSB * 2 * BOX_BYTES;
+    const uint32_t th_lo_s = th_hi_s + th_bytes;
+    const uint32_t upan0 = th_lo_s + th_bytes;                           // NUP panels
+    float* sp = reinterpret_cast<float*>(smem + (size_t)NSB * 2 * BOX_BYTES + 2 * (size_t)th_bytes +
+                                         (size_t)NUP * BOX_BYTES);       // p, then alpha*s
+    float* sas = sp + ACC_COLS;
+
+    const uint32_t bar0 = smem_u32(bars);
+    auto xfull = [&](int s) { return bar0 + 8u * s; };
+    auto xsplit = [&](int s) { return bar0 + 8u * (MAX_RING + s); };
+    auto xfree = [&](int s) { return bar0 + 8u * (2 * MAX_RING + s); };
+    auto ufull = [&](int s) { return bar0 + 8u * (3 * MAX_RING + s); };
+    auto ufree = [&](int s) { return bar0 + 8u * (4 * MAX_RING + s); };
+    auto accfull = [&](int a) { return bar0 + 8u * (5 * MAX_RING + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (5 * MAX_RING + 2 + a); };
+    const uint32_t thfull = bar0 + 8u * (5 * MAX_RING + 4);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_RING; ++s) {
+            mbar_init(xfull(s), 1); mbar_init(xsplit(s), 4); mbar_init(xfree(s), 1);
+            mbar_init(ufull(s), 1); mbar_init(ufree(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4); }
+        mbar_init(thfull, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    for (int j = threadIdx.x; j < ACC_COLS; j += NTHREADS) {
+        sp[j] = (j < r) ? p[j] : 0.f;
+        sas[j] = (j < r) ? alpha_s[j] : 0.f;
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int64_t n_tiles = (n + TILE_M - 1) / TILE_M;
+    const float cf = ctl->c_f;
+    const float two_alpha = 2.0f * alpha;
+    double sa = 0.0, sb = 0.0, sh = 0.0;
+    double csum[8];                      // epilogue thread (col, quarter): running column sums, one per panel
+#pragma unroll
+    for (int i = 0; i < 8; ++i) csum[i] = 0.0;
+
+    if (warp == 0) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            mbar_expect_tx(thfull, 2 * th_bytes);
+            bulk_load_1d(th_hi_s, img_hi, th_bytes, thfull);
+            bulk_load_1d(th_lo_s, img_lo, th_bytes, thfull);
+            int i = 0;
+            for (int64_t t = blockIdx.x; t < n_tiles && !abort_flag; t += gridDim.x, ++i) {
+                const int row0 = (int)(t * TILE_M);
+                for (int b = 0; b < NB; ++b) {
+                    const int g = i * NB + b, s = g % NSB;
+                    if (g >= NSB) mbar_wait(xfree(s), ((g / NSB) - 1) & 1, &abort_flag, ctl);
+                    mbar_expect_tx(xfull(s), BOX_BYTES);
+                    tma_load_2d(stage0 + (uint32_t)s * 2 * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
+                }
+                for (int pn = 0; pn < NPAN; ++pn) {
+                    const int h = i * NPAN + pn, sl = h % NUP;
+                    if (h >= NUP) mbar_wait(ufree(sl), ((h / NUP) - 1) & 1, &abort_flag, ctl);
+                    mbar_expect_tx(ufull(sl), BOX_BYTES);
+                    tma_load_2d(upan0 + (uint32_t)sl * BOX_BYTES, &tmU, pn * 32, row0, ufull(sl));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_tf32(TILE_M, NP, 0, 0);
+            mbar_wait(thfull, 0, &abort_flag, ctl);
+            int i = 0;
+            for (int64_t t = blockIdx.x; t < n_tiles && !abort_flag; t += gridDim.x, ++i) {
+                const int a = i & 1;
+                if (i >= 2) mbar_wait(accfree(a), ((i >> 1) - 1) & 1, &abort_flag, ctl);
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(a * ACC_COLS);
+                for (int b = 0; b < NB; ++b) {
+                    const int g = i * NB + b, s = g % NSB;
+                    mbar_wait(xsplit(s), (g / NSB) & 1, &abort_flag, ctl);
+                    tc_fence_after();
+                    const uint32_t a_hi = stage0 + (uint32_t)s * 2 * BOX_BYTES, a_lo = a_hi + BOX_BYTES;
+                    const uint32_t b_hi = th_hi_s + (uint32_t)b * NP * 128, b_lo = th_lo_s + (uint32_t)b * NP * 128;
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t da_hi = umma_desc_sw128(a_hi + ks * 32, 16, 1024);
+                        const uint64_t da_lo = umma_desc_sw128(a_lo + ks * 32, 16, 1024);
+                        const uint64_t db_hi = umma_desc_sw128(b_hi + ks * 32, 16, 1024);
+                        const uint64_t db_lo = umma_desc_sw128(b_lo + ks * 32, 16, 1024);
+                        umma_tf32(tacc, da_hi, db_hi, idesc, (b | ks) ? 1u : 0u);
+                        umma_tf32(tacc, da_lo, db_hi, idesc, 1u);
+                        umma_tf32(tacc, da_hi, db_lo, idesc, 1u);
+                    }
+                    umma_commit(xfree(s));
+                }
+                umma_commit(accfull(a));
+            }
+        }
+    } else if (warp >= 6) {
+        // ------------------------------ split: box -> hi (in place), lo ------------------------------
+        const int st = threadIdx.x - 6 * 32;              // 0..127
+        int i = 0;
+        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
+            for (int b = 0; b < NB; ++b) {
+                const int g = i * NB + b, s = g % NSB;
+                mbar_wait(xfull(s), (g / NSB) & 1, &abort_flag, ctl);
+                const uint32_t hi_a = stage0 + (uint32_t)s * 2 * BOX_BYTES, lo_a = hi_a + BOX_BYTES;
+#pragma unroll
+                for (int k = 0; k < BOX_BYTES / 16 / 128; ++k) {
+                    const uint32_t off = (uint32_t)(k * 128 + st) * 16;
+                    const float4 x = lds128(hi_a + off);
+                    const float4 hi = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
+                    sts128(hi_a + off, hi);
+                    sts128(lo_a + off, make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w));
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(xsplit(s));
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (warps 2..5) ------------------------------
+        const int q = warp & 3;                           // TMEM lane quarter of this warp
+        const int rl = q * 32 + lane;                     // row of the tile owned by this thread
+        const int et = threadIdx.x - 2 * 32;              // 0..127 among the epilogue threads
+        const int cs_col = et & 31, cs_q = et >> 5;       // column-sum sweep: column, row quarter
+        int i = 0;
+        int stores_in_flight = 0, prev_slot = -1;
+        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
+            const int a = i & 1;
+            const int64_t row = t * TILE_M + rl;
+            const bool valid = row < n;
+            const float nay = valid ? -alpha * ybar[row] : 0.f;
+            mbar_wait(accfull(a), (i >> 1) & 1, &abort_flag, ctl);
+            tc_fence_after();
+            for (int pn = 0; pn < NPAN; ++pn) {
+                const int h = i * NPAN + pn, sl = h % NUP;
+                const uint32_t pan = upan0 + (uint32_t)sl * BOX_BYTES;
+                mbar_wait(ufull(sl), (h / NUP) & 1, &abort_flag, ctl);
+                float acc[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * ACC_COLS + pn * 32), acc);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t addr = pan + (uint32_t)rl * 128 + (uint32_t)((c ^ (rl & 7)) << 4);
+                    const float4 w4 = lds128(addr);
+                    const float wold[4] = {w4.x, w4.y, w4.z, w4.w};
+                    float wn[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int col = pn * 32 + 4 * c + e;
+                        const float u = cf * wold[e];
+                        float v = fmaf(two_alpha, acc[4 * c + e], u);
+                        v = fmaf(nay, sp[col], v);
+                        v -= sas[col];
+                        const float w = (valid && col < r) ? fmaxf(v, 0.f) : 0.f;
+                        const double wd = (double)w, ud = (valid && col < r) ? (double)u : 0.0;
+                        sa = fma(wd, wd, sa);
+                        sb = fma(ud, ud, sb);
+                        sh = fma(wd, ud, sh);
+                        wn[e] = w;
+                    }
+                    sts128(addr, make_float4(wn[0], wn[1], wn[2], wn[3]));
+                }
+                fence_proxy_async();
+                named_bar_sync(1, 128);
+                if (et == 0) {
+                    tma_store_2d(&tmU, pn * 32, (int)(t * TILE_M), pan);
+                    bulk_commit();
+                }
+                // column sums of this panel: thread (column, row quarter) adds 32 rows
+                {
+                    float cs = 0.f;
+#pragma unroll 8
+                    for (int rr = 0; rr < 32; ++rr) {
+                        const int row_l = cs_q * 32 + rr;
+                        const uint32_t addr = pan + (uint32_t)row_l * 128 +
+                                              (uint32_t)((((cs_col >> 2) ^ (row_l & 7)) << 4) + (cs_col & 3) * 4);
+                        float v;
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+                        cs += v;
+                    }
+                    csum[pn & 7] += (double)cs;
+                }
+                named_bar_sync(1, 128);
+                if (et == 0) {
+                    // the store issued one panel ago has finished reading its panel: release that slot
+                    if (prev_slot >= 0) { bulk_wait_read<1>(); mbar_arrive(ufree(prev_slot)); }
+                    prev_slot = sl;
+                    ++stores_in_flight;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(accfree(a));
+        }
+        if (et == 0) {
+            bulk_wait_read<0>();
+            if (prev_slot >= 0) mbar_arrive(ufree(prev_slot));
+            bulk_wait<0>();
+        }
+        (void)stores_in_flight;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
+
+    // ---- CTA partial: a, b, h and the column sums of W ----
+    const int PS = 4 + r;
+    sa = block_sum<NTHREADS>(sa, sred);
+    sb = block_sum<NTHREADS>(sb, sred);
+    sh = block_sum<NTHREADS>(sh, sred);
+    double* scol = reinterpret_cast<double*>(smem);        // [4 quarters][NPAN * 32]
+    if (warp >= 2 && warp < 6) {
+        const int et = threadIdx.x - 2 * 32;
+        for (int pn = 0; pn < NPAN; ++pn) scol[(size_t)(et >> 5) * ACC_COLS + pn * 32 + (et & 31)] = csum[pn & 7];
+    }
+    __syncthreads();
+    double* out = part + (size_t)blockIdx.x * PS;
+    if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; out[2] = sh; out[3] = 0.0; }
+    for (int j = threadIdx.x; j < r; j += NTHREADS)
+        out[4 + j] = ((scol[j] + scol[ACC_COLS + j]) + scol[2 * ACC_COLS + j]) + scol[3 * ACC_COLS + j];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned prev = atomicAdd(&ctl->counter[1], 1u);
+        is_last = (prev == gridDim.x - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int G = gridDim.x;
+    double a = 0.0, b = 0.0, hh = 0.0;
+    for (int i = threadIdx.x; i < G; i += NTHREADS) {
+        a += __ldcg(part + (size_t)i * PS + 0);
+        b += __ldcg(part + (size_t)i * PS + 1);
+        hh += __ldcg(part + (size_t)i * PS + 2);
+    }
+    a = block_sum<NTHREADS>(a, sred);
+    b = block_sum<NTHREADS>(b, sred);
+    hh = block_sum<NTHREADS>(hh, sred);
+    if (threadIdx.x == 0) {
+        double c;
+        sok = fin2_scalars(ctl, a, b, hh, K, eps_d, &c) ? 1 : 0;
+        sc = c;
+        ctl->counter[1] = 0;
+    }
+    __syncthreads();
+    if (!sok) return;
+    for (int j = threadIdx.x; j < r; j += NTHREADS) {
+        double v = 0.0;
+        for (int i = 0; i < G; ++i) v += __ldcg(part + (size_t)i * PS + 4 + j);
+        p_out[j] = (float)(sc * v);
+    }
+}
+
+}  // namespace tc
+
+bool tc_plan(const Problem& pb, TcPlan* pl, float* img_storage)
+{
+    const int d = pb.P.d, r = pb.P.r;
+    if (d % 32 != 0 || r % 4 != 0 || r < 8 || r > 256 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
+    const int NB = d / 32;
+    const int NP = (r + 15) / 16 * 16;
+    const int NPAN = (r + 31) / 32;
+    if (NPAN > 8) return false;
+    const size_t th = (size_t)NB * NP * 128;
+    const size_t fixed = 2 * th + (size_t)2 * NPAN * 32 * 4 + 1024;
+    // choose ring sizes under the 227 KB limit: at least 2 stages and 2 panels
+    const size_t limit = 227 * 1024 - 2048;
+    int NSB = 0, NUP = 0;
+    for (int nsb = 6; nsb >= 2 && !NSB; --nsb)
+        for (int nup = 4; nup >= 2; --nup)
+            if (fixed + (size_t)nsb * 2 * tc::BOX_BYTES + (size_t)nup * tc::BOX_BYTES <= limit) { NSB = nsb; NUP = nup; break; }
+    if (!NSB) return false;
+    pl->NP = NP; pl->NSB = NSB; pl->NUP = NUP;
+    pl->smem2 = fixed + (size_t)NSB * 2 * tc::BOX_BYTES + (size_t)NUP * tc::BOX_BYTES;
+    pl->img_hi = img_storage;
+    pl->img_lo = img_storage + (size_t)NB * 32 * NP;
+    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc::TILE_M, 32)) return false;
+    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tc::TILE_M, 32)) return false;
+    const int64_t tiles = (pb.P.n + tc::TILE_M - 1) / tc::TILE_M;
+    pl->g2 = (int)(tiles < kSMs ? tiles : kSMs);
+    if (cudaFuncSetAttribute(tc::k_pass2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
+        return false;
+    return true;
+}
+
+void tc_launch_second(const Problem& pb, const TcPlan& pl)
+{
+    const int d = pb.P.d, r = pb.P.r;
+    const int total = d * pl.NP;
+    tc::k_theta_images<<<(total + 255) / 256, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NP, pb.ctl(), pl.img_hi, pl.img_lo);
+    tc::k_pass2_tc<<<pl.g2, tc::NTHREADS, pl.smem2, pb.stream>>>(
+        pl.tmX, pl.tmU, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NP,
+        pl.NSB, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
+    pb.count(2);
+}
+
+}  // namespace gemnlr

@@ -28,7 +28,7 @@ struct Ctl {
 };
 
 struct Layout {
-    size_t ctl, p, s, alpha_s, theta, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
+    size_t ctl, p, s, alpha_s, theta, thimg, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
     int g1x, g1y_d, g1y_r;   // generic pass-1 grid: row chunks, d tiles, r tiles
     int gv;                  // vector kernel CTAs
     int g2x, g2y;            // generic pass-2 grid: row-tile CTAs, column tiles

@@ -1,0 +1,25 @@
+// Launch interface of the 3xTF32 tcgen05 kernel family (kernels_tc.cu).
+#pragma once
+#include <cuda.h>
+#include "nlr_common.cuh"
+
+namespace gemnlr {
+
+struct TcPlan {
+    alignas(64) CUtensorMap tmX;   // X-hat boxes: 128 rows x 32 features
+    alignas(64) CUtensorMap tmU;   // U panels: 128 rows x 32 columns (load and store)
+    int NP;                        // r padded to a multiple of 16 (MMA N)
+    int NSB, NUP;                  // stage ring / panel ring sizes
+    int g2;                        // persistent grid
+    size_t smem2;
+    float* img_hi;                 // pre-split Theta^T images in the workspace
+    float* img_lo;
+};
+
+// True if the shape is covered (d a multiple of 32, r a multiple of 4 in [8, 256], Theta images
+// fit in shared memory) and the tensor maps could be encoded.  img_storage: 2 * d * NP floats.
+bool tc_plan(const Problem& pb, TcPlan* plan, float* img_storage);
+// Theta image build + fused second product, statistics, scalar step.
+void tc_launch_second(const Problem& pb, const TcPlan& plan);
+
+}  // namespace gemnlr

@@ -1,0 +1,56 @@
+"""GPU parity of the tcgen05 3xTF32 family (second product) against the CPU oracle."""
+import numpy as np
+import pytest
+
+import oracle
+import synth
+import paper_2609_36074_b200 as gem
+from gpu_helpers import make_solver, rel, teacher_forced_steps, u_err
+
+pytestmark = pytest.mark.gpu
+TOL_U, TOL_F = 1e-4, 1e-5
+
+
+def _problem(n, d, K, seed=0):
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, seed)
+    X, lab, _ = synth.make_mixture(spec)
+    Xhat, _, _ = oracle.normalize(X)
+    return Xhat, synth.make_u0(n, K, K, seed=seed)
+
+
+# (n, d, r): one and several U panels, ragged last tile, more tiles than CTAs, r not a multiple of 16 or 32
+TC_SHAPES = [(4000, 128, 16), (3001, 64, 100), (2500, 64, 16), (40003, 128, 16), (20011, 64, 100),
+             (3000, 32, 8), (5000, 96, 36)]
+
+
+@pytest.mark.parametrize("n,d,K", TC_SHAPES)
+def test_tc_second_product_teacher_forced(n, d, K):
+    Xhat, U0 = _problem(n, d, K)
+    hp = synth.default_hparams(K)
+    s = make_solver(Xhat, U0, K, hp, precision=1)
+    assert s.path().endswith("tf32x3"), s.path()
+    s.destroy()
+    recs = teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U, solver_kw=dict(precision=1))
+    for rec in recs:
+        assert rec["a"] <= 1e-6 and rec["b"] <= 1e-6 and rec["h"] <= 1e-6, rec
+        assert rec["c"] <= 2e-7 and rec["delta"] <= 1e-6, rec
+        assert rec["rho"] <= 1e-5 and rec["fhat"] <= TOL_F, rec
+        assert rec["dual"][0] == rec["dual"][1] and rec["stop"][0] == rec["stop"][1], rec
+
+
+@pytest.mark.parametrize("n,d,K", [(9000, 128, 16), (6000, 64, 100)])
+def test_tc_trajectory_matches_oracle_and_is_reproducible(n, d, K):
+    Xhat, U0 = _problem(n, d, K)
+    hp = dict(synth.default_hparams(K), eps_d=0.2)
+    T = 30
+    outs = []
+    for _ in range(2):
+        s = make_solver(Xhat, U0, K, hp, T=T, precision=1)
+        rc, info, iters = s.run()
+        assert rc == gem.ITER_CAP and iters == T, (rc, s.last_error())
+        outs.append((s.U.cpu().numpy().copy(), info))
+        s.destroy()
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    Uo, _, infoo, _, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, hp["T_min"])
+    assert u_err(outs[0][0], Uo) <= TOL_U
+    assert rel(outs[0][1]["rho"], infoo["rho"]) <= 1e-4
