@@ -7,14 +7,15 @@
 // representable in TF32, and the product is accumulated as hi*hi' + lo*hi' + hi*lo' (three MMAs
 // into the same TMEM accumulator); the dropped lo*lo' term is below 2^-22 relative.
 //
-// One persistent CTA per SM, ten warps:
+// One persistent CTA per SM, 22 warps:
 //   warp 0      producer: TMA loads of X-hat boxes (128 rows x 32 features, 128-byte swizzle = the
 //               K-major UMMA operand layout) and of U panels (128 rows x 32 columns); the pre-split
 //               Theta^T images are brought in once per CTA.
-//   warps 6-9   split: rewrite each box as hi (in place) and lo (second buffer).
+//   warps 18-21 split: rewrite each box as hi (in place) and lo (second buffer).
 //   warp 1      MMA issuer: per box 4 k-steps x 3 tcgen05.mma (M = 128 rows, N = padded r);
 //               tcgen05.commit frees the stage and publishes the accumulator (two TMEM buffers).
-//   warps 2-5   epilogue: thread = row; tcgen05.ld of 32 columns at a time, entrywise update
+//   warps 2-17  epilogue, four groups taking the panels of a tile round-robin: thread = row;
+//               tcgen05.ld of 16 columns at a time, entrywise update
 //               against the U panel in shared memory, FP64 statistics, W written back into the
 //               panel and stored with a TMA tile store; column sums by a transposed second sweep.
 // The last CTA reduces the per-CTA partials in CTA order and runs the scalar step.
@@ -32,7 +33,9 @@ namespace tc {
 
 constexpr int TILE_M = 128;
 constexpr int BOX_BYTES = TILE_M * 128;       // 128 rows x 32 floats
-constexpr int NTHREADS = 320;
+constexpr int NGROUPS = 4;               // epilogue warp groups; group g owns panels pn = g (mod 4)
+constexpr int NTHREADS = (2 + 4 * NGROUPS + 4) * 32;   // producer, MMA, 16 epilogue, 4 split warps
+constexpr int GROUP_THREADS = 128;
 constexpr int MAX_RING = 8;
 
 // Theta (d x r, FP32 row-major) -> two images of Theta^T in the K-major 128-byte-swizzled UMMA
@@ -58,13 +61,13 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU,
            const float* __restrict__ img_hi, const float* __restrict__ img_lo,
            const float* __restrict__ ybar, const float* __restrict__ p, const float* __restrict__ alpha_s,
-           Ctl* __restrict__ ctl, int64_t n, int d, int r, int NP, int NSB, int NUP, float alpha, int K,
+           Ctl* __restrict__ ctl, int64_t n, int d, int r, int NP, int PW, int NSB, int NLO, int NUP, float alpha, int K,
            double eps_d, double* __restrict__ part, float* __restrict__ p_out)
 {
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[5 * MAX_RING + 5];
+    __shared__ __align__(8) uint64_t bars[6 * MAX_RING + 5];
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t tmem_base_s;
     __shared__ double sred[32];
@@ -74,19 +77,22 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NB = d / 32;                         // boxes (k blocks) per tile
-    const int NPAN = (r + 31) / 32;                // 32-column panels of U per tile
-    const int ACC_COLS = NPAN * 32;                // TMEM columns per accumulator buffer
+    const int NPAN = (r + PW - 1) / PW;            // PW-column panels of U per tile (PW = 16 or 32)
+    const int ACC_COLS = (NPAN * PW + 31) / 32 * 32;   // TMEM columns per accumulator buffer
+    const int PAN_BYTES = TILE_M * PW * 4;
+    const int CS_ROWS = PW / 2;                    // rows per thread in the column-sum sweep
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * ACC_COLS) tmem_cols <<= 1;
     const uint32_t th_bytes = (uint32_t)NB * NP * 128;
 
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t stage0 = smem_base;                                   // NSB x (hi, lo)
-    const uint32_t th_hi_s = stage0 + (uint32_t)NSB * 2 * BOX_BYTES;
+    const uint32_t stage0 = smem_base;                                   // NSB boxes: raw, then hi in place
+    const uint32_t lo0 = stage0 + (uint32_t)NSB * BOX_BYTES;             // NLO boxes: lo parts
+    const uint32_t th_hi_s = lo0 + (uint32_t)NLO * BOX_BYTES;
     const uint32_t th_lo_s = th_hi_s + th_bytes;
     const uint32_t upan0 = th_lo_s + th_bytes;                           // NUP panels
-    float* sp = reinterpret_cast<float*>(smem + (size_t)NSB * 2 * BOX_BYTES + 2 * (size_t)th_bytes +
-                                         (size_t)NUP * BOX_BYTES);       // p, then alpha*s
+    float* sp = reinterpret_cast<float*>(smem + (size_t)(NSB + NLO) * BOX_BYTES + (size_t)NUP * PAN_BYTES +
+                                         2 * (size_t)th_bytes);          // p, then alpha*s
     float* sas = sp + ACC_COLS;
 
     const uint32_t bar0 = smem_u32(bars);
@@ -95,16 +101,17 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     auto xfree = [&](int s) { return bar0 + 8u * (2 * MAX_RING + s); };
     auto ufull = [&](int s) { return bar0 + 8u * (3 * MAX_RING + s); };
     auto ufree = [&](int s) { return bar0 + 8u * (4 * MAX_RING + s); };
-    auto accfull = [&](int a) { return bar0 + 8u * (5 * MAX_RING + a); };
-    auto accfree = [&](int a) { return bar0 + 8u * (5 * MAX_RING + 2 + a); };
-    const uint32_t thfull = bar0 + 8u * (5 * MAX_RING + 4);
+    auto lofree = [&](int s) { return bar0 + 8u * (5 * MAX_RING + s); };
+    auto accfull = [&](int a) { return bar0 + 8u * (6 * MAX_RING + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (6 * MAX_RING + 2 + a); };
+    const uint32_t thfull = bar0 + 8u * (6 * MAX_RING + 4);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_RING; ++s) {
             mbar_init(xfull(s), 1); mbar_init(xsplit(s), 4); mbar_init(xfree(s), 1);
-            mbar_init(ufull(s), 1); mbar_init(ufree(s), 1);
+            mbar_init(ufull(s), 1); mbar_init(ufree(s), 1); mbar_init(lofree(s), 1);
         }
-        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4 * NGROUPS); }
         mbar_init(thfull, 1);
         abort_flag = 0;
         fence_barrier_init();
@@ -140,13 +147,13 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     const int g = i * NB + b, s = g % NSB;
                     if (g >= NSB) mbar_wait(xfree(s), ((g / NSB) - 1) & 1, &abort_flag, ctl);
                     mbar_expect_tx(xfull(s), BOX_BYTES);
-                    tma_load_2d(stage0 + (uint32_t)s * 2 * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
+                    tma_load_2d(stage0 + (uint32_t)s * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
                 }
                 for (int pn = 0; pn < NPAN; ++pn) {
                     const int h = i * NPAN + pn, sl = h % NUP;
                     if (h >= NUP) mbar_wait(ufree(sl), ((h / NUP) - 1) & 1, &abort_flag, ctl);
-                    mbar_expect_tx(ufull(sl), BOX_BYTES);
-                    tma_load_2d(upan0 + (uint32_t)sl * BOX_BYTES, &tmU, pn * 32, row0, ufull(sl));
+                    mbar_expect_tx(ufull(sl), PAN_BYTES);
+                    tma_load_2d(upan0 + (uint32_t)sl * PAN_BYTES, &tmU, pn * PW, row0, ufull(sl));
                 }
             }
         }
@@ -162,10 +169,10 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * ACC_COLS);
                 for (int b = 0; b < NB; ++b) {
-                    const int g = i * NB + b, s = g % NSB;
+                    const int g = i * NB + b, s = g % NSB, l = g % NLO;
                     mbar_wait(xsplit(s), (g / NSB) & 1, &abort_flag, ctl);
                     tc_fence_after();
-                    const uint32_t a_hi = stage0 + (uint32_t)s * 2 * BOX_BYTES, a_lo = a_hi + BOX_BYTES;
+                    const uint32_t a_hi = stage0 + (uint32_t)s * BOX_BYTES, a_lo = lo0 + (uint32_t)l * BOX_BYTES;
                     const uint32_t b_hi = th_hi_s + (uint32_t)b * NP * 128, b_lo = th_lo_s + (uint32_t)b * NP * 128;
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
@@ -178,23 +185,29 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                         umma_tf32(tacc, da_hi, db_lo, idesc, 1u);
                     }
                     umma_commit(xfree(s));
+                    umma_commit(lofree(l));
                 }
                 umma_commit(accfull(a));
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= 2 + 4 * NGROUPS) {
         // ------------------------------ split: box -> hi (in place), lo ------------------------------
-        const int st = threadIdx.x - 6 * 32;              // 0..127
+        const int st = threadIdx.x - (2 + 4 * NGROUPS) * 32;   // 0..127
         int i = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
             for (int b = 0; b < NB; ++b) {
-                const int g = i * NB + b, s = g % NSB;
+                const int g = i * NB + b, s = g % NSB, l = g % NLO;
                 mbar_wait(xfull(s), (g / NSB) & 1, &abort_flag, ctl);
-                const uint32_t hi_a = stage0 + (uint32_t)s * 2 * BOX_BYTES, lo_a = hi_a + BOX_BYTES;
+                if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+                const uint32_t hi_a = stage0 + (uint32_t)s * BOX_BYTES, lo_a = lo0 + (uint32_t)l * BOX_BYTES;
+#pragma unroll
+                float4 xin[BOX_BYTES / 16 / 128];
+#pragma unroll
+                for (int k = 0; k < BOX_BYTES / 16 / 128; ++k) xin[k] = lds128(hi_a + (uint32_t)(k * 128 + st) * 16);
 #pragma unroll
                 for (int k = 0; k < BOX_BYTES / 16 / 128; ++k) {
                     const uint32_t off = (uint32_t)(k * 128 + st) * 16;
-                    const float4 x = lds128(hi_a + off);
+                    const float4 x = xin[k];
                     const float4 hi = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
                     sts128(hi_a + off, hi);
                     sts128(lo_a + off, make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w));
@@ -205,13 +218,19 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             }
         }
     } else {
-        // ------------------------------ epilogue (warps 2..5) ------------------------------
+        // ------------------------------ epilogue (warps 2..17) ------------------------------
+        // Four groups of four warps (one warp per TMEM lane quarter).  Group g processes the panels
+        // pn = g, g + 4, ... of every tile, so the panels of a tile are in flight concurrently and
+        // their latency chains (panel wait, TMEM load, FP64 chains, store hand-off) overlap.
+        // Thread = one row of the tile, all PW columns of the panel, 16 at a time.
+        // Panel layout: PW = 32: 128-byte rows, 128-byte swizzle; PW = 16: plain 64-byte rows.
         const int q = warp & 3;                           // TMEM lane quarter of this warp
+        const int grp = (warp - 2) >> 2;                  // epilogue group
         const int rl = q * 32 + lane;                     // row of the tile owned by this thread
-        const int et = threadIdx.x - 2 * 32;              // 0..127 among the epilogue threads
-        const int cs_col = et & 31, cs_q = et >> 5;       // column-sum sweep: column, row quarter
+        const int gt = (q * 32 + lane);                   // 0..127 inside the group (any bijection works)
+        const int cs_col = gt % PW, cs_o = gt / PW;       // column-sum sweep: column, row group
+        const int CS_ROWS_G = TILE_M / (GROUP_THREADS / PW);
         int i = 0;
-        int stores_in_flight = 0, prev_slot = -1;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
             const int a = i & 1;
             const int64_t row = t * TILE_M + rl;
@@ -219,72 +238,77 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             const float nay = valid ? -alpha * ybar[row] : 0.f;
             mbar_wait(accfull(a), (i >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
-            for (int pn = 0; pn < NPAN; ++pn) {
+#pragma unroll 1
+            for (int pn = grp; pn < NPAN; pn += NGROUPS) {
                 const int h = i * NPAN + pn, sl = h % NUP;
-                const uint32_t pan = upan0 + (uint32_t)sl * BOX_BYTES;
+                const uint32_t pan = upan0 + (uint32_t)sl * PAN_BYTES;
                 mbar_wait(ufull(sl), (h / NUP) & 1, &abort_flag, ctl);
-                float acc[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * ACC_COLS + pn * 32), acc);
+#pragma unroll 1
+                for (int hf = 0; hf < PW / 16; ++hf) {
+                    float acc[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * ACC_COLS + pn * PW + hf * 16), acc);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t addr = pan + (uint32_t)rl * 128 + (uint32_t)((c ^ (rl & 7)) << 4);
-                    const float4 w4 = lds128(addr);
-                    const float wold[4] = {w4.x, w4.y, w4.z, w4.w};
-                    float wn[4];
+                    for (int cc = 0; cc < 4; ++cc) {
+                        const int c = hf * 4 + cc;
+                        const int col0 = pn * PW + 4 * c;
+                        const uint32_t addr = (PW == 32) ? pan + (uint32_t)rl * 128 + (uint32_t)((c ^ (rl & 7)) << 4)
+                                                         : pan + (uint32_t)rl * 64 + (uint32_t)(c << 4);
+                        const float4 w4 = lds128(addr);
+                        const float4 p4 = *reinterpret_cast<const float4*>(sp + col0);
+                        const float4 s4 = *reinterpret_cast<const float4*>(sas + col0);
+                        const float wold[4] = {w4.x, w4.y, w4.z, w4.w};
+                        const float pj[4] = {p4.x, p4.y, p4.z, p4.w};
+                        const float sj[4] = {s4.x, s4.y, s4.z, s4.w};
+                        float wn[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int col = pn * 32 + 4 * c + e;
-                        const float u = cf * wold[e];
-                        float v = fmaf(two_alpha, acc[4 * c + e], u);
-                        v = fmaf(nay, sp[col], v);
-                        v -= sas[col];
-                        const float w = (valid && col < r) ? fmaxf(v, 0.f) : 0.f;
-                        const double wd = (double)w, ud = (valid && col < r) ? (double)u : 0.0;
-                        sa = fma(wd, wd, sa);
-                        sb = fma(ud, ud, sb);
-                        sh = fma(wd, ud, sh);
-                        wn[e] = w;
+                        for (int e = 0; e < 4; ++e) {
+                            const bool live = valid && (col0 + e < r);
+                            const float u = live ? cf * wold[e] : 0.f;
+                            float v = fmaf(two_alpha, acc[4 * cc + e], u);
+                            v = fmaf(nay, pj[e], v);
+                            v -= sj[e];
+                            const float w = live ? fmaxf(v, 0.f) : 0.f;
+                            const double wd = (double)w, ud = (double)u;
+                            sa = fma(wd, wd, sa);
+                            sb = fma(ud, ud, sb);
+                            sh = fma(wd, ud, sh);
+                            wn[e] = w;
+                        }
+                        sts128(addr, make_float4(wn[0], wn[1], wn[2], wn[3]));
                     }
-                    sts128(addr, make_float4(wn[0], wn[1], wn[2], wn[3]));
                 }
                 fence_proxy_async();
-                named_bar_sync(1, 128);
-                if (et == 0) {
-                    tma_store_2d(&tmU, pn * 32, (int)(t * TILE_M), pan);
+                named_bar_sync(1 + grp, GROUP_THREADS);
+                if (gt == 0) {
+                    tma_store_2d(&tmU, pn * PW, (int)(t * TILE_M), pan);
                     bulk_commit();
                 }
-                // column sums of this panel: thread (column, row quarter) adds 32 rows
+                // column sums of this panel: thread (column, row group) adds its rows
                 {
                     float cs = 0.f;
 #pragma unroll 8
-                    for (int rr = 0; rr < 32; ++rr) {
-                        const int row_l = cs_q * 32 + rr;
-                        const uint32_t addr = pan + (uint32_t)row_l * 128 +
-                                              (uint32_t)((((cs_col >> 2) ^ (row_l & 7)) << 4) + (cs_col & 3) * 4);
+                    for (int rr = 0; rr < CS_ROWS_G; ++rr) {
+                        const int row_l = cs_o * CS_ROWS_G + rr;
+                        const uint32_t addr = (PW == 32)
+                            ? pan + (uint32_t)row_l * 128 + (uint32_t)((((cs_col >> 2) ^ (row_l & 7)) << 4) + (cs_col & 3) * 4)
+                            : pan + (uint32_t)row_l * 64 + (uint32_t)(cs_col * 4);
                         float v;
                         asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
                         cs += v;
                     }
-                    csum[pn & 7] += (double)cs;
+                    csum[(pn / NGROUPS) & 7] += (double)cs;
                 }
-                named_bar_sync(1, 128);
-                if (et == 0) {
-                    // the store issued one panel ago has finished reading its panel: release that slot
-                    if (prev_slot >= 0) { bulk_wait_read<1>(); mbar_arrive(ufree(prev_slot)); }
-                    prev_slot = sl;
-                    ++stores_in_flight;
-                }
+                // the store has read the panel (its wait overlapped the sweep above) and every thread of
+                // the group is done with it: hand the slot back to the producer
+                if (gt == 0) bulk_wait_read<0>();
+                named_bar_sync(1 + grp, GROUP_THREADS);
+                if (gt == 0) mbar_arrive(ufree(sl));
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(accfree(a));
         }
-        if (et == 0) {
-            bulk_wait_read<0>();
-            if (prev_slot >= 0) mbar_arrive(ufree(prev_slot));
-            bulk_wait<0>();
-        }
-        (void)stores_in_flight;
+        if (gt == 0) bulk_wait<0>();
     }
     tc_fence_before();
     __syncthreads();
@@ -295,16 +319,20 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     sa = block_sum<NTHREADS>(sa, sred);
     sb = block_sum<NTHREADS>(sb, sred);
     sh = block_sum<NTHREADS>(sh, sred);
-    double* scol = reinterpret_cast<double*>(smem);        // [4 quarters][NPAN * 32]
-    if (warp >= 2 && warp < 6) {
-        const int et = threadIdx.x - 2 * 32;
-        for (int pn = 0; pn < NPAN; ++pn) scol[(size_t)(et >> 5) * ACC_COLS + pn * 32 + (et & 31)] = csum[pn & 7];
+    double* scol = reinterpret_cast<double*>(smem);        // [128 / PW row groups][ACC_COLS]
+    if (warp >= 2 && warp < 2 + 4 * NGROUPS) {
+        const int grp = (warp - 2) >> 2, gt = (warp & 3) * 32 + lane;
+        for (int pn = grp; pn < NPAN; pn += NGROUPS)
+            scol[(size_t)(gt / PW) * ACC_COLS + pn * PW + (gt % PW)] = csum[(pn / NGROUPS) & 7];
     }
     __syncthreads();
     double* out = part + (size_t)blockIdx.x * PS;
     if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; out[2] = sh; out[3] = 0.0; }
-    for (int j = threadIdx.x; j < r; j += NTHREADS)
-        out[4 + j] = ((scol[j] + scol[ACC_COLS + j]) + scol[2 * ACC_COLS + j]) + scol[3 * ACC_COLS + j];
+    for (int j = threadIdx.x; j < r; j += NTHREADS) {
+        double v = 0.0;
+        for (int o = 0; o < GROUP_THREADS / PW; ++o) v += scol[(size_t)o * ACC_COLS + j];
+        out[4 + j] = v;
+    }
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -347,23 +375,32 @@ bool tc_plan(const Problem& pb, TcPlan* pl, float* img_storage)
     if (d % 32 != 0 || r % 4 != 0 || r < 8 || r > 256 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
     const int NB = d / 32;
     const int NP = (r + 15) / 16 * 16;
-    const int NPAN = (r + 31) / 32;
+    const int PW = (r <= 16) ? 16 : 32;
+    const int NPAN = (r + PW - 1) / PW;
     if (NPAN > 8) return false;
+    const int ACC_COLS = (NPAN * PW + 31) / 32 * 32;
+    const size_t pan_bytes = (size_t)tc::TILE_M * PW * 4;
     const size_t th = (size_t)NB * NP * 128;
-    const size_t fixed = 2 * th + (size_t)2 * NPAN * 32 * 4 + 1024;
-    // choose ring sizes under the 227 KB limit: at least 2 stages and 2 panels
+    const size_t fixed = 2 * th + (size_t)2 * ACC_COLS * 4 + 1024;
     const size_t limit = 227 * 1024 - 2048;
-    int NSB = 0, NUP = 0;
-    for (int nsb = 6; nsb >= 2 && !NSB; --nsb)
-        for (int nup = 4; nup >= 2; --nup)
-            if (fixed + (size_t)nsb * 2 * tc::BOX_BYTES + (size_t)nup * tc::BOX_BYTES <= limit) { NSB = nsb; NUP = nup; break; }
+    // Ring sizes under the 227 KB limit.  The U panel ring comes first (a slot is released one
+    // panel after its store was issued, so fewer than 4 slots serialises the panel loads); then
+    // the lo boxes (split -> MMA -> free round trip); the raw X-hat box ring takes what is left
+    // and sets how far the TMA loads run ahead.
+    int NSB = 0, NUP = 0, NLO = 0;
+    for (int nup = 4; nup >= 2 && !NSB; --nup)
+        for (int nlo = 3; nlo >= 2 && !NSB; --nlo)
+            for (int nsb = tc::MAX_RING; nsb >= (nlo == 3 ? 4 : 2); --nsb)
+                if (fixed + (size_t)(nsb + nlo) * tc::BOX_BYTES + (size_t)nup * pan_bytes <= limit) {
+                    NSB = nsb; NUP = nup; NLO = nlo; break;
+                }
     if (!NSB) return false;
-    pl->NP = NP; pl->NSB = NSB; pl->NUP = NUP;
-    pl->smem2 = fixed + (size_t)NSB * 2 * tc::BOX_BYTES + (size_t)NUP * tc::BOX_BYTES;
+    pl->NP = NP; pl->PW = PW; pl->NSB = NSB; pl->NLO = NLO; pl->NUP = NUP;
+    pl->smem2 = fixed + (size_t)(NSB + NLO) * tc::BOX_BYTES + (size_t)NUP * pan_bytes;
     pl->img_hi = img_storage;
     pl->img_lo = img_storage + (size_t)NB * 32 * NP;
     if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc::TILE_M, 32)) return false;
-    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tc::TILE_M, 32)) return false;
+    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tc::TILE_M, PW)) return false;
     const int64_t tiles = (pb.P.n + tc::TILE_M - 1) / tc::TILE_M;
     pl->g2 = (int)(tiles < kSMs ? tiles : kSMs);
     if (cudaFuncSetAttribute(tc::k_pass2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
@@ -378,7 +415,7 @@ void tc_launch_second(const Problem& pb, const TcPlan& pl)
     tc::k_theta_images<<<(total + 255) / 256, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NP, pb.ctl(), pl.img_hi, pl.img_lo);
     tc::k_pass2_tc<<<pl.g2, tc::NTHREADS, pl.smem2, pb.stream>>>(
         pl.tmX, pl.tmU, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NP,
-        pl.NSB, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
+        pl.PW, pl.NSB, pl.NLO, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
     pb.count(2);
 }
 

@@ -96,7 +96,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, float4 v)
 }
 
 // Host: 2-D FP32 tensor map over a row-major rows x cols matrix, box = box_rows x box_cols,
-// 128-byte swizzle (box_cols * 4 must be 128).  Out-of-range elements read as zero.
+// 128-byte swizzle when box_cols * 4 == 128, no swizzle otherwise.  Out-of-range elements read as zero.
 // Returns false if the driver entry point is missing or the encode fails.
 bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int cols, int box_rows,
                         int box_cols);

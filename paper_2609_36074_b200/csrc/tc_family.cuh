@@ -9,7 +9,8 @@ struct TcPlan {
     alignas(64) CUtensorMap tmX;   // X-hat boxes: 128 rows x 32 features
     alignas(64) CUtensorMap tmU;   // U panels: 128 rows x 32 columns (load and store)
     int NP;                        // r padded to a multiple of 16 (MMA N)
-    int NSB, NUP;                  // stage ring / panel ring sizes
+    int PW;                        // columns per U panel: 16 (plain rows) or 32 (128-byte swizzle)
+    int NSB, NLO, NUP;             // raw/hi box ring, lo box ring, U panel ring sizes
     int g2;                        // persistent grid
     size_t smem2;
     float* img_hi;                 // pre-split Theta^T images in the workspace
