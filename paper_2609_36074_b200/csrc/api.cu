@@ -84,8 +84,10 @@ struct gem_nlr {
     const char* path;
     bool use_ffma;         // first (and, unless use_tc, second) product by the FFMA family
     bool use_tc;           // second product by the tcgen05 family
+    bool use_tc1;          // first product by the tcgen05 family
     FfmaPlan ffma;
     TcPlan tc;
+    Tc1Plan tc1;
     char err[256];
     int64_t launches;      // kernels launched by this handle
     int pi_iters;          // power iterations taken by the last setup
@@ -150,7 +152,10 @@ static void launch_iteration(gem_nlr_t* h)
     const bool prof = h->profile && h->ev_used + 3 <= h->ev_cap;
     cudaEvent_t* e = prof ? h->ev + h->ev_used : nullptr;
     if (prof) cudaEventRecord(e[0], h->pb.stream);
-    if (h->use_ffma) {
+    if (h->use_tc1) {
+        tc1_launch_first(h->pb, h->tc1);
+        red1_fused_launch(h->pb, h->tc1.grid, 0);
+    } else if (h->use_ffma) {
         ffma_launch_first(h->pb, h->ffma, 0);
     } else {
         launch_vector_pass(h->pb);
@@ -240,6 +245,10 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
         tc_plan(h->pb, &h->tc, reinterpret_cast<float*>((char*)workspace_dev + L.thimg))) {
         h->use_tc = true;
         h->path = h->use_ffma ? "ffma+tf32x3" : "generic+tf32x3";
+        if (tc1_plan(h->pb, &h->tc1)) {
+            h->use_tc1 = true;
+            h->path = "tf32x3";
+        }
     }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||
         cudaMallocHost((void**)&h->host_scratch, 64) != cudaSuccess) {

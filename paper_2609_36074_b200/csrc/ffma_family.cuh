@@ -16,6 +16,8 @@ struct FfmaPlan {
 bool ffma_plan(const Problem& pb, FfmaPlan* plan);
 // Vector pass + Theta = X-hat^T U + reductions + the scalar step finishing the previous iteration.
 void ffma_launch_first(const Problem& pb, const FfmaPlan& plan, int mode);
+// Reduction of g per-CTA partial records [d*r Theta | r s | sum q^2 | sum ytilde q] (FP64) + scalar step.
+void red1_fused_launch(const Problem& pb, int g, int mode);
 // Fused second product, statistics, scalar step (multiplier, movement, gate, p).
 void ffma_launch_second(const Problem& pb, const FfmaPlan& plan);
 

@@ -24,7 +24,7 @@
 namespace gemnlr {
 
 bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int cols, int box_rows,
-                        int box_cols)
+                        int box_cols, bool atom32)
 {
     static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     if (!encode) {
@@ -41,7 +41,8 @@ bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int c
     cuuint32_t estr[2] = {1, 1};
     CUresult rc = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)base, gdim, gstride, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         box_cols * sizeof(float) == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                         box_cols * sizeof(float) != 128 ? CU_TENSOR_MAP_SWIZZLE_NONE
+                             : (atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B),
                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return rc == CUDA_SUCCESS;
 }
@@ -586,15 +587,21 @@ bool ffma_plan(const Problem& pb, FfmaPlan* pl)
     return ok;
 }
 
+void red1_fused_launch(const Problem& pb, int g, int mode)
+{
+    const int dr = pb.P.d * pb.P.r;
+    ffma::k_red1_fused<<<(dr + 63) / 64, 256, 0, pb.stream>>>(
+        pb.part1(), g, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
+        pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0);
+    pb.count(1);
+}
+
 void ffma_launch_first(const Problem& pb, const FfmaPlan& pl, int mode)
 {
     using namespace ffma;
     FFMA_DISPATCH(pl.shape_id, pass1(pb, pl));
-    const int dr = pb.P.d * pb.P.r;
-    k_red1_fused<<<(dr + 63) / 64, 256, 0, pb.stream>>>(
-        pb.part1(), pl.g1, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
-        pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0);
-    pb.count(2);
+    pb.count(1);
+    red1_fused_launch(pb, pl.g1, mode);
 }
 
 void ffma_launch_second(const Problem& pb, const FfmaPlan& pl)

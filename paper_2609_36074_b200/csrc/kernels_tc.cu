@@ -174,16 +174,14 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     tc_fence_after();
                     const uint32_t a_hi = stage0 + (uint32_t)s * BOX_BYTES, a_lo = lo0 + (uint32_t)l * BOX_BYTES;
                     const uint32_t b_hi = th_hi_s + (uint32_t)b * NP * 128, b_lo = th_lo_s + (uint32_t)b * NP * 128;
+                    // descriptors once per box; a k-step (8 features = 32 bytes inside the 128-byte
+                    // swizzled row) advances the start-address field by 2
+                    const uint64_t da_hi = umma_desc_sw128(a_hi, 16, 1024), da_lo = umma_desc_sw128(a_lo, 16, 1024);
+                    const uint64_t db_hi = umma_desc_sw128(b_hi, 16, 1024), db_lo = umma_desc_sw128(b_lo, 16, 1024);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t da_hi = umma_desc_sw128(a_hi + ks * 32, 16, 1024);
-                        const uint64_t da_lo = umma_desc_sw128(a_lo + ks * 32, 16, 1024);
-                        const uint64_t db_hi = umma_desc_sw128(b_hi + ks * 32, 16, 1024);
-                        const uint64_t db_lo = umma_desc_sw128(b_lo + ks * 32, 16, 1024);
-                        umma_tf32(tacc, da_hi, db_hi, idesc, (b | ks) ? 1u : 0u);
-                        umma_tf32(tacc, da_lo, db_hi, idesc, 1u);
-                        umma_tf32(tacc, da_hi, db_lo, idesc, 1u);
-                    }
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
+                                     (b | ks) ? 1u : 0u);
                     umma_commit(xfree(s));
                     umma_commit(lofree(l));
                 }

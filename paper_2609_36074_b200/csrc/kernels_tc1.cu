@@ -1,0 +1,303 @@
+// 3xTF32 tensor-core family (tcgen05 + TMEM): the first product of the iteration with the vector
+// pass fused in,
+//   Theta = X-hat^T U   (d x r),   u = c_f w,  q = u.p - 1,  gated ytilde += gamma q,
+//   ybar = ytilde + gamma q,  s = U^T ybar,  sum q^2,  sum ytilde q            (Algorithm 2, call sites 1-3, 8-11)
+// for shapes where FP32 FFMA cannot keep up with HBM (r > 16).
+//
+// The contraction runs over the data rows, so both operands are "MN-major": a TMA box of TR rows x
+// 32 columns with the 128-byte swizzle of 32-byte atoms is the canonical MN-major layout of TF32 UMMA
+// operands (128-byte rows along K in 4-row swizzle periods, 32-column chunks LBO bytes apart along M / N).  The accumulator is Theta^T:
+// TMEM lane = column j of U (M = 128, columns beyond r are zero-filled by TMA), TMEM column =
+// feature f (N = d).  Each k-step of 8 rows takes three MMAs (hi*hi, lo*hi, hi*lo).
+//
+// One persistent CTA per SM, 14 warps:
+//   warp 0       producer: per stage of TR = 32 rows, ceil(r/32) U boxes and d/32 X-hat boxes.
+//   warps 10-13  vector + split: 4 lanes per row do the row-local vector work on the U boxes, then
+//                rewrite every box as hi (in place) and lo (separate ring).
+//   warp 1       MMA issuer.  Every FLUSH stages the accumulator is handed to the epilogue and the
+//                other TMEM buffer is started from zero, so FP32 accumulation chains stay short.
+//   warps 2-9    epilogue: add each handed-over accumulator into this CTA's FP64 partial of Theta^T
+//                (thread = column j of U and half of the features).
+// Partials have the layout of the FFMA family's first product, so k_red1_fused reduces them.
+// Every mbarrier wait is bounded (GEM_NLR_E_TIMEOUT; the kernel runs to its end and frees its TMEM).
+#include "nlr_common.cuh"
+#include "device_utils.cuh"
+#include "pipeline.cuh"
+#include "tc_common.cuh"
+#include "tc_family.cuh"
+
+namespace gemnlr {
+namespace tc1 {
+
+constexpr int TR = 32;                         // data rows per stage (4 k-steps)
+constexpr int CHUNK_BYTES = TR * 128;          // one box: TR rows x 32 floats
+constexpr int NTHREADS = 14 * 32;
+constexpr int MAX_RING = 8;
+constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU,
+           float* __restrict__ ytilde, float* __restrict__ ybar, Ctl* __restrict__ ctl,
+           const float* __restrict__ p, int64_t n, int d, int r, int NSR, int NLO, double gamma,
+           double* __restrict__ part)
+{
+    if (ctl->stopped) return;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t bars[4 * MAX_RING + 4];
+    __shared__ uint32_t abort_flag;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ __align__(16) float sp[128];
+    __shared__ double sq[2][4];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int NBX = d / 32;                        // X-hat boxes per stage
+    const int NBU = (r + 31) / 32;                 // U boxes per stage (M = 128 reads 4; missing ones are never written: see below)
+    const int STAGE = (4 + NBX) * CHUNK_BYTES;     // U boxes always occupy 4 chunks so that M = 128 stays in the stage
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * d) tmem_cols <<= 1;
+
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t raw0 = smem_base;                                   // NSR stages: [4 U chunks][NBX X chunks], hi in place
+    const uint32_t lo0 = raw0 + (uint32_t)NSR * STAGE;                 // NLO stages of lo parts
+
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto split = [&](int s) { return bar0 + 8u * (MAX_RING + s); };
+    auto rawfree = [&](int s) { return bar0 + 8u * (2 * MAX_RING + s); };
+    auto lofree = [&](int s) { return bar0 + 8u * (3 * MAX_RING + s); };
+    auto accfull = [&](int a) { return bar0 + 8u * (4 * MAX_RING + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (4 * MAX_RING + 2 + a); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_RING; ++s) {
+            mbar_init(full(s), 1); mbar_init(split(s), 4); mbar_init(rawfree(s), 1); mbar_init(lofree(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 8); }
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (threadIdx.x < 128) sp[threadIdx.x] = (threadIdx.x < r) ? p[threadIdx.x] : 0.f;
+    // U chunks that no TMA box ever fills (r <= 96) must read as zeros: clear them once in every stage
+    for (int s = 0; s < NSR + NLO; ++s)
+        for (int c = NBU; c < 4; ++c)
+            for (int e = threadIdx.x; e < CHUNK_BYTES / 16; e += NTHREADS)
+                sts128((s < NSR ? raw0 + (uint32_t)s * STAGE : lo0 + (uint32_t)(s - NSR) * STAGE) + c * CHUNK_BYTES + e * 16,
+                       make_float4(0.f, 0.f, 0.f, 0.f));
+    fence_proxy_async();
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    // contiguous block of stages per CTA
+    const int64_t n_stages = (n + TR - 1) / TR;
+    const int64_t base_cnt = n_stages / gridDim.x, rem_cnt = n_stages % gridDim.x;
+    const int64_t g_lo = (int64_t)blockIdx.x * base_cnt + ((int64_t)blockIdx.x < rem_cnt ? blockIdx.x : rem_cnt);
+    const int my_stages = (int)(base_cnt + ((int64_t)blockIdx.x < rem_cnt ? 1 : 0));
+    const int n_periods = (my_stages + FLUSH - 1) / FLUSH;
+
+    const float cf = ctl->c_f;
+    const int dual = ctl->dual_pending;
+    double qq = 0.0, yq = 0.0;
+    float s_acc[32];                               // vector warps: s partial of this lane's 32 columns
+#pragma unroll
+    for (int k = 0; k < 32; ++k) s_acc[k] = 0.f;
+    double* const out = part + (size_t)blockIdx.x * ((size_t)d * r + r + 2);
+
+    if (warp == 0) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            for (int g = 0; g < my_stages && !abort_flag; ++g) {
+                const int s = g % NSR;
+                if (g >= NSR) mbar_wait(rawfree(s), ((g / NSR) - 1) & 1, &abort_flag, ctl);
+                const int row0 = (int)((g_lo + g) * TR);
+                const uint32_t dst = raw0 + (uint32_t)s * STAGE;
+                mbar_expect_tx(full(s), (uint32_t)(NBU + NBX) * CHUNK_BYTES);
+                for (int c = 0; c < NBU; ++c) tma_load_2d(dst + c * CHUNK_BYTES, &tmU, c * 32, row0, full(s));
+                for (int b = 0; b < NBX; ++b) tma_load_2d(dst + (4 + b) * CHUNK_BYTES, &tmX, b * 32, row0, full(s));
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_tf32(128, d, 1, 1);
+            for (int g = 0; g < my_stages && !abort_flag; ++g) {
+                const int s = g % NSR, l = g % NLO;
+                const int period = g / FLUSH, a = period & 1, in_period = g % FLUSH;
+                if (in_period == 0 && period >= 2) mbar_wait(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
+                mbar_wait(split(s), (g / NSR) & 1, &abort_flag, ctl);
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(a * d);
+                const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, lo_s = lo0 + (uint32_t)l * STAGE;
+                // A = U chunks (M), B = X-hat chunks (N); chunks are CHUNK_BYTES apart (LBO), a k-step is 1 KB
+                // (4-row swizzle periods of 512 bytes along K: SBO)
+                const uint64_t da_hi = umma_desc_sw128_atom32(hi_s, CHUNK_BYTES, 512), da_lo = umma_desc_sw128_atom32(lo_s, CHUNK_BYTES, 512);
+                const uint64_t db_hi = umma_desc_sw128_atom32(hi_s + 4 * CHUNK_BYTES, CHUNK_BYTES, 512);
+                const uint64_t db_lo = umma_desc_sw128_atom32(lo_s + 4 * CHUNK_BYTES, CHUNK_BYTES, 512);
+#pragma unroll
+                for (int ks = 0; ks < TR / 8; ++ks)
+                    umma_tf32_x3(tacc, da_hi + 64 * ks, da_lo + 64 * ks, db_hi + 64 * ks, db_lo + 64 * ks, idesc,
+                                 (in_period | ks) ? 1u : 0u);
+                umma_commit(rawfree(s));
+                umma_commit(lofree(l));
+                if (in_period == FLUSH - 1 || g == my_stages - 1) umma_commit(accfull(a));
+            }
+        }
+    } else if (warp >= 10) {
+        // ------------------------------ vector pass + split ------------------------------
+        const int vt = threadIdx.x - 10 * 32;              // 0..127
+        const int rl = vt >> 2, sub = vt & 3;              // row of the stage, U chunk (32 columns) of this lane
+        for (int g = 0; g < my_stages; ++g) {
+            const int s = g % NSR, l = g % NLO;
+            const int64_t row = (g_lo + g) * TR + rl;
+            const bool valid = row < n;
+            float yt = (valid && sub == 0) ? ytilde[row] : 0.f;
+            mbar_wait(full(s), (g / NSR) & 1, &abort_flag, ctl);
+            if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+            const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, lo_s = lo0 + (uint32_t)l * STAGE;
+            // ---- row-local vector work on this lane's 32 columns of u ----
+            float u[32];
+            float dot = 0.f;
+            const uint32_t ub = (uint32_t)(sub * CHUNK_BYTES + rl * 128);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 w4 = lds128(hi_s + ub + (uint32_t)((((c >> 1) ^ (rl & 3)) << 5) | ((c & 1) << 4)));
+                const float4 p4 = *reinterpret_cast<const float4*>(sp + sub * 32 + 4 * c);
+                u[4 * c + 0] = cf * w4.x; u[4 * c + 1] = cf * w4.y; u[4 * c + 2] = cf * w4.z; u[4 * c + 3] = cf * w4.w;
+                dot = fmaf(u[4 * c + 0], p4.x, dot); dot = fmaf(u[4 * c + 1], p4.y, dot);
+                dot = fmaf(u[4 * c + 2], p4.z, dot); dot = fmaf(u[4 * c + 3], p4.w, dot);
+            }
+            dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+            dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+            const float q = dot - 1.0f;
+            float yb = 0.f;
+            if (sub == 0) {
+                if (dual) yt = (float)((double)yt + gamma * (double)q);
+                yb = (float)((double)yt + gamma * (double)q);
+                if (valid) {
+                    if (dual) ytilde[row] = yt;
+                    ybar[row] = yb;
+                    qq = fma((double)q, (double)q, qq);
+                    yq = fma((double)yt, (double)q, yq);
+                }
+            }
+            yb = __shfl_sync(0xffffffffu, yb, lane & ~3);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) s_acc[k] = fmaf(u[k], yb, s_acc[k]);    // rows beyond n have u = 0
+            // ---- split of this lane's U chunk row ----
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t off = ub + (uint32_t)((((c >> 1) ^ (rl & 3)) << 5) | ((c & 1) << 4));
+                const float4 hi = make_float4(tf32_hi(u[4 * c]), tf32_hi(u[4 * c + 1]), tf32_hi(u[4 * c + 2]), tf32_hi(u[4 * c + 3]));
+                sts128(hi_s + off, hi);
+                sts128(lo_s + off, make_float4(u[4 * c] - hi.x, u[4 * c + 1] - hi.y, u[4 * c + 2] - hi.z, u[4 * c + 3] - hi.w));
+            }
+            // ---- split of the X-hat boxes: 256 float4 per box over 128 threads ----
+            for (int b = 0; b < NBX; ++b) {
+                const uint32_t base = (uint32_t)((4 + b) * CHUNK_BYTES);
+                const float4 x0 = lds128(hi_s + base + (uint32_t)vt * 16);
+                const float4 x1 = lds128(hi_s + base + (uint32_t)(128 + vt) * 16);
+                const float4 h0 = make_float4(tf32_hi(x0.x), tf32_hi(x0.y), tf32_hi(x0.z), tf32_hi(x0.w));
+                const float4 h1 = make_float4(tf32_hi(x1.x), tf32_hi(x1.y), tf32_hi(x1.z), tf32_hi(x1.w));
+                sts128(hi_s + base + (uint32_t)vt * 16, h0);
+                sts128(hi_s + base + (uint32_t)(128 + vt) * 16, h1);
+                sts128(lo_s + base + (uint32_t)vt * 16, make_float4(x0.x - h0.x, x0.y - h0.y, x0.z - h0.z, x0.w - h0.w));
+                sts128(lo_s + base + (uint32_t)(128 + vt) * 16, make_float4(x1.x - h1.x, x1.y - h1.y, x1.z - h1.z, x1.w - h1.w));
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(split(s));
+        }
+        qq = warp_sum(qq);
+        yq = warp_sum(yq);
+        if (lane == 0) { sq[0][warp - 10] = qq; sq[1][warp - 10] = yq; }
+    }
+    if (warp >= 2 && warp < 10) {
+        // ------------------------------ epilogue: FP64 fold of the accumulator ------------------------------
+        // Thread = column j of U (TMEM lane) and half of the features.  Each hand-over adds the FP32
+        // accumulator of the period into this CTA's FP64 partial record (Theta^T entry (j, f) lives at
+        // out[f * r + j]; every thread owns its addresses, lanes are contiguous in j).
+        const int q4 = warp & 3;                          // TMEM lane quarter
+        const int fh = (warp - 2) >> 2;                   // feature half
+        const int j = q4 * 32 + lane;                     // column of U
+        const int f_per = d / 2;                          // features per thread (multiple of 16)
+        for (int period = 0; period < n_periods; ++period) {
+            const int a = period & 1;
+            mbar_wait(accfull(a), (period >> 1) & 1, &abort_flag, ctl);
+            tc_fence_after();
+            for (int c = 0; c * 16 < f_per; ++c) {
+                float v[16];
+                tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * d + fh * f_per + c * 16), v);
+                if (j < r) {
+                    double* o = out + (size_t)(fh * f_per + c * 16) * r + j;
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const double prev = (period == 0) ? 0.0 : o[(size_t)k * r];
+                        o[(size_t)k * r] = prev + (double)v[k];
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(accfree(a));
+        }
+    }
+    // Every MMA has completed (the epilogue waited for the last hand-over): the rings are scratch now.
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
+    float* sscr = reinterpret_cast<float*>(smem);             // [32 rows][128 columns]
+    if (warp >= 10) {
+        const int vt = threadIdx.x - 10 * 32, rl = vt >> 2, sub = vt & 3;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) sscr[rl * 128 + sub * 32 + k] = s_acc[k];
+    }
+    __syncthreads();
+    if (threadIdx.x < r) {
+        double v = 0.0;
+        for (int k = 0; k < 32; ++k) v += (double)sscr[k * 128 + threadIdx.x];
+        out[(size_t)d * r + threadIdx.x] = v;
+    }
+    if (threadIdx.x == 0) {
+        out[(size_t)d * r + r] = ((sq[0][0] + sq[0][1]) + sq[0][2]) + sq[0][3];
+        out[(size_t)d * r + r + 1] = ((sq[1][0] + sq[1][1]) + sq[1][2]) + sq[1][3];
+    }
+}
+
+}  // namespace tc1
+
+bool tc1_plan(const Problem& pb, Tc1Plan* pl)
+{
+    const int d = pb.P.d, r = pb.P.r;
+    if (d % 32 != 0 || d > 256 || r % 4 != 0 || r < 8 || r > 128 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
+    if ((size_t)d * r > 16384) return false;          // partial records of the shared reduction kernel
+    const int NBX = d / 32;
+    const size_t stage = (size_t)(4 + NBX) * tc1::CHUNK_BYTES;
+    const size_t limit = 227 * 1024 - 2048;
+    int NLO = 0, NSR = 0;
+    for (int nlo = 3; nlo >= 2 && !NSR; --nlo)
+        for (int nsr = tc1::MAX_RING; nsr >= 2; --nsr)
+            if ((size_t)(nsr + nlo) * stage + 1024 <= limit) { NSR = nsr; NLO = nlo; break; }
+    if (!NSR) return false;
+    pl->NSR = NSR; pl->NLO = NLO;
+    pl->smem = (size_t)(NSR + NLO) * stage + 1024;
+    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc1::TR, 32, true)) return false;
+    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tc1::TR, 32, true)) return false;
+    const int64_t stages = (pb.P.n + tc1::TR - 1) / tc1::TR;
+    pl->grid = (int)(stages < kSMs ? stages : kSMs);
+    if (cudaFuncSetAttribute(tc1::k_pass1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess)
+        return false;
+    return true;
+}
+
+void tc1_launch_first(const Problem& pb, const Tc1Plan& pl)
+{
+    tc1::k_pass1_tc<<<pl.grid, tc1::NTHREADS, pl.smem, pb.stream>>>(
+        pl.tmX, pl.tmU, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.P.d, pb.P.r, pl.NSR, pl.NLO, pb.gamma,
+        pb.part1());
+    pb.count(1);
+}
+
+}  // namespace gemnlr

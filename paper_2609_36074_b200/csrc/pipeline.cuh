@@ -83,6 +83,12 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
         ::"r"(dst), "l"((uint64_t)src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// Hint: bring `bytes` (multiple of 16) starting at the 16-byte aligned global address into L2.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"((uint64_t)src), "r"(bytes) : "memory");
+}
+
 __device__ __forceinline__ float4 lds128(uint32_t addr)
 {
     float4 v;
@@ -96,9 +102,11 @@ __device__ __forceinline__ void sts128(uint32_t addr, float4 v)
 }
 
 // Host: 2-D FP32 tensor map over a row-major rows x cols matrix, box = box_rows x box_cols,
-// 128-byte swizzle when box_cols * 4 == 128, no swizzle otherwise.  Out-of-range elements read as zero.
+// 128-byte swizzle when box_cols * 4 == 128 (16-byte atoms: chunk index XOR row mod 8; or, with
+// atom32, 32-byte atoms: 32-byte chunk index XOR row mod 4 -- the layout MN-major TF32 UMMA operands
+// need), no swizzle otherwise.  Out-of-range elements read as zero.
 // Returns false if the driver entry point is missing or the encode fails.
 bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int cols, int box_rows,
-                        int box_cols);
+                        int box_cols, bool atom32 = false);
 
 }  // namespace gemnlr

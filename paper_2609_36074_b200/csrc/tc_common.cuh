@@ -22,6 +22,19 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
     return d;
 }
 
+// Same for the 128-byte swizzle with 32-byte atoms (layout type 1), the only layout MN-major TF32
+// operands may use: 128-byte rows along K, the 32-byte chunk index XORed with the row index mod 4.
+__device__ __forceinline__ uint64_t umma_desc_sw128_atom32(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;          // version
+    d |= (uint64_t)1 << 61;          // SWIZZLE_128B_BASE32B
+    return d;
+}
+
 // Instruction descriptor for kind::tf32, FP32 accumulate, M x N tile; a_mn / b_mn: operand is
 // MN-major (1) or K-major (0).
 __host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N, int a_mn, int b_mn)
@@ -39,6 +52,22 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint6
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+
+// The three products of one k-step of the split scheme, D (+)= Ahi*Bhi + Alo*Bhi + Ahi*Blo, from one
+// asm block so that the issuing thread spends as few instructions as possible per MMA.
+__device__ __forceinline__ void umma_tf32_x3(uint32_t tmem_d, uint64_t a_hi, uint64_t a_lo, uint64_t b_hi,
+                                             uint64_t b_lo, uint32_t idesc, uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, t;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "setp.eq.b32 t, %7, %7;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %3, %5, {%7, %7, %7, %7}, p;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %2, %3, %5, {%7, %7, %7, %7}, t;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %4, %5, {%7, %7, %7, %7}, t;\n\t}"
+        ::"r"(tmem_d), "l"(a_hi), "l"(a_lo), "l"(b_hi), "l"(b_lo), "r"(idesc), "r"(accumulate_first), "r"(0u)
         : "memory");
 }
 

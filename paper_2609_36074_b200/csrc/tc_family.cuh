@@ -24,3 +24,20 @@ bool tc_plan(const Problem& pb, TcPlan* plan, float* img_storage);
 void tc_launch_second(const Problem& pb, const TcPlan& plan);
 
 }  // namespace gemnlr
+
+namespace gemnlr {
+
+// First product + vector pass on tcgen05 (kernels_tc1.cu): d a multiple of 32 up to 256,
+// r a multiple of 4 in [8, 128], d * r <= 16384.
+struct Tc1Plan {
+    alignas(64) CUtensorMap tmX;   // X-hat boxes: 32 rows x 32 features
+    alignas(64) CUtensorMap tmU;   // U boxes: 32 rows x 32 columns
+    int NSR, NLO;                  // raw stage ring, lo stage ring
+    int grid;
+    size_t smem;
+};
+bool tc1_plan(const Problem& pb, Tc1Plan* plan);
+// Theta partials, s, sum q^2, sum ytilde q (reduced afterwards by the FFMA family's k_red1_fused).
+void tc1_launch_first(const Problem& pb, const Tc1Plan& plan);
+
+}  // namespace gemnlr
