@@ -237,17 +237,25 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     h->path = "generic";
     h->err[0] = 0;
     h->pb.launches = &h->launches;
-    if (params->precision != 2 && ffma_plan(h->pb, &h->ffma)) {
+    // Kernel families by shape.  precision 2: generic only.  precision 0: FFMA family where a shape is
+    // instantiated, else generic.  precision 1: tensor cores wherever they are available.  precision -1:
+    // FFMA for the skinny shapes (r <= 16: there the FP32 pipes keep up and the tensor-core path would
+    // issue one MMA triple per 8 rows for 16 useful columns), tensor cores for r >= 32, else generic.
+    const bool want_ffma = params->precision != 2;
+    const bool want_tc = params->precision == 1 || (params->precision == -1 && params->r >= 32);
+    if (want_ffma && ffma_plan(h->pb, &h->ffma)) {
         h->use_ffma = true;
         h->path = "ffma";
     }
-    if (params->precision == 1 &&
-        tc_plan(h->pb, &h->tc, reinterpret_cast<float*>((char*)workspace_dev + L.thimg))) {
-        h->use_tc = true;
-        h->path = h->use_ffma ? "ffma+tf32x3" : "generic+tf32x3";
-        if (tc1_plan(h->pb, &h->tc1)) {
-            h->use_tc1 = true;
-            h->path = "tf32x3";
+    if (want_tc && !(params->precision == -1 && h->use_ffma)) {
+        float* img = reinterpret_cast<float*>((char*)workspace_dev + L.thimg);
+        if (tc_plan(h->pb, &h->tc, img)) {
+            h->use_tc = true;
+            h->path = h->use_ffma ? "ffma+tf32x3" : "generic+tf32x3";
+            if (tc1_plan(h->pb, &h->tc1)) {
+                h->use_tc1 = true;
+                h->path = "tf32x3";
+            }
         }
     }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||

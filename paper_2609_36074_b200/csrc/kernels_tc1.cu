@@ -12,12 +12,12 @@
 //
 // One persistent CTA per SM, 14 warps:
 //   warp 0       producer: per stage of TR = 32 rows, ceil(r/32) U boxes and d/32 X-hat boxes.
-//   warps 10-13  vector + split: 4 lanes per row do the row-local vector work on the U boxes, then
-//                rewrite every box as hi (in place) and lo (separate ring).
+//   warps 6-13   vector + split: one warp per row does the row-local vector work on the U boxes and
+//                rewrites them as hi (in place) and lo (separate ring); then the X-hat boxes are split.
 //   warp 1       MMA issuer.  Every FLUSH stages the accumulator is handed to the epilogue and the
 //                other TMEM buffer is started from zero, so FP32 accumulation chains stay short.
-//   warps 2-9    epilogue: add each handed-over accumulator into this CTA's FP64 partial of Theta^T
-//                (thread = column j of U and half of the features).
+//   warps 2-5    epilogue: add each handed-over accumulator into this CTA's FP64 partial of Theta^T
+//                (thread = column j of U).
 // Partials have the layout of the FFMA family's first product, so k_red1_fused reduces them.
 // Every mbarrier wait is bounded (GEM_NLR_E_TIMEOUT; the kernel runs to its end and frees its TMEM).
 #include "nlr_common.cuh"
@@ -48,7 +48,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t tmem_base_s;
     __shared__ __align__(16) float sp[128];
-    __shared__ double sq[2][4];
+    __shared__ double sq[2][8];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NBX = d / 32;                        // X-hat boxes per stage
@@ -73,7 +73,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         for (int s = 0; s < MAX_RING; ++s) {
             mbar_init(full(s), 1); mbar_init(split(s), 4); mbar_init(rawfree(s), 1); mbar_init(lofree(s), 1);
         }
-        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 8); }
+        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4); }
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -101,9 +101,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     const float cf = ctl->c_f;
     const int dual = ctl->dual_pending;
     double qq = 0.0, yq = 0.0;
-    float s_acc[32];                               // vector warps: s partial of this lane's 32 columns
-#pragma unroll
-    for (int k = 0; k < 32; ++k) s_acc[k] = 0.f;
+    float s_acc[4] = {0.f, 0.f, 0.f, 0.f};         // vector warps: s partial of this lane's 4 columns
     double* const out = part + (size_t)blockIdx.x * ((size_t)d * r + r + 2);
 
     if (warp == 0) {
@@ -145,66 +143,91 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 if (in_period == FLUSH - 1 || g == my_stages - 1) umma_commit(accfull(a));
             }
         }
-    } else if (warp >= 10) {
+    } else if (warp >= 6) {
         // ------------------------------ vector pass + split ------------------------------
-        const int vt = threadIdx.x - 10 * 32;              // 0..127
-        const int rl = vt >> 2, sub = vt & 3;              // row of the stage, U chunk (32 columns) of this lane
-        for (int g = 0; g < my_stages; ++g) {
+        // One warp per row at a time: lane = (U chunk, 16-byte piece), i.e. the 32 lanes read the 4 x 8
+        // pieces of one row -- every quarter-warp covers one full 128-byte line, no bank conflicts.
+        // Two teams of four warps take alternate stages, so the fixed latencies of a stage (barrier
+        // wake-ups, fence, hand-over to the MMA issuer) of one team overlap the work of the other.
+        const int vw = warp - 6;                           // 0..7
+        const int team = vw >> 2, tw = vw & 3;             // team; rows tw + 4 k (k = 0..7) of the team's stages
+        const int tt = (vw & 3) * 32 + lane;               // 0..127 inside the team
+        const int box = lane >> 3, c = lane & 7;           // U chunk (32 columns) and logical 16-byte piece inside it
+        const int col0 = box * 32 + 4 * c;                 // first of this lane's 4 columns of u
+        const float4 p4 = *reinterpret_cast<const float4*>(sp + col0);
+        for (int g = team; g < my_stages; g += 2) {
             const int s = g % NSR, l = g % NLO;
-            const int64_t row = (g_lo + g) * TR + rl;
-            const bool valid = row < n;
-            float yt = (valid && sub == 0) ? ytilde[row] : 0.f;
+            const int64_t srow0 = (g_lo + g) * TR;
+            // ytilde of this warp's eight rows (lane k < 8 holds row tw + 4 k), fetched before the waits
+            const int64_t myrow = srow0 + tw + 4 * (lane & 7);
+            float yt_l = (lane < 8 && myrow < n) ? ytilde[myrow] : 0.f;
+            float yb_l = 0.f;
             mbar_wait(full(s), (g / NSR) & 1, &abort_flag, ctl);
             if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
             const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, lo_s = lo0 + (uint32_t)l * STAGE;
-            // ---- row-local vector work on this lane's 32 columns of u ----
-            float u[32];
-            float dot = 0.f;
-            const uint32_t ub = (uint32_t)(sub * CHUNK_BYTES + rl * 128);
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const float4 w4 = lds128(hi_s + ub + (uint32_t)((((c >> 1) ^ (rl & 3)) << 5) | ((c & 1) << 4)));
-                const float4 p4 = *reinterpret_cast<const float4*>(sp + sub * 32 + 4 * c);
-                u[4 * c + 0] = cf * w4.x; u[4 * c + 1] = cf * w4.y; u[4 * c + 2] = cf * w4.z; u[4 * c + 3] = cf * w4.w;
-                dot = fmaf(u[4 * c + 0], p4.x, dot); dot = fmaf(u[4 * c + 1], p4.y, dot);
-                dot = fmaf(u[4 * c + 2], p4.z, dot); dot = fmaf(u[4 * c + 3], p4.w, dot);
-            }
-            dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-            dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-            const float q = dot - 1.0f;
-            float yb = 0.f;
-            if (sub == 0) {
-                if (dual) yt = (float)((double)yt + gamma * (double)q);
-                yb = (float)((double)yt + gamma * (double)q);
-                if (valid) {
-                    if (dual) ytilde[row] = yt;
-                    ybar[row] = yb;
-                    qq = fma((double)q, (double)q, qq);
-                    yq = fma((double)yt, (double)q, yq);
+            for (int half = 0; half < 2; ++half) {
+                // four independent rows at a time: loads first, reductions interleaved, then scalars and stores
+                uint32_t off[4];
+                float4 u4[4];
+                float dot[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int rl = tw + 4 * (half * 4 + k);
+                    off[k] = (uint32_t)(box * CHUNK_BYTES + rl * 128) + (uint32_t)((((c >> 1) ^ (rl & 3)) << 5) | ((c & 1) << 4));
+                }
+                {
+                    float4 w4[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) w4[k] = lds128(hi_s + off[k]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        u4[k] = make_float4(cf * w4[k].x, cf * w4[k].y, cf * w4[k].z, cf * w4[k].w);
+                        dot[k] = fmaf(u4[k].x, p4.x, fmaf(u4[k].y, p4.y, fmaf(u4[k].z, p4.z, u4[k].w * p4.w)));
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) dot[k] += __shfl_xor_sync(0xffffffffu, dot[k], o);
+                // row scalars: lane 4 half + k owns row tw + 4 (4 half + k) (dot[] is the same in every lane)
+                {
+                    const int kk = lane & 3;
+                    const float q = (kk == 0) ? dot[0] : (kk == 1) ? dot[1] : (kk == 2) ? dot[2] : dot[3];
+                    const float qm1 = q - 1.0f;
+                    if ((lane >> 2) == half) {
+                        if (dual) yt_l = (float)((double)yt_l + gamma * (double)qm1);
+                        yb_l = (float)((double)yt_l + gamma * (double)qm1);
+                        if (myrow < n) {
+                            qq = fma((double)qm1, (double)qm1, qq);
+                            yq = fma((double)yt_l, (double)qm1, yq);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float yb = __shfl_sync(0xffffffffu, yb_l, half * 4 + k);
+                    s_acc[0] = fmaf(u4[k].x, yb, s_acc[0]); s_acc[1] = fmaf(u4[k].y, yb, s_acc[1]);   // rows beyond n: u = 0
+                    s_acc[2] = fmaf(u4[k].z, yb, s_acc[2]); s_acc[3] = fmaf(u4[k].w, yb, s_acc[3]);
+                    const float4 hi = make_float4(tf32_hi(u4[k].x), tf32_hi(u4[k].y), tf32_hi(u4[k].z), tf32_hi(u4[k].w));
+                    sts128(hi_s + off[k], hi);
+                    sts128(lo_s + off[k], make_float4(u4[k].x - hi.x, u4[k].y - hi.y, u4[k].z - hi.z, u4[k].w - hi.w));
                 }
             }
-            yb = __shfl_sync(0xffffffffu, yb, lane & ~3);
-#pragma unroll
-            for (int k = 0; k < 32; ++k) s_acc[k] = fmaf(u[k], yb, s_acc[k]);    // rows beyond n have u = 0
-            // ---- split of this lane's U chunk row ----
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t off = ub + (uint32_t)((((c >> 1) ^ (rl & 3)) << 5) | ((c & 1) << 4));
-                const float4 hi = make_float4(tf32_hi(u[4 * c]), tf32_hi(u[4 * c + 1]), tf32_hi(u[4 * c + 2]), tf32_hi(u[4 * c + 3]));
-                sts128(hi_s + off, hi);
-                sts128(lo_s + off, make_float4(u[4 * c] - hi.x, u[4 * c + 1] - hi.y, u[4 * c + 2] - hi.z, u[4 * c + 3] - hi.w));
+            if (lane < 8 && myrow < n) {
+                if (dual) ytilde[myrow] = yt_l;
+                ybar[myrow] = yb_l;
             }
-            // ---- split of the X-hat boxes: 256 float4 per box over 128 threads ----
+            // ---- split of the X-hat boxes: 256 float4 per box, two per thread of the team ----
             for (int b = 0; b < NBX; ++b) {
-                const uint32_t base = (uint32_t)((4 + b) * CHUNK_BYTES);
-                const float4 x0 = lds128(hi_s + base + (uint32_t)vt * 16);
-                const float4 x1 = lds128(hi_s + base + (uint32_t)(128 + vt) * 16);
+                const uint32_t o0 = (uint32_t)((4 + b) * CHUNK_BYTES) + (uint32_t)tt * 16, o1 = o0 + 128 * 16;
+                const float4 x0 = lds128(hi_s + o0), x1 = lds128(hi_s + o1);
                 const float4 h0 = make_float4(tf32_hi(x0.x), tf32_hi(x0.y), tf32_hi(x0.z), tf32_hi(x0.w));
                 const float4 h1 = make_float4(tf32_hi(x1.x), tf32_hi(x1.y), tf32_hi(x1.z), tf32_hi(x1.w));
-                sts128(hi_s + base + (uint32_t)vt * 16, h0);
-                sts128(hi_s + base + (uint32_t)(128 + vt) * 16, h1);
-                sts128(lo_s + base + (uint32_t)vt * 16, make_float4(x0.x - h0.x, x0.y - h0.y, x0.z - h0.z, x0.w - h0.w));
-                sts128(lo_s + base + (uint32_t)(128 + vt) * 16, make_float4(x1.x - h1.x, x1.y - h1.y, x1.z - h1.z, x1.w - h1.w));
+                sts128(hi_s + o0, h0);
+                sts128(hi_s + o1, h1);
+                sts128(lo_s + o0, make_float4(x0.x - h0.x, x0.y - h0.y, x0.z - h0.z, x0.w - h0.w));
+                sts128(lo_s + o1, make_float4(x1.x - h1.x, x1.y - h1.y, x1.z - h1.z, x1.w - h1.w));
             }
             fence_proxy_async();
             __syncwarp();
@@ -212,26 +235,24 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         }
         qq = warp_sum(qq);
         yq = warp_sum(yq);
-        if (lane == 0) { sq[0][warp - 10] = qq; sq[1][warp - 10] = yq; }
+        if (lane == 0) { sq[0][vw] = qq; sq[1][vw] = yq; }
     }
-    if (warp >= 2 && warp < 10) {
+    if (warp >= 2 && warp < 6) {
         // ------------------------------ epilogue: FP64 fold of the accumulator ------------------------------
-        // Thread = column j of U (TMEM lane) and half of the features.  Each hand-over adds the FP32
+        // Thread = column j of U (TMEM lane).  Each hand-over adds the FP32
         // accumulator of the period into this CTA's FP64 partial record (Theta^T entry (j, f) lives at
         // out[f * r + j]; every thread owns its addresses, lanes are contiguous in j).
         const int q4 = warp & 3;                          // TMEM lane quarter
-        const int fh = (warp - 2) >> 2;                   // feature half
         const int j = q4 * 32 + lane;                     // column of U
-        const int f_per = d / 2;                          // features per thread (multiple of 16)
         for (int period = 0; period < n_periods; ++period) {
             const int a = period & 1;
             mbar_wait(accfull(a), (period >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
-            for (int c = 0; c * 16 < f_per; ++c) {
+            for (int c = 0; c * 16 < d; ++c) {
                 float v[16];
-                tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * d + fh * f_per + c * 16), v);
+                tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * d + c * 16), v);
                 if (j < r) {
-                    double* o = out + (size_t)(fh * f_per + c * 16) * r + j;
+                    double* o = out + (size_t)(c * 16) * r + j;
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const double prev = (period == 0) ? 0.0 : o[(size_t)k * r];
@@ -248,21 +269,23 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
-    float* sscr = reinterpret_cast<float*>(smem);             // [32 rows][128 columns]
-    if (warp >= 10) {
-        const int vt = threadIdx.x - 10 * 32, rl = vt >> 2, sub = vt & 3;
+    float* sscr = reinterpret_cast<float*>(smem);             // [8 vector warps][128 columns]
+    if (warp >= 6) {
+        const int col0 = (lane >> 3) * 32 + 4 * (lane & 7);
 #pragma unroll
-        for (int k = 0; k < 32; ++k) sscr[rl * 128 + sub * 32 + k] = s_acc[k];
+        for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + col0 + k] = s_acc[k];
     }
     __syncthreads();
     if (threadIdx.x < r) {
         double v = 0.0;
-        for (int k = 0; k < 32; ++k) v += (double)sscr[k * 128 + threadIdx.x];
+        for (int k = 0; k < 8; ++k) v += (double)sscr[k * 128 + threadIdx.x];
         out[(size_t)d * r + threadIdx.x] = v;
     }
     if (threadIdx.x == 0) {
-        out[(size_t)d * r + r] = ((sq[0][0] + sq[0][1]) + sq[0][2]) + sq[0][3];
-        out[(size_t)d * r + r + 1] = ((sq[1][0] + sq[1][1]) + sq[1][2]) + sq[1][3];
+        double a0 = 0.0, a1 = 0.0;
+        for (int w = 0; w < 8; ++w) { a0 += sq[0][w]; a1 += sq[1][w]; }
+        out[(size_t)d * r + r] = a0;
+        out[(size_t)d * r + r + 1] = a1;
     }
 }
 
@@ -277,8 +300,8 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     const size_t stage = (size_t)(4 + NBX) * tc1::CHUNK_BYTES;
     const size_t limit = 227 * 1024 - 2048;
     int NLO = 0, NSR = 0;
-    for (int nlo = 3; nlo >= 2 && !NSR; --nlo)
-        for (int nsr = tc1::MAX_RING; nsr >= 2; --nsr)
+    for (int nlo = 4; nlo >= 2 && !NSR; --nlo)
+        for (int nsr = tc1::MAX_RING; nsr >= (nlo >= 3 ? 4 : 2); --nsr)
             if ((size_t)(nsr + nlo) * stage + 1024 <= limit) { NSR = nsr; NLO = nlo; break; }
     if (!NSR) return false;
     pl->NSR = NSR; pl->NLO = NLO;
