@@ -105,9 +105,12 @@ size_t gem_nlr_paper_storage_bytes(const gem_nlr_params *params);
 int gem_nlr_create(gem_nlr_t **out, const gem_nlr_params *params, float *X_dev, float *U_dev,
                    void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
 
-/* Setup of Section 3: column mean (if center), a = ||X_c||_2 by power iteration on X_c^T X_c
- * applied implicitly (one pass over X per iteration), then X-hat = X_c / a written over X_dev
- * (x_inplace) or into the workspace.  *a_out receives a.  Synchronizes.                        */
+/* Setup of Section 3: column mean (if center), a = ||X_c||_2, then X-hat = X_c / a written over
+ * X_dev (x_inplace) or into the workspace.  a comes from applying X_c^T X_c implicitly to unit
+ * vectors (one streaming pass over X per application, the power-iteration kernel pair) combined
+ * by a Lanczos recurrence on the host: the estimate is the largest Ritz value, never above the
+ * true norm; it stops when the estimate moves by less than pi_tol (relative) twice in a row or
+ * after pi_max_iters passes.  *a_out receives a.  Synchronizes.                                */
 int gem_nlr_spectral_norm(gem_nlr_t *h, double *a_out);
 
 /* Declare that X_dev already holds X-hat (normalized elsewhere); a is recorded only.           */

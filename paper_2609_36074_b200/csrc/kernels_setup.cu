@@ -1,7 +1,7 @@
 // Setup of the normalized model (Section 3): X_c = X - 1 xbar^T, a = ||X_c||_2, X-hat = X_c / a.
-// The paper does not say how a is computed; here it is a power iteration on X_c^T X_c applied
-// implicitly, one streaming pass over X per iteration:  w = sum_i z_i (x_i - xbar),
-// z_i = (x_i - xbar) . v,  sigma = sqrt(||w||) for ||v|| = 1,  v <- w / ||w||.
+// The paper does not say how a is computed; here X_c^T X_c is applied implicitly to a unit vector,
+// one streaming pass over X per application:  w = sum_i z_i (x_i - xbar),  z_i = (x_i - xbar) . v.
+// The host combines the applications (Krylov / Lanczos form of the power iteration, see below).
 // All sums are FP64 and combined in a fixed order.
 #include "nlr_common.cuh"
 #include "device_utils.cuh"
@@ -80,23 +80,15 @@ k_pi_pass(const float* __restrict__ X, int64_t n, int d, const double* __restric
     }
 }
 
-// w = sum of partials; sigma = sqrt(||w||); v <- w / ||w||.  scal[0] = sigma, scal[1] = ||w||.
+// w = sum of the per-CTA partials in CTA order (the result of one application of X_c^T X_c to v).
 __global__ void __launch_bounds__(256)
-k_pi_fin(const double* __restrict__ part, int g, int d, double* __restrict__ v,
-         double* __restrict__ scal)
+k_pi_fin(const double* __restrict__ part, int g, int d, double* __restrict__ w)
 {
-    __shared__ double sred[32];
-    double nrm2 = 0.0;
-    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < d; j += gridDim.x * blockDim.x) {
         double t = 0.0;
         for (int b = 0; b < g; ++b) t += part[(size_t)b * d + j];
-        v[j] = t;
-        nrm2 += t * t;
+        w[j] = t;
     }
-    nrm2 = block_sum<256>(nrm2, sred);
-    const double nrm = sqrt(nrm2);
-    for (int j = threadIdx.x; j < d; j += blockDim.x) v[j] = (nrm > 0.0) ? v[j] / nrm : 0.0;
-    if (threadIdx.x == 0) { scal[0] = sqrt(nrm); scal[1] = nrm; }
 }
 
 // X-hat = FP32((X - mean) * (1/a)), evaluated in FP64.
@@ -135,16 +127,48 @@ static inline uint64_t splitmix64(uint64_t x)
     return x ^ (x >> 31);
 }
 
+// Largest eigenvalue of the symmetric tridiagonal matrix (alpha[0..m-1], beta[0..m-2]) by bisection
+// on the Sturm sequence (host).
+static double tridiag_max_eig(const std::vector<double>& alpha, const std::vector<double>& beta, int m)
+{
+    double lo = alpha[0], hi = alpha[0];
+    for (int i = 0; i < m; ++i) {
+        const double off = (i > 0 ? fabs(beta[i - 1]) : 0.0) + (i + 1 < m ? fabs(beta[i]) : 0.0);
+        if (alpha[i] - off < lo) lo = alpha[i] - off;
+        if (alpha[i] + off > hi) hi = alpha[i] + off;
+    }
+    for (int it = 0; it < 200 && hi - lo > 1e-15 * fabs(hi); ++it) {
+        const double mid = 0.5 * (lo + hi);
+        // number of eigenvalues greater than mid = number of positive terms of the Sturm recurrence
+        int greater = 0;
+        double q = alpha[0] - mid;
+        if (q > 0) ++greater;
+        for (int i = 1; i < m; ++i) {
+            const double den = (fabs(q) < 1e-300) ? (q < 0 ? -1e-300 : 1e-300) : q;
+            q = alpha[i] - mid - beta[i - 1] * beta[i - 1] / den;
+            if (q > 0) ++greater;
+        }
+        if (greater >= 1) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+// a = ||X_c||_2.  Every pass applies X_c^T X_c to a unit vector on the device (k_pi_pass + k_pi_fin: the
+// power-iteration kernel pair).  The passes are driven by a Lanczos recurrence on the host (d-vectors,
+// full reorthogonalisation): the largest Ritz value of the tridiagonal matrix is the best estimate of
+// lambda_max in the span of the iterates v, Av, A^2 v, ... -- never above lambda_max, and it converges in
+// far fewer passes than the plain iteration v <- Av / ||Av|| when the leading singular values are close.
 int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, double* a_out,
                       double* host_scratch)
 {
+    (void)host_scratch;
     const auto& P = pb.P;
     const int d = P.d;
     const int g = pb.L.gs;
     double* mean = pb.setup();              // [d]
     double* v = mean + d;                   // [d]
-    double* scal = v + d;                   // [4]
-    double* part = scal + 4;                // [g][d]
+    double* wdev = v + d;                   // [d]
+    double* part = wdev + d;                // [g][d]
     cudaStream_t st = pb.stream;
 
     if (P.center) {
@@ -155,38 +179,59 @@ int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, dou
         cudaMemsetAsync(mean, 0, sizeof(double) * d, st);
     }
     // seeded Gaussian start, normalized
-    std::vector<double> v0(d);
+    std::vector<std::vector<double>> V;
+    std::vector<double> vk(d), w(d);
     double nrm2 = 0.0;
     for (int j = 0; j < d; ++j) {
         uint64_t a = splitmix64(P.pi_seed * 0x100000001B3ull + 2 * (uint64_t)j);
         uint64_t b = splitmix64(P.pi_seed * 0x100000001B3ull + 2 * (uint64_t)j + 1);
         double u1 = ((double)(a >> 11) + 1.0) / 9007199254740993.0;
         double u2 = (double)(b >> 11) / 9007199254740992.0;
-        v0[j] = sqrt(-2.0 * log(u1)) * cos(6.283185307179586 * u2);
-        nrm2 += v0[j] * v0[j];
+        vk[j] = sqrt(-2.0 * log(u1)) * cos(6.283185307179586 * u2);
+        nrm2 += vk[j] * vk[j];
     }
-    for (int j = 0; j < d; ++j) v0[j] /= sqrt(nrm2);
-    if (cudaMemcpyAsync(v, v0.data(), sizeof(double) * d, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return GEM_NLR_E_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return GEM_NLR_E_CUDA;   // v0 is a local
+    for (int j = 0; j < d; ++j) vk[j] /= sqrt(nrm2);
 
     const size_t smem = sizeof(double) * ((size_t)PI_WARPS * d + 2 * (size_t)d);
     if (smem > 48 * 1024)
         cudaFuncSetAttribute(k_pi_pass, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    const int max_it = P.pi_max_iters > 0 ? P.pi_max_iters : 100;
+    int max_it = P.pi_max_iters > 0 ? P.pi_max_iters : 100;
+    if (max_it > d) max_it = d;             // the Krylov space is exhausted after d steps
     const double tol = P.pi_tol > 0.0 ? P.pi_tol : 1e-7;
+    std::vector<double> alpha, beta;
     double sigma_prev = -1.0, sigma = 0.0;
+    int calm = 0;
     for (int it = 0; it < max_it; ++it) {
+        if (cudaMemcpyAsync(v, vk.data(), sizeof(double) * d, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return GEM_NLR_E_CUDA;
         k_pi_pass<<<g, PI_WARPS * 32, smem, st>>>(X_in, P.n, d, mean, v, part);
-        k_pi_fin<<<1, 256, 0, st>>>(part, g, d, v, scal);
+        k_pi_fin<<<(d + 255) / 256, 256, 0, st>>>(part, g, d, wdev);
         pb.count(2);
-        if (cudaMemcpyAsync(host_scratch, scal, 2 * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        if (cudaMemcpyAsync(w.data(), wdev, sizeof(double) * d, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return GEM_NLR_E_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return GEM_NLR_E_CUDA;
-        sigma = host_scratch[0];
-        if (!isfinite(sigma)) return GEM_NLR_E_NONFINITE;
-        if (sigma_prev >= 0.0 && fabs(sigma - sigma_prev) <= tol * sigma) break;
+        double ak = 0.0;
+        for (int j = 0; j < d; ++j) ak += vk[j] * w[j];
+        if (!isfinite(ak)) return GEM_NLR_E_NONFINITE;
+        alpha.push_back(ak);
+        V.push_back(vk);
+        // w <- w - (projection on all previous Lanczos vectors), twice for numerical orthogonality
+        for (int pass = 0; pass < 2; ++pass)
+            for (const auto& vj : V) {
+                double dot = 0.0;
+                for (int j = 0; j < d; ++j) dot += vj[j] * w[j];
+                for (int j = 0; j < d; ++j) w[j] -= dot * vj[j];
+            }
+        double bk = 0.0;
+        for (int j = 0; j < d; ++j) bk += w[j] * w[j];
+        bk = sqrt(bk);
+        const double theta = tridiag_max_eig(alpha, beta, (int)alpha.size());
+        sigma = sqrt(theta > 0.0 ? theta : 0.0);
+        if (sigma_prev >= 0.0 && fabs(sigma - sigma_prev) <= tol * sigma) { if (++calm >= 2) break; } else calm = 0;
         sigma_prev = sigma;
+        if (!(bk > 1e-14 * (fabs(ak) + 1e-300))) break;   // invariant subspace: the Ritz value is exact
+        beta.push_back(bk);
+        for (int j = 0; j < d; ++j) vk[j] = w[j] / bk;
     }
     if (!(sigma > 0.0)) return GEM_NLR_E_BREAKDOWN;
     *a_out = sigma;

@@ -1,0 +1,102 @@
+"""Full-size parity: the benchmark shapes at their full n, in the launch configuration bench.py
+times (automatic kernel-family selection, library-side setup), one teacher-forced iteration from
+the seeded starting factor compared with the CPU oracle on every entry of U, plus the setup
+(spectral norm, X-hat) and the label read-out.
+
+Config 4 (n = 2e6, d = 768, K = 1000) costs the oracle about 6 TFLOP in FP64 per iteration, so it is
+checked on a reduced-n twin with the same d, K and distribution."""
+import dataclasses
+
+import numpy as np
+import psutil
+import pytest
+import torch
+
+import oracle
+import synth
+import paper_2609_36074_b200 as gem
+
+pytestmark = pytest.mark.gpu
+TOL_U, TOL_F = 1e-4, 1e-5
+
+
+def _rel(a, b):
+    return abs(a - b) / max(abs(b), 1e-300)
+
+
+def _chunked_max_abs_diff(A: np.ndarray, B: np.ndarray, rows: int = 1 << 20) -> float:
+    m = 0.0
+    for lo in range(0, A.shape[0], rows):
+        m = max(m, float(np.abs(A[lo:lo + rows].astype(np.float64) - B[lo:lo + rows]).max()))
+    return m
+
+
+def _run(spec, expect_path=None):
+    n, d, K = spec.n, spec.d, spec.K
+    need = 2.2 * 4 * n * d + 5 * 4 * n * K + (1 << 30)
+    if psutil.virtual_memory().available < need:
+        pytest.skip(f"needs about {need / 2**30:.0f} GiB of host memory")
+    if torch.cuda.mem_get_info()[0] < 4 * n * (d + 2 * K + 8) + (1 << 30):
+        pytest.skip("not enough device memory")
+    hp = synth.default_hparams(K)
+    X, _, _ = synth.make_mixture(spec)
+    a_ref, mean = oracle.spectral_norm(X)
+    rng = np.random.default_rng(7)
+    rows = np.sort(rng.choice(n, size=min(n, 4096), replace=False))
+    X_rows = X[rows].astype(np.float64)
+    U0 = synth.make_u0(n, K, K)
+
+    Xd = torch.from_numpy(X).cuda()
+    del X
+    Ud = torch.from_numpy(U0).cuda()
+    s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"],
+                   T=spec.iters, T_min=spec.iters)
+    if expect_path:
+        assert s.path() == expect_path, s.path()
+
+    # ---- S0: spectral norm by power iteration against the exact Gram eigenvalue; X-hat on sampled rows ----
+    a = s.spectral_norm()
+    assert a <= a_ref * (1 + 1e-9) and _rel(a, a_ref) <= 1e-5, (a, a_ref)
+    Xhat = Xd.cpu().numpy()
+    ref_rows = ((X_rows - mean) / a_ref)
+    assert np.abs(Xhat[rows] - ref_rows).max() <= 2e-5 * np.abs(ref_rows).max()
+
+    # ---- one iteration from (U0, y = 0): both sides on the library's X-hat ----
+    st = oracle.State(Xhat, U0)
+    ref = st.step(K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], spec.iters)
+    rc, info = s.step()
+    assert rc >= 0, (rc, s.last_error())
+    Ug = s.U.cpu().numpy()
+    scale = float(np.abs(st.U).max())
+    err = _chunked_max_abs_diff(Ug, st.U) / scale
+    assert err <= TOL_U, err
+    assert _rel(info["a"], ref["a"]) <= 1e-6 and _rel(info["b"], ref["b"]) <= 1e-6 and _rel(info["h"], ref["h"]) <= 1e-6
+    assert _rel(info["c"], ref["c"]) <= 2e-7 and abs(info["delta_hat"] - ref["delta_hat"]) <= 1e-6
+    assert _rel(info["rho"], ref["rho"]) <= 1e-5 and _rel(info["fhat"], ref["fhat"]) <= TOL_F
+    assert info["dual_applied"] == ref["dual"] and info["stop"] == ref["stop"]
+    yt, t = s.get_state()
+    assert t == 1 and float(np.abs(yt.cpu().numpy() - st.ytilde).max()) <= 1e-9
+
+    # ---- S7: argmax labels; where the two sides differ the row must be a numerical tie ----
+    lab_g = s.labels().cpu().numpy()
+    lab_o = oracle.labels(st.U)
+    diff = np.nonzero(lab_g != lab_o)[0]
+    if diff.size:
+        top_o = st.U[diff, lab_o[diff]].astype(np.float64)
+        alt_o = st.U[diff, lab_g[diff]].astype(np.float64)
+        assert ((top_o - alt_o) <= 2 * TOL_U * scale).all()
+    assert diff.size <= 1e-4 * n
+    s.destroy()
+    return dict(a=a, err=err, label_ties=int(diff.size))
+
+
+@pytest.mark.parametrize("cfg,path", [(2, "ffma"), (3, "tf32x3"), (5, "ffma")])
+def test_full_size_iteration_matches_oracle(cfg, path):
+    out = _run(synth.config(cfg), expect_path=path)
+    print(f"config {cfg}: a={out['a']:.6g} U err={out['err']:.2e} label ties={out['label_ties']}")
+
+
+def test_embedding_shape_reduced_n_twin():
+    """Config 4's d = 768, K = 1000 and unit-sphere data at n = 20,000 (generic kernel family)."""
+    out = _run(dataclasses.replace(synth.config(4), n=20_000, name="embedding-n20000"))
+    print(f"config 4 twin: a={out['a']:.6g} U err={out['err']:.2e} label ties={out['label_ties']}")
