@@ -422,6 +422,119 @@ __global__ void k_labels(const float* __restrict__ U, int64_t n, int r, int32_t*
 }
 
 // ------------------------------------------------------------------------------------------
+// Thread-per-row variants of the vector pass and of the column sums for narrow factors
+// (r = 4 R4 <= 32): a thread reads its whole row with 16-byte loads (consecutive threads read
+// consecutive rows, so a warp still covers one contiguous span) and keeps the row's share of s in
+// registers.  Same outputs as k_rowvec / k_colsum.
+// ------------------------------------------------------------------------------------------
+template <int R4, bool MATERIALIZE>
+__global__ void __launch_bounds__(256)
+k_rowvec_small(float* __restrict__ U, float* __restrict__ ytilde, float* __restrict__ ybar,
+               const Ctl* __restrict__ ctl, const float* __restrict__ p, int64_t n, double gamma,
+               double* __restrict__ part, int ignore_stop)
+{
+    constexpr int R = 4 * R4;
+    if (!ignore_stop && ctl->stopped) return;
+    __shared__ float ssum[8][R];
+    __shared__ double sred[32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float cf = ctl->c_f;
+    const int dual = ctl->dual_pending;
+    float pr[R], sacc[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) { pr[j] = p[j]; sacc[j] = 0.f; }
+    double qq = 0.0, yq = 0.0;
+    for (int64_t row = (int64_t)blockIdx.x * 256 + threadIdx.x; row < n; row += (int64_t)gridDim.x * 256) {
+        float4* up = reinterpret_cast<float4*>(U + row * R);
+        float u[R];
+#pragma unroll
+        for (int c = 0; c < R4; ++c) {
+            const float4 w = up[c];
+            u[4 * c] = cf * w.x; u[4 * c + 1] = cf * w.y; u[4 * c + 2] = cf * w.z; u[4 * c + 3] = cf * w.w;
+        }
+        float dot = 0.f;
+#pragma unroll
+        for (int j = 0; j < R; ++j) dot = fmaf(u[j], pr[j], dot);
+        const float q = dot - 1.0f;
+        float yt = ytilde[row];
+        if (dual) { yt = (float)((double)yt + gamma * (double)q); ytilde[row] = yt; }
+        const float yb = (float)((double)yt + gamma * (double)q);
+        ybar[row] = yb;
+        qq = fma((double)q, (double)q, qq);
+        yq = fma((double)yt, (double)q, yq);
+#pragma unroll
+        for (int j = 0; j < R; ++j) sacc[j] = fmaf(u[j], yb, sacc[j]);
+        if (MATERIALIZE) {
+#pragma unroll
+            for (int c = 0; c < R4; ++c) up[c] = make_float4(u[4 * c], u[4 * c + 1], u[4 * c + 2], u[4 * c + 3]);
+        }
+    }
+    // block partial of s: lanes by butterfly, warps in warp order
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+        const float v = warp_sum(sacc[j]);
+        if (lane == 0) ssum[warp][j] = v;
+    }
+    qq = block_sum<256>(qq, sred);
+    yq = block_sum<256>(yq, sred);
+    double* out = part + (size_t)blockIdx.x * (R + 2);
+    if (threadIdx.x < R) {
+        double v = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += (double)ssum[w][threadIdx.x];
+        out[threadIdx.x] = v;
+    }
+    if (threadIdx.x == 0) { out[R] = qq; out[R + 1] = yq; }
+}
+
+template <int R4>
+__global__ void __launch_bounds__(256)
+k_colsum_small(const float* __restrict__ U, const Ctl* __restrict__ ctl, int64_t n, double* __restrict__ part)
+{
+    constexpr int R = 4 * R4;
+    __shared__ double ssum[8][R];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float cf = ctl->c_f;
+    double acc[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) acc[j] = 0.0;
+    for (int64_t row0 = (int64_t)blockIdx.x * 256 + threadIdx.x; row0 < n; row0 += (int64_t)gridDim.x * 256 * 8) {
+        // eight rows per thread in FP32, then folded into the FP64 running sums
+        float part32[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) part32[j] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int64_t row = row0 + (int64_t)k * gridDim.x * 256;
+            if (row < n) {
+                const float4* up = reinterpret_cast<const float4*>(U + row * R);
+#pragma unroll
+                for (int c = 0; c < R4; ++c) {
+                    const float4 w = up[c];
+                    part32[4 * c] += cf * w.x; part32[4 * c + 1] += cf * w.y;
+                    part32[4 * c + 2] += cf * w.z; part32[4 * c + 3] += cf * w.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < R; ++j) acc[j] += (double)part32[j];
+    }
+#pragma unroll
+    for (int j = 0; j < R; ++j) {
+        const double v = warp_sum(acc[j]);
+        if (lane == 0) ssum[warp][j] = v;
+    }
+    __syncthreads();
+    double* out = part + (size_t)blockIdx.x * (R + 2);
+    if (threadIdx.x < R) {
+        double v = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) v += ssum[w][threadIdx.x];
+        out[threadIdx.x] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Host-side launchers
 // ------------------------------------------------------------------------------------------
 static size_t rv_smem(int r) { return (size_t)RV_WARPS * r * sizeof(double); }
@@ -437,31 +550,82 @@ static void set_rv_attr(int r)
     }
 }
 
+static bool small_r(int r) { return r % 4 == 0 && r >= 4 && r <= 32; }
+static int small_grid(const Problem& pb)
+{
+    int64_t g = (pb.P.n + 255) / 256;
+    if (g > pb.L.gv) g = pb.L.gv;
+    return (int)(g < 1 ? 1 : g);
+}
+
+template <bool MAT>
+static void launch_rowvec_small(const Problem& pb, int grid, int ignore_stop)
+{
+    const auto& P = pb.P;
+#define RV_CASE(R4) case R4: k_rowvec_small<R4, MAT><<<grid, 256, 0, pb.stream>>>(pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, pb.gamma, pb.part1v(), ignore_stop); break;
+    switch (P.r / 4) { RV_CASE(1) RV_CASE(2) RV_CASE(3) RV_CASE(4) RV_CASE(5) RV_CASE(6) RV_CASE(7) RV_CASE(8) default: break; }
+#undef RV_CASE
+}
+
+// Vector pass (optionally applying the pending multiplier to the U buffer); returns the number of
+// per-block partial records it wrote.
+static int launch_rowvec(const Problem& pb, bool materialize, int ignore_stop)
+{
+    const auto& P = pb.P;
+    if (small_r(P.r)) {
+        const int grid = small_grid(pb);
+        if (materialize) launch_rowvec_small<true>(pb, grid, ignore_stop);
+        else launch_rowvec_small<false>(pb, grid, ignore_stop);
+        pb.count();
+        return grid;
+    }
+    set_rv_attr(P.r);
+    if (materialize)
+        k_rowvec<true><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
+            pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
+    else
+        k_rowvec<false><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
+            pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
+    pb.count();
+    return pb.L.gv;
+}
+
+static void launch_fin1_g(const Problem& pb, int mode, int gv);
+
 void launch_init_colsum(const Problem& pb)
 {
     const auto& P = pb.P;
-    set_rv_attr(P.r);
-    k_colsum<<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(pb.U, pb.ctl(), P.n, P.r, pb.part1v());
-    k_fin_colsum<<<1, 256, 0, pb.stream>>>(pb.part1v(), pb.L.gv, P.r, pb.p());
+    int grid = pb.L.gv;
+    if (small_r(P.r)) {
+        grid = small_grid(pb);
+#define CS_CASE(R4) case R4: k_colsum_small<R4><<<grid, 256, 0, pb.stream>>>(pb.U, pb.ctl(), P.n, pb.part1v()); break;
+        switch (P.r / 4) { CS_CASE(1) CS_CASE(2) CS_CASE(3) CS_CASE(4) CS_CASE(5) CS_CASE(6) CS_CASE(7) CS_CASE(8) default: break; }
+#undef CS_CASE
+    } else {
+        set_rv_attr(P.r);
+        k_colsum<<<grid, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(pb.U, pb.ctl(), P.n, P.r, pb.part1v());
+    }
+    k_fin_colsum<<<1, 256, 0, pb.stream>>>(pb.part1v(), grid, P.r, pb.p());
     pb.count(2);
 }
 
 void launch_vector_pass(const Problem& pb)
 {
+    launch_rowvec(pb, false, 0);
+}
+
+static void launch_fin1_g(const Problem& pb, int mode, int gv)
+{
     const auto& P = pb.P;
-    set_rv_attr(P.r);
-    k_rowvec<false><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
-        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), 0);
+    k_fin1<<<1, 256, 0, pb.stream>>>(pb.ctl(), pb.part1v(), gv, pb.red1(), pb.L.nred1, P.r, P.n,
+                                     P.alpha, pb.gamma, P.eps_c, P.T_min, pb.s(), pb.alpha_s(),
+                                     pb.hist(), mode);
     pb.count();
 }
 
 void launch_fin1(const Problem& pb, int mode)
 {
-    const auto& P = pb.P;
-    k_fin1<<<1, 256, 0, pb.stream>>>(pb.ctl(), pb.part1v(), pb.L.gv, pb.red1(), pb.L.nred1, P.r, P.n,
-                                     P.alpha, pb.gamma, P.eps_c, P.T_min, pb.s(), pb.alpha_s(),
-                                     pb.hist(), mode);
-    pb.count();
+    launch_fin1_g(pb, mode, small_r(pb.P.r) ? small_grid(pb) : pb.L.gv);
 }
 
 void launch_fin2(const Problem& pb, int gx, int gy, int cols_per)
@@ -496,26 +660,18 @@ void launch_generic_pass2_kernel(const Problem& pb)
 
 void launch_tail(const Problem& pb)
 {
-    const auto& P = pb.P;
-    set_rv_attr(P.r);
-    k_rowvec<true><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
-        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), 1);
-    pb.count();
-    launch_fin1(pb, 1);
+    const int g = launch_rowvec(pb, true, 1);
+    launch_fin1_g(pb, 1, g);
 }
 
 void launch_objective(const Problem& pb)
 {
-    const auto& P = pb.P;
-    set_rv_attr(P.r);
     // Called after the tail: no gate is pending and the multiplier is 1, so the vector pass has
     // no side effect on the dual.  The objective is also wanted after a stop, so the stop flag
     // is ignored.
-    k_rowvec<false><<<pb.L.gv, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(
-        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), 1);
-    pb.count();
+    const int g = launch_rowvec(pb, false, 1);
     launch_generic_pass1(pb, 1);
-    launch_fin1(pb, 2);
+    launch_fin1_g(pb, 2, g);
 }
 
 void launch_labels(const Problem& pb, int32_t* labels)

@@ -80,6 +80,66 @@ k_pi_pass(const float* __restrict__ X, int64_t n, int d, const double* __restric
     }
 }
 
+// Same pass for d = 4 LPR NCH (LPR a power of two <= 32): LPR lanes share a row, each lane owns NCH
+// 16-byte chunks (columns 4 (sub + k LPR) .. +3), so a warp streams 32 / LPR rows per step with
+// 16-byte loads and keeps its column accumulators in registers.
+template <int LPR, int NCH>
+__global__ void __launch_bounds__(PI_WARPS * 32)
+k_pi_pass_vec(const float* __restrict__ X, int64_t n, const double* __restrict__ mean,
+              const double* __restrict__ v, double* __restrict__ part)
+{
+    constexpr int D = 4 * LPR * NCH;
+    constexpr int RPW = 32 / LPR;                       // rows per warp and step
+    __shared__ double sv[D], smean[D];
+    __shared__ double sacc[PI_WARPS][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rg = lane / LPR;
+    for (int j = threadIdx.x; j < D; j += blockDim.x) { sv[j] = v[j]; smean[j] = mean[j]; }
+    __syncthreads();
+    double acc[NCH * 4];
+#pragma unroll
+    for (int k = 0; k < NCH * 4; ++k) acc[k] = 0.0;
+    const int64_t stride = (int64_t)gridDim.x * PI_WARPS * RPW;
+    // The loop bound is the warp's base row, identical in all 32 lanes: the shuffles below are
+    // executed by the whole warp even when only some of its RPW rows exist.
+    for (int64_t rbase = ((int64_t)blockIdx.x * PI_WARPS + warp) * RPW; rbase < n; rbase += stride) {
+        const int64_t row = rbase + rg;
+        const bool valid = row < n;
+        double xc[NCH * 4];
+        double z = 0.0;
+#pragma unroll
+        for (int k = 0; k < NCH; ++k) {
+            const int col = 4 * (sub + k * LPR);
+            const float4 x = valid ? __ldcs(reinterpret_cast<const float4*>(X + row * D + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            xc[4 * k + 0] = valid ? (double)x.x - smean[col + 0] : 0.0;
+            xc[4 * k + 1] = valid ? (double)x.y - smean[col + 1] : 0.0;
+            xc[4 * k + 2] = valid ? (double)x.z - smean[col + 2] : 0.0;
+            xc[4 * k + 3] = valid ? (double)x.w - smean[col + 3] : 0.0;
+            z = fma(xc[4 * k + 0], sv[col + 0], z); z = fma(xc[4 * k + 1], sv[col + 1], z);
+            z = fma(xc[4 * k + 2], sv[col + 2], z); z = fma(xc[4 * k + 3], sv[col + 3], z);
+        }
+#pragma unroll
+        for (int o = 1; o < LPR; o <<= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+#pragma unroll
+        for (int k = 0; k < NCH * 4; ++k) acc[k] = fma(z, xc[k], acc[k]);
+    }
+    // fold the row groups of the warp (lanes with equal sub), then the warps in warp order
+#pragma unroll
+    for (int k = 0; k < NCH * 4; ++k) {
+        double t = acc[k];
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (rg == 0) sacc[warp][4 * (sub + (k >> 2) * LPR) + (k & 3)] = t;
+    }
+    __syncthreads();
+    for (int j = threadIdx.x; j < D; j += blockDim.x) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < PI_WARPS; ++w) t += sacc[w][j];
+        part[(size_t)blockIdx.x * D + j] = t;
+    }
+}
+
 // w = sum of the per-CTA partials in CTA order (the result of one application of X_c^T X_c to v).
 __global__ void __launch_bounds__(256)
 k_pi_fin(const double* __restrict__ part, int g, int d, double* __restrict__ w)
@@ -204,7 +264,13 @@ int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, dou
     for (int it = 0; it < max_it; ++it) {
         if (cudaMemcpyAsync(v, vk.data(), sizeof(double) * d, cudaMemcpyHostToDevice, st) != cudaSuccess)
             return GEM_NLR_E_CUDA;
-        k_pi_pass<<<g, PI_WARPS * 32, smem, st>>>(X_in, P.n, d, mean, v, part);
+        switch (d) {
+#define PI_CASE(DD, LPR, NCH) case DD: k_pi_pass_vec<LPR, NCH><<<g, PI_WARPS * 32, 0, st>>>(X_in, P.n, mean, v, part); break;
+            PI_CASE(16, 4, 1) PI_CASE(32, 8, 1) PI_CASE(64, 16, 1) PI_CASE(128, 32, 1) PI_CASE(256, 32, 2)
+            PI_CASE(384, 32, 3) PI_CASE(512, 32, 4)
+#undef PI_CASE
+            default: k_pi_pass<<<g, PI_WARPS * 32, smem, st>>>(X_in, P.n, d, mean, v, part); break;
+        }
         k_pi_fin<<<(d + 255) / 256, 256, 0, st>>>(part, g, d, wdev);
         pb.count(2);
         if (cudaMemcpyAsync(w.data(), wdev, sizeof(double) * d, cudaMemcpyDeviceToHost, st) != cudaSuccess)
