@@ -71,8 +71,9 @@ typedef struct {
     int32_t  pi_max_iters;  /* power-iteration cap for ||X_c||_2 (<=0: 100)                      */
     double   pi_tol;        /* stop when |sigma_k - sigma_{k-1}| <= pi_tol * sigma_k (<=0: 1e-7) */
     uint64_t pi_seed;       /* seed of the starting vector                                       */
-    int32_t  precision;     /* contraction arithmetic: 0 FP32 FFMA, 1 3xTF32 tensor cores,       */
-                            /* 2 the generic FFMA kernels whatever the shape (cross-checks),     */
+    int32_t  precision;     /* contraction arithmetic: 0 FP32 FFMA, 1 3xTF32 tcgen05 tensor      */
+                            /* cores, 2 the generic FFMA kernels whatever the shape              */
+                            /* (cross-checks), 3 3xTF32 warp-level MMA (skinny shapes),          */
                             /* -1 let the library choose by shape                                */
     int32_t  history;       /* 1: keep one gem_nlr_iter_info per iteration in the workspace      */
 } gem_nlr_params;

@@ -21,7 +21,7 @@ static bool valid_params(const gem_nlr_params& P)
     if (P.r > 7168 || P.d > 2816) return false;       // shared-memory accumulators of the vector / setup passes
     if (!(P.alpha > 0.f) || !(P.beta > 0.f)) return false;
     if (P.T < 0 || P.T_min < 0 || P.eps_d < 0.0 || P.eps_c < 0.0) return false;
-    if (P.precision < -1 || P.precision > 2) return false;
+    if (P.precision < -1 || P.precision > 3) return false;
     return true;
 }
 
@@ -83,6 +83,7 @@ struct gem_nlr {
     double* host_scratch;  // pinned
     const char* path;
     bool use_ffma;         // first (and, unless use_tc, second) product by the FFMA family
+    bool use_mma;          // with use_ffma: the warp-level TF32 tensor-core kernels of that family
     bool use_tc;           // second product by the tcgen05 family
     bool use_tc1;          // first product by the tcgen05 family
     FfmaPlan ffma;
@@ -156,7 +157,8 @@ static void launch_iteration(gem_nlr_t* h)
         tc1_launch_first(h->pb, h->tc1);
         red1_fused_launch(h->pb, h->tc1.grid, 0);
     } else if (h->use_ffma) {
-        ffma_launch_first(h->pb, h->ffma, 0);
+        if (h->use_mma) mma_launch_first(h->pb, h->ffma, 0);
+        else ffma_launch_first(h->pb, h->ffma, 0);
     } else {
         launch_vector_pass(h->pb);
         launch_generic_pass1(h->pb, 0);
@@ -165,6 +167,7 @@ static void launch_iteration(gem_nlr_t* h)
     if (prof) cudaEventRecord(e[1], h->pb.stream);
     if (h->use_tc || h->use_ffma) {
         if (h->use_tc) tc_launch_second(h->pb, h->tc);
+        else if (h->use_mma) mma_launch_second(h->pb, h->ffma);
         else ffma_launch_second(h->pb, h->ffma);
         if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
         return;
@@ -237,13 +240,19 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     h->path = "generic";
     h->err[0] = 0;
     h->pb.launches = &h->launches;
-    // Kernel families by shape.  precision 2: generic only.  precision 0: FFMA family where a shape is
+    // Kernel families by shape.  precision 3: the warp-level TF32 (mma.sync, 3-product split) kernels
+    // where instantiated, else generic; precision -1 prefers them to the FFMA kernels for d >= 64.
+    // precision 2: generic only.  precision 0: FFMA family where a shape is
     // instantiated, else generic.  precision 1: tensor cores wherever they are available.  precision -1:
     // FFMA for the skinny shapes (r <= 16: there the FP32 pipes keep up and the tensor-core path would
     // issue one MMA triple per 8 rows for 16 useful columns), tensor cores for r >= 32, else generic.
     const bool want_ffma = params->precision != 2;
+    const bool want_mma = params->precision == 3 || params->precision == -1;
     const bool want_tc = params->precision == 1 || (params->precision == -1 && params->r >= 32);
-    if (want_ffma && ffma_plan(h->pb, &h->ffma)) {
+    if (want_mma && mma_plan(h->pb, &h->ffma)) {
+        h->use_ffma = h->use_mma = true;
+        h->path = "mma.tf32x3";
+    } else if (want_ffma && params->precision != 3 && ffma_plan(h->pb, &h->ffma)) {
         h->use_ffma = true;
         h->path = "ffma";
     }

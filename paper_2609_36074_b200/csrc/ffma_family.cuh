@@ -21,4 +21,10 @@ void red1_fused_launch(const Problem& pb, int g, int mode);
 // Fused second product, statistics, scalar step (multiplier, movement, gate, p).
 void ffma_launch_second(const Problem& pb, const FfmaPlan& plan);
 
+
+// Same interface for the warp-level tensor-core kernels (kernels_mma.cu: mma.sync TF32, 3-product split).
+bool mma_plan(const Problem& pb, FfmaPlan* plan);
+void mma_launch_first(const Problem& pb, const FfmaPlan& plan, int mode);
+void mma_launch_second(const Problem& pb, const FfmaPlan& plan);
+
 }  // namespace gemnlr

@@ -265,16 +265,57 @@ FFMA_SHAPES = [(5000, 32, 8), (3333, 128, 16), (2500, 64, 16), (4097, 64, 8), (3
 def test_ffma_family_teacher_forced(n, d, K):
     _, _, Xhat, U0 = _problem(n, d, K)
     hp = synth.default_hparams(K)
-    s = make_solver(Xhat, U0, K, hp)
+    s = make_solver(Xhat, U0, K, hp, precision=0)
     assert s.path() == "ffma"
     s.destroy()
-    recs = teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U)
+    recs = teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U, solver_kw=dict(precision=0))
+    _check_recs(recs)
+
+
+def _check_recs(recs):
     for rec in recs:
         assert rec["a"] <= 1e-6 and rec["b"] <= 1e-6 and rec["h"] <= 1e-6, rec
         assert rec["c"] <= 2e-7 and rec["delta"] <= 1e-6, rec
         assert rec["rho"] <= 1e-5 and rec["fhat"] <= TOL_F, rec
         assert rec["dual"][0] == rec["dual"][1] and rec["stop"][0] == rec["stop"][1], rec
         assert rec["yt"] <= 1e-9, rec
+
+
+# ---- warp-level tensor-core kernels of the same family (mma.sync TF32, 3-product split) ----------
+MMA_SHAPES = [(3333, 128, 16), (2500, 64, 16), (4097, 64, 8), (1024, 128, 8), (40003, 128, 16), (50001, 64, 16)]
+
+
+@pytest.mark.parametrize("n,d,K", MMA_SHAPES)
+def test_mma_family_teacher_forced(n, d, K):
+    _, _, Xhat, U0 = _problem(n, d, K)
+    hp = synth.default_hparams(K)
+    s = make_solver(Xhat, U0, K, hp)          # automatic selection takes these kernels for d >= 64
+    assert s.path() == "mma.tf32x3"
+    s.destroy()
+    _check_recs(teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U, solver_kw=dict(precision=3)))
+
+
+@pytest.mark.parametrize("n,d,K", [(9000, 128, 16), (12000, 64, 8)])
+def test_mma_family_trajectory_matches_oracle(n, d, K):
+    _, _, Xhat, U0 = _problem(n, d, K)
+    hp = dict(synth.default_hparams(K), eps_d=0.2)
+    T = 40
+    outs = []
+    for _ in range(2):
+        s = make_solver(Xhat, U0, K, hp, T=T, precision=3, history=1)
+        assert s.path() == "mma.tf32x3"
+        rc, info, iters = s.run()
+        assert rc == gem.ITER_CAP and iters == T
+        outs.append((s.U.cpu().numpy().copy(), s.get_state()[0].cpu().numpy().copy(), info, s.history(T)))
+        s.destroy()
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][2] == outs[1][2]
+    Uo, yto, infoo, iterso, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"],
+                                           T, hp["T_min"])
+    U, yt, info, hist = outs[0]
+    assert any(h["dual_applied"] for h in hist)
+    assert u_err(U, Uo) <= TOL_U
+    assert np.abs(yt - yto).max() <= 1e-4 * max(np.abs(yto).max(), 1e-30)
+    assert rel(info["rho"], infoo["rho"]) <= 1e-4 and abs(info["delta_hat"] - infoo["delta_hat"]) <= 1e-6
 
 
 @pytest.mark.parametrize("n,d,K", [(20000, 32, 8), (9000, 128, 16)])
