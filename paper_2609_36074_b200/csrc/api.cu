@@ -249,7 +249,8 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     const bool want_ffma = params->precision != 2;
     const bool want_mma = params->precision == 3 || params->precision == -1;
     const bool want_tc = params->precision == 1 || (params->precision == -1 && params->r >= 32);
-    if (want_mma && mma_plan(h->pb, &h->ffma)) {
+    // the wide-factor mma.sync shapes (r > 16) are slower than the tcgen05 pair: explicit request only
+    if (want_mma && (params->precision == 3 || params->r <= 16) && mma_plan(h->pb, &h->ffma)) {
         h->use_ffma = h->use_mma = true;
         h->path = "mma.tf32x3";
     } else if (want_ffma && params->precision != 3 && ffma_plan(h->pb, &h->ffma)) {

@@ -21,46 +21,10 @@
 #include "pipeline.cuh"
 #include "tc_common.cuh"
 #include "ffma_family.cuh"
+#include "mma_common.cuh"
 
 namespace gemnlr {
 namespace mma {
-
-constexpr int NCW = 8;
-constexpr int NTHREADS = (NCW + 1) * 32;
-
-template <int TM>
-__device__ __forceinline__ uint32_t x_chunk_off(int rl, int c)
-{
-    return (uint32_t)((c >> 3) * (TM * 128) + rl * 128 + (((c & 7) ^ (rl & 7)) << 4));
-}
-
-__device__ __forceinline__ void mma_tf32(float* c, const uint32_t* a, uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t* r)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-
-__device__ __forceinline__ float lds32(uint32_t addr)
-{
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo)
-{
-    const float h = tf32_hi(x);
-    hi = __float_as_uint(h);
-    lo = __float_as_uint(x - h);
-}
 
 // ------------------------------------------------------------------------------------------------
 template <int D, int R, int TM, int NST>
@@ -197,22 +161,34 @@ k_pass1_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ U
                     split_tf32(lds32(us + (uint32_t)(ka * R + 8 * nn + g) * 4), bh[nn][0], bl[nn][0]);
                     split_tf32(lds32(us + (uint32_t)(kb * R + 8 * nn + g) * 4), bh[nn][1], bl[nn][1]);
                 }
+                // A fragment (16 features x 8 rows): a0 = x[row ka][f g], a1 = x[row ka][f g + 8],
+                //                                    a2 = x[row kb][f g], a3 = x[row kb][f g + 8].
+                // M tiles go in pairs and the three products are issued product by product, so that
+                // MMAs on the same accumulator are 2 NT instructions apart (their latency is ~4 issue slots).
+                constexpr int MP = (MT >= 2) ? 2 : 1;
 #pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    // A fragment (16 features x 8 rows): a0 = x[row ka][f g], a1 = x[row ka][f g + 8],
-                    //                                    a2 = x[row kb][f g], a3 = x[row kb][f g + 8]
-                    const int f0 = 16 * m + g, f1 = f0 + 8;
-                    uint32_t ah[4], al[4];
-                    split_tf32(lds32(xs + x_chunk_off<TM>(ka, f0 >> 2) + (f0 & 3) * 4), ah[0], al[0]);
-                    split_tf32(lds32(xs + x_chunk_off<TM>(ka, f1 >> 2) + (f1 & 3) * 4), ah[1], al[1]);
-                    split_tf32(lds32(xs + x_chunk_off<TM>(kb, f0 >> 2) + (f0 & 3) * 4), ah[2], al[2]);
-                    split_tf32(lds32(xs + x_chunk_off<TM>(kb, f1 >> 2) + (f1 & 3) * 4), ah[3], al[3]);
+                for (int m0 = 0; m0 < MT; m0 += MP) {
+                    uint32_t ah[MP][4], al[MP][4];
 #pragma unroll
-                    for (int nn = 0; nn < NT; ++nn) {
-                        mma_tf32(acc[m][nn], ah, bh[nn][0], bh[nn][1]);
-                        mma_tf32(acc[m][nn], al, bh[nn][0], bh[nn][1]);
-                        mma_tf32(acc[m][nn], ah, bl[nn][0], bl[nn][1]);
+                    for (int mm = 0; mm < MP; ++mm) {
+                        const int f0 = 16 * (m0 + mm) + g, f1 = f0 + 8;
+                        split_tf32(lds32(xs + x_chunk_off<TM>(ka, f0 >> 2) + (f0 & 3) * 4), ah[mm][0], al[mm][0]);
+                        split_tf32(lds32(xs + x_chunk_off<TM>(ka, f1 >> 2) + (f1 & 3) * 4), ah[mm][1], al[mm][1]);
+                        split_tf32(lds32(xs + x_chunk_off<TM>(kb, f0 >> 2) + (f0 & 3) * 4), ah[mm][2], al[mm][2]);
+                        split_tf32(lds32(xs + x_chunk_off<TM>(kb, f1 >> 2) + (f1 & 3) * 4), ah[mm][3], al[mm][3]);
                     }
+#pragma unroll
+                    for (int mm = 0; mm < MP; ++mm)
+#pragma unroll
+                        for (int nn = 0; nn < NT; ++nn) mma_tf32(acc[m0 + mm][nn], ah[mm], bh[nn][0], bh[nn][1]);
+#pragma unroll
+                    for (int mm = 0; mm < MP; ++mm)
+#pragma unroll
+                        for (int nn = 0; nn < NT; ++nn) mma_tf32(acc[m0 + mm][nn], al[mm], bh[nn][0], bh[nn][1]);
+#pragma unroll
+                    for (int mm = 0; mm < MP; ++mm)
+#pragma unroll
+                        for (int nn = 0; nn < NT; ++nn) mma_tf32(acc[m0 + mm][nn], ah[mm], bl[nn][0], bl[nn][1]);
                 }
             }
             fence_proxy_async();
@@ -370,11 +346,12 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
             const float yb0 = v0 ? ybar[row0] : 0.f;
             const float yb1 = v1 ? ybar[row1] : 0.f;
             mbar_wait(full_bar(s), (it / NST) & 1, &abort_flag, ctl);
-            float acc[NT][4];
+            // one accumulator per product (hi*hi, lo*hi, hi*lo) and N tile: 3 NT independent MMA chains
+            float acc[NT][4], acc1[NT][4], acc2[NT][4];
 #pragma unroll
             for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
-                for (int k = 0; k < 4; ++k) acc[nn][k] = 0.f;
+                for (int k = 0; k < 4; ++k) acc[nn][k] = acc1[nn][k] = acc2[nn][k] = 0.f;
 #pragma unroll 4
             for (int ks = 0; ks < D / 8; ++ks) {
                 uint32_t a[4], ah[4], al[4], bh[4], bl[4];
@@ -384,12 +361,16 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
 #pragma unroll
                 for (int k = 0; k < 4; ++k) split_tf32(__uint_as_float(a[k]), ah[k], al[k]);
 #pragma unroll
-                for (int nn = 0; nn < NT; ++nn) {
-                    mma_tf32(acc[nn], ah, bh[2 * nn], bh[2 * nn + 1]);
-                    mma_tf32(acc[nn], al, bh[2 * nn], bh[2 * nn + 1]);
-                    mma_tf32(acc[nn], ah, bl[2 * nn], bl[2 * nn + 1]);
-                }
+                for (int nn = 0; nn < NT; ++nn) mma_tf32(acc[nn], ah, bh[2 * nn], bh[2 * nn + 1]);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) mma_tf32(acc1[nn], al, bh[2 * nn], bh[2 * nn + 1]);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn) mma_tf32(acc2[nn], ah, bl[2 * nn], bl[2 * nn + 1]);
             }
+#pragma unroll
+            for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) acc[nn][k] += acc1[nn][k] + acc2[nn][k];
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar(s));
 
@@ -521,6 +502,7 @@ using S_128_8  = Shape<128, 8,  128, 3,  3>;
 
 }  // namespace mma
 
+
 bool mma_plan(const Problem& pb, FfmaPlan* pl)
 {
     const int d = pb.P.d, r = pb.P.r;
@@ -529,8 +511,16 @@ bool mma_plan(const Problem& pb, FfmaPlan* pl)
     else if (d == 64 && r == 16) id = 1;
     else if (d == 64 && r == 8) id = 2;
     else if (d == 128 && r == 8) id = 3;
+    // wide factors: r in a multiple-of-4 window below the instantiated N-tile count
+    if (id < 0 && r % 4 == 0) {
+        const int nt = (r + 7) / 8;
+        if (d == 64 && nt == 13) id = 100;
+        else if (d == 64 && nt == 8) id = 101;
+        else if (d == 32 && nt == 13) id = 102;
+    }
     if (id < 0 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
     pl->shape_id = id;
+    if (id >= 100) return mmaw_plan(pb, pl);
     using namespace mma;
     switch (id) {
         case 0: return S_128_16::plan(pb, pl);
@@ -543,6 +533,7 @@ bool mma_plan(const Problem& pb, FfmaPlan* pl)
 
 void mma_launch_first(const Problem& pb, const FfmaPlan& pl, int mode)
 {
+    if (pl.shape_id >= 100) { mmaw_pass1(pb, pl); pb.count(1); red1_fused_launch(pb, pl.g1, mode); return; }
     using namespace mma;
     switch (pl.shape_id) {
         case 0: S_128_16::pass1(pb, pl); break;
@@ -556,6 +547,7 @@ void mma_launch_first(const Problem& pb, const FfmaPlan& pl, int mode)
 
 void mma_launch_second(const Problem& pb, const FfmaPlan& pl)
 {
+    if (pl.shape_id >= 100) { mmaw_pass2(pb, pl); pb.count(1); return; }
     using namespace mma;
     switch (pl.shape_id) {
         case 0: S_128_16::pass2(pb, pl); break;

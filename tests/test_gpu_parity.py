@@ -295,7 +295,21 @@ def test_mma_family_teacher_forced(n, d, K):
     _check_recs(teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U, solver_kw=dict(precision=3)))
 
 
-@pytest.mark.parametrize("n,d,K", [(9000, 128, 16), (12000, 64, 8)])
+# wide factors: r in N tiles of 8 columns, the last one partly filled (r = 100, 60) or full (104, 64)
+MMAW_SHAPES = [(3000, 64, 100), (2050, 64, 64), (5000, 32, 104), (3001, 64, 60), (30011, 64, 100)]
+
+
+@pytest.mark.parametrize("n,d,K", MMAW_SHAPES)
+def test_mma_wide_family_teacher_forced(n, d, K):
+    _, _, Xhat, U0 = _problem(n, d, K)
+    hp = synth.default_hparams(K)
+    s = make_solver(Xhat, U0, K, hp, precision=3)
+    assert s.path() == "mma.tf32x3"
+    s.destroy()
+    _check_recs(teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U, solver_kw=dict(precision=3)))
+
+
+@pytest.mark.parametrize("n,d,K", [(9000, 128, 16), (12000, 64, 8), (8000, 64, 100)])
 def test_mma_family_trajectory_matches_oracle(n, d, K):
     _, _, Xhat, U0 = _problem(n, d, K)
     hp = dict(synth.default_hparams(K), eps_d=0.2)
