@@ -59,7 +59,8 @@ Layout make_layout(const gem_nlr_params& P)
     size_t p2 = sizeof(double) * (size_t)L.g2x * L.g2y * (3 + G2_RT);
     size_t p2_fast = sizeof(double) * (size_t)kSMs * 4 * (4 + (size_t)r);
     L.part2 = take(p2 > p2_fast ? p2 : p2_fast);
-    L.red1 = take(sizeof(double) * (size_t)L.nred1);
+    // generic family: nred1 block shares; fused reduction: one share per 16 entries of a record + r + 2 sums
+    L.red1 = take(sizeof(double) * ((size_t)L.nred1 + ((size_t)d * r + r + 2 + 15) / 16 + r + 2 + 8));
     L.setup = take(sizeof(double) * (3 * (size_t)d + 4 + (size_t)L.gs * d));
     L.hist = take(P.history ? sizeof(gem_nlr_iter_info) * (size_t)(P.T > 0 ? P.T : 1) : 0);
     L.xhat = take(P.x_inplace ? 0 : sizeof(float) * (size_t)n * d);

@@ -142,6 +142,11 @@ k_pass1_ffma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
         float preg[CPL];
 #pragma unroll
         for (int c = 0; c < CPL; ++c) preg[c] = p[v_sub * CPL + c];
+        float yt_next;
+        {
+            const int64_t row_f = (int64_t)blockIdx.x * TM + warp * RW + v_row;
+            yt_next = (row_f < n) ? ytilde[row_f] : 0.f;
+        }
         int it = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
             const int s = it % NST;
@@ -151,7 +156,13 @@ k_pass1_ffma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
             const int rl_v = warp * RW + v_row;
             const int64_t row_v = t * TM + rl_v;
             const bool valid = row_v < n;
-            float yt = valid ? ytilde[row_v] : 0.f;
+            // ytilde of this tile was requested one tile ago (its DRAM latency would otherwise stall
+            // every warp once per tile); request the next tile's now
+            float yt = yt_next;
+            {
+                const int64_t row_n = row_v + (int64_t)gridDim.x * TM;
+                yt_next = (row_n < n) ? ytilde[row_n] : 0.f;
+            }
             mbar_wait(full_bar(s), (it / NST) & 1, &abort_flag, ctl);
 
             // ---- vector phase on the warp's own rows ----
@@ -269,9 +280,12 @@ k_pass1_ffma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
     }
 }
 
-// Theta[e] = FP32(sum_g part[g][e]) in ascending g (four interleaved slices combined in order).
-// The last block to finish also sums s, sum q^2, sum ytilde q and ||Theta||_F^2 and runs the
-// scalar step that finishes the previous iteration (fin1_scalars).
+// Sums the g per-CTA records [d*r Theta | r s | sum q^2 | sum ytilde q] (FP64) entry by entry: a block
+// takes 16 entries x 16 interleaved slices of the records (independent loads, combined in slice
+// order, so the result does not depend on scheduling).  Theta is stored as FP32 with the block's
+// share of ||Theta||_F^2; the r + 2 trailing sums go to a small FP64 array.  The last block to
+// finish turns those into s, alpha s and the scalar step that finishes the previous iteration.
+constexpr int RED1_EB = 16;
 __global__ void __launch_bounds__(256)
 k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, Ctl* __restrict__ ctl,
              float* __restrict__ theta, double* __restrict__ red, float* __restrict__ s,
@@ -279,21 +293,31 @@ k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, 
              gem_nlr_iter_info* __restrict__ hist, int mode, int ignore_stop)
 {
     if (!ignore_stop && ctl->stopped) return;
-    __shared__ double sl[4][64];
+    __shared__ double sl[16][RED1_EB];
     __shared__ double sred[32];
     __shared__ int is_last;
-    const int e_local = threadIdx.x & 63, slice = threadIdx.x >> 6;
-    const int e = blockIdx.x * 64 + e_local;
+    double* extra = red + gridDim.x;           // [r + 2] behind the per-block ||Theta||^2 shares
+    const int e_local = threadIdx.x & (RED1_EB - 1), slice = threadIdx.x >> 4;
+    const int e = blockIdx.x * RED1_EB + e_local;
     double v = 0.0;
-    if (e < dr)
-        for (int b = slice; b < g; b += 4) v += part[(size_t)b * stride + e];
+    if (e < stride) {
+        const double* src = part + e;
+#pragma unroll 4
+        for (int b = slice; b < g; b += 16) v += __ldcg(src + (size_t)b * stride);
+    }
     sl[slice][e_local] = v;
     __syncthreads();
     double t2 = 0.0;
-    if (slice == 0 && e < dr) {
-        const double tot = ((sl[0][e_local] + sl[1][e_local]) + sl[2][e_local]) + sl[3][e_local];
-        theta[e] = (float)tot;
-        t2 = tot * tot;
+    if (slice == 0 && e < stride) {
+        double tot = sl[0][e_local];
+#pragma unroll
+        for (int k = 1; k < 16; ++k) tot += sl[k][e_local];
+        if (e < dr) {
+            theta[e] = (float)tot;
+            t2 = tot * tot;
+        } else {
+            extra[e - dr] = tot;
+        }
     }
     t2 = block_sum<256>(t2, sred);
     if (threadIdx.x == 0) {
@@ -306,24 +330,16 @@ k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, 
     if (!is_last) return;
     __threadfence();
     for (int j = threadIdx.x; j < r; j += blockDim.x) {
-        double acc = 0.0;
-        for (int b = 0; b < g; ++b) acc += part[(size_t)b * stride + dr + j];
-        const float sf = (float)acc;
+        const float sf = (float)__ldcg(extra + j);
         s[j] = sf;
         alpha_s[j] = alpha * sf;
     }
-    double qq = 0.0, yq = 0.0, tt = 0.0;
-    for (int b = threadIdx.x; b < g; b += blockDim.x) {
-        qq += part[(size_t)b * stride + dr + r];
-        yq += part[(size_t)b * stride + dr + r + 1];
-    }
+    double tt = 0.0;
     for (int b = threadIdx.x; b < (int)gridDim.x; b += blockDim.x) tt += __ldcg(red + b);
-    qq = block_sum<256>(qq, sred);
-    yq = block_sum<256>(yq, sred);
     tt = block_sum<256>(tt, sred);
     if (threadIdx.x == 0) {
         ctl->counter[0] = 0;
-        fin1_scalars(ctl, qq, yq, tt, n, gamma, eps_c, T_min, hist, mode);
+        fin1_scalars(ctl, __ldcg(extra + r), __ldcg(extra + r + 1), tt, n, gamma, eps_c, T_min, hist, mode);
     }
 }
 
@@ -590,7 +606,7 @@ bool ffma_plan(const Problem& pb, FfmaPlan* pl)
 void red1_fused_launch(const Problem& pb, int g, int mode)
 {
     const int dr = pb.P.d * pb.P.r;
-    ffma::k_red1_fused<<<(dr + 63) / 64, 256, 0, pb.stream>>>(
+    ffma::k_red1_fused<<<(dr + pb.P.r + 2 + ffma::RED1_EB - 1) / ffma::RED1_EB, 256, 0, pb.stream>>>(
         pb.part1(), g, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
         pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0);
     pb.count(1);

@@ -101,6 +101,11 @@ k_pass1_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ U
         float preg[CPL];
 #pragma unroll
         for (int c = 0; c < CPL; ++c) preg[c] = p[v_sub * CPL + c];
+        float yt_next;
+        {
+            const int64_t row_f = (int64_t)blockIdx.x * TM + warp * RW + v_row;
+            yt_next = (row_f < n) ? ytilde[row_f] : 0.f;
+        }
         int it = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
             const int s = it % NST;
@@ -109,7 +114,13 @@ k_pass1_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ U
             const int rl_v = warp * RW + v_row;
             const int64_t row_v = t * TM + rl_v;
             const bool valid = row_v < n;
-            float yt = valid ? ytilde[row_v] : 0.f;
+            // ytilde of this tile was requested one tile ago (its DRAM latency would otherwise stall
+            // every warp once per tile); request the next tile's now
+            float yt = yt_next;
+            {
+                const int64_t row_n = row_v + (int64_t)gridDim.x * TM;
+                yt_next = (row_n < n) ? ytilde[row_n] : 0.f;
+            }
             mbar_wait(full_bar(s), (it / NST) & 1, &abort_flag, ctl);
 
             // ---- vector phase on the warp's own rows (u written back into the stage) ----
