@@ -155,12 +155,19 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         const int box = lane >> 3, c = lane & 7;           // U chunk (32 columns) and logical 16-byte piece inside it
         const int col0 = box * 32 + 4 * c;                 // first of this lane's 4 columns of u
         const float4 p4 = *reinterpret_cast<const float4*>(sp + col0);
+        // ytilde of this warp's eight rows (lane k < 8 holds row tw + 4 k) is requested one of the team's
+        // stages ahead, so its DRAM latency is not paid inside the stage
+        float yt_next = 0.f;
+        if (team < my_stages) {
+            const int64_t row_f = (g_lo + team) * TR + tw + 4 * (lane & 7);
+            if (lane < 8 && row_f < n) yt_next = ytilde[row_f];
+        }
         for (int g = team; g < my_stages; g += 2) {
             const int s = g % NSR, l = g % NLO;
             const int64_t srow0 = (g_lo + g) * TR;
-            // ytilde of this warp's eight rows (lane k < 8 holds row tw + 4 k), fetched before the waits
             const int64_t myrow = srow0 + tw + 4 * (lane & 7);
-            float yt_l = (lane < 8 && myrow < n) ? ytilde[myrow] : 0.f;
+            float yt_l = yt_next;
+            yt_next = (g + 2 < my_stages && lane < 8 && myrow + 2 * TR < n) ? ytilde[myrow + 2 * TR] : 0.f;
             float yb_l = 0.f;
             mbar_wait(full(s), (g / NSR) & 1, &abort_flag, ctl);
             if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
