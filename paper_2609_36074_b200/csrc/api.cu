@@ -48,7 +48,7 @@ Layout make_layout(const gem_nlr_params& P)
     L.s = take(sizeof(float) * r);
     L.alpha_s = take(sizeof(float) * r);
     L.theta = take(sizeof(float) * (size_t)d * r);
-    L.thimg = take(sizeof(float) * 2 * (size_t)((d + 31) / 32 * 32) * ((r + 15) / 16 * 16));
+    L.thimg = take(sizeof(float) * 2 * (size_t)((d + 31) / 32 * 32) * (r > 256 ? (r + 255) / 256 * 256 : (r + 15) / 16 * 16));
     L.ytilde = take(sizeof(float) * (size_t)n);
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families
@@ -87,9 +87,11 @@ struct gem_nlr {
     bool use_mma;          // with use_ffma: the warp-level TF32 tensor-core kernels of that family
     bool use_tc;           // second product by the tcgen05 family
     bool use_tc1;          // first product by the tcgen05 family
+    bool use_tcg;          // second product by the tiled tcgen05 kernel (wide d, r)
     FfmaPlan ffma;
     TcPlan tc;
     Tc1Plan tc1;
+    TcgPlan tcg;
     char err[256];
     int64_t launches;      // kernels launched by this handle
     int pi_iters;          // power iterations taken by the last setup
@@ -166,8 +168,9 @@ static void launch_iteration(gem_nlr_t* h)
         launch_fin1(h->pb, 0);
     }
     if (prof) cudaEventRecord(e[1], h->pb.stream);
-    if (h->use_tc || h->use_ffma) {
-        if (h->use_tc) tc_launch_second(h->pb, h->tc);
+    if (h->use_tc || h->use_ffma || h->use_tcg) {
+        if (h->use_tcg) tcg_launch_second(h->pb, h->tcg);
+        else if (h->use_tc) tc_launch_second(h->pb, h->tc);
         else if (h->use_mma) mma_launch_second(h->pb, h->ffma);
         else ffma_launch_second(h->pb, h->ffma);
         if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
@@ -267,6 +270,10 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
                 h->use_tc1 = true;
                 h->path = "tf32x3";
             }
+        }
+        else if (tcg_plan(h->pb, &h->tcg, img)) {
+            h->use_tcg = true;
+            h->path = "generic+tf32x3.tiled";
         }
     }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||

@@ -1,0 +1,389 @@
+// Tiled 3xTF32 tcgen05 second product for wide problems (d and r too large for the resident-Theta
+// kernel: the embedding-sized shape d = 768, r = 1000):
+//   acc = X-hat Theta ;  W = [U + 2 alpha acc - alpha (ybar p^T + 1 s^T)]_+ in place ;  FP64 a, b, h ;
+//   column sums of W                                               (Eq. "entrywise-fusion", Algorithm 2 call 4)
+//
+// Work item = (128-row tile, 256-column block).  The K loop streams d in chunks of 16 features:
+// a stage holds the X-hat box (128 rows x 64 bytes, TMA with the 64-byte swizzle = K-major UMMA
+// operand) and the matching boxes of the pre-split Theta^T images (256 columns x 64 bytes, hi and
+// lo, already swizzled in global memory, one bulk copy each).  With M = 128, N = 256 a TF32
+// tcgen05.mma runs at the tensor pipe's full rate, and the accumulator (256 TMEM columns) is
+// double-buffered, so the epilogue of one item overlaps the MMAs of the next.
+//
+//   warp 0       producer (TMA / bulk copies, 4-stage ring)
+//   warp 1       MMA issuer: per chunk 2 k-steps x 3 products; commits free the stage
+//   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); thread = row; 16 columns at a
+//                time: tcgen05.ld, old U entries straight from global memory (each thread reads and
+//                writes whole 32-byte sectors of its row), FP64 statistics; column sums by a
+//                shuffle transpose-reduce, combined across the four quarters in fixed order
+//   warps 10-13  split of the X-hat box into hi (in place) and lo (second ring)
+// Every mbarrier wait is bounded (error status GEM_NLR_E_TIMEOUT, kernel runs to its end, TMEM freed).
+#include "nlr_common.cuh"
+#include "device_utils.cuh"
+#include "fin_logic.cuh"
+#include "pipeline.cuh"
+#include "tc_common.cuh"
+#include "tc_family.cuh"
+
+namespace gemnlr {
+namespace tcg {
+
+constexpr int TILE_M = 128;
+constexpr int NBLK = 256;                     // columns per item = MMA N
+constexpr int KC = 16;                        // features per chunk (64-byte rows)
+constexpr int A_BOX = TILE_M * KC * 4;        // 8 KB
+constexpr int B_BOX = NBLK * KC * 4;          // 16 KB
+constexpr int STAGE = A_BOX + 2 * B_BOX;      // 40 KB: X-hat raw/hi, Theta^T hi, Theta^T lo
+constexpr int NS = 4, NLO = 3;
+constexpr int NEPI = 8;                       // epilogue warps
+constexpr int NTHREADS = (2 + NEPI + 4) * 32;
+constexpr size_t SMEM_RING = (size_t)NS * STAGE + (size_t)NLO * A_BOX;
+
+// Shared-memory matrix descriptor, K-major operand with the 64-byte swizzle: 64-byte rows, groups
+// of 8 rows 512 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_sw64(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+    d |= (uint64_t)(16u >> 4) << 16;
+    d |= (uint64_t)(512u >> 4) << 32;
+    d |= (uint64_t)1 << 46;          // version
+    d |= (uint64_t)4 << 61;          // SWIZZLE_64B
+    return d;
+}
+
+// Theta (d x r, FP32 row-major) -> hi / lo images of Theta^T as K-major 64-byte-swizzled boxes:
+// box (kb, cb) = features 16 kb .. 16 kb + 15 of columns 256 cb .. 256 cb + 255 (zero beyond r).
+__global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, int NCB, const Ctl* __restrict__ ctl,
+                                 float* __restrict__ img_hi, float* __restrict__ img_lo)
+{
+    if (ctl->stopped) return;
+    const int64_t total = (int64_t)d * NCB * NBLK;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int j = (int)(e / (NCB * NBLK)), k = (int)(e % (NCB * NBLK));     // feature, column
+        const float v = (k < r) ? theta[(size_t)j * r + k] : 0.f;
+        const float hi = tf32_hi(v);
+        const int kb = j >> 4, jj = j & 15, c = jj >> 2, w = jj & 3;
+        const int cb = k >> 8, kr = k & 255;
+        const size_t off = ((size_t)(kb * NCB + cb) * NBLK + kr) * KC + (size_t)(((c ^ ((kr >> 1) & 3)) << 2) + w);
+        img_hi[off] = hi;
+        img_lo[off] = v - hi;
+    }
+}
+
+// Column sums of a 32-row x 16-column block held one row per lane (v[16]): after the exchange
+// lane l holds the sum of column 8 b4 + 4 b3 + 2 b2 + b1 (bits of l) over the 32 rows.
+__device__ __forceinline__ float colsum16(const float* v, int lane)
+{
+    float a8[8], a4[4], a2[2], a1;
+    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float send = h16 ? v[i] : v[i + 8];
+        const float keep = h16 ? v[i + 8] : v[i];
+        a8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float send = h8 ? a8[i] : a8[i + 4];
+        const float keep = h8 ? a8[i + 4] : a8[i];
+        a4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float send = h4 ? a4[i] : a4[i + 2];
+        const float keep = h4 ? a4[i + 2] : a4[i];
+        a2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    {
+        const float send = h2 ? a2[0] : a2[1];
+        const float keep = h2 ? a2[1] : a2[0];
+        a1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    return a1 + __shfl_xor_sync(0xffffffffu, a1, 1);
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ img_hi,
+            const float* __restrict__ img_lo, float* __restrict__ U, const float* __restrict__ ybar,
+            const float* __restrict__ p, const float* __restrict__ alpha_s, Ctl* __restrict__ ctl, int64_t n, int d,
+            int r, int NCB, float alpha, int K, double eps_d, double* __restrict__ part, float* __restrict__ p_out)
+{
+    if (ctl->stopped) return;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t bars[3 * NS + NLO + 4];
+    __shared__ uint32_t abort_flag;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ double sred[32];
+    __shared__ int is_last;
+    __shared__ double sc;
+    __shared__ int sok;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int KB = d / KC;
+    const int RP = NCB * NBLK;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t stage0 = smem_base;
+    const uint32_t lo0 = stage0 + (uint32_t)NS * STAGE;
+    unsigned char* tail = smem + SMEM_RING;
+    float* sp = reinterpret_cast<float*>(tail);                         // [RP] p
+    float* sas = sp + RP;                                               // [RP] alpha s
+    double* scol = reinterpret_cast<double*>(sas + RP);                 // [RP] running column sums of W
+    float* stmp = reinterpret_cast<float*>(scol + RP);                  // [2][4][NBLK] per-quarter column sums of an item
+
+    const uint32_t bar0 = smem_u32(bars);
+    auto xfull = [&](int s) { return bar0 + 8u * s; };
+    auto xsplit = [&](int s) { return bar0 + 8u * (NS + s); };
+    auto xfree = [&](int s) { return bar0 + 8u * (2 * NS + s); };
+    auto lofree = [&](int l) { return bar0 + 8u * (3 * NS + l); };
+    auto accfull = [&](int a) { return bar0 + 8u * (3 * NS + NLO + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (3 * NS + NLO + 2 + a); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(xfull(s), 1); mbar_init(xsplit(s), 4); mbar_init(xfree(s), 1); }
+        for (int l = 0; l < NLO; ++l) mbar_init(lofree(l), 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), NEPI); }
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    for (int j = threadIdx.x; j < RP; j += NTHREADS) {
+        sp[j] = (j < r) ? p[j] : 0.f;
+        sas[j] = (j < r) ? alpha_s[j] : 0.f;
+        scol[j] = 0.0;
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    const int64_t n_tiles = (n + TILE_M - 1) / TILE_M;
+    const int64_t n_items = n_tiles * NCB;
+    const float cf = ctl->c_f;
+    const float two_alpha = 2.0f * alpha;
+    double sa = 0.0, sb = 0.0, sh = 0.0;
+
+    if (warp == 0) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            int64_t g = 0;
+            for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x) {
+                const int64_t t = w / NCB;
+                const int cb = (int)(w % NCB);
+                const int row0 = (int)(t * TILE_M);
+                for (int kb = 0; kb < KB; ++kb, ++g) {
+                    const int s = (int)(g % NS);
+                    if (g >= NS) mbar_wait(xfree(s), (uint32_t)((g / NS) - 1) & 1, &abort_flag, ctl);
+                    const uint32_t dst = stage0 + (uint32_t)s * STAGE;
+                    const size_t boff = ((size_t)(kb * NCB + cb) * NBLK) * KC;
+                    mbar_expect_tx(xfull(s), STAGE);
+                    tma_load_2d(dst, &tmX, kb * KC, row0, xfull(s));
+                    bulk_load_1d(dst + A_BOX, img_hi + boff, B_BOX, xfull(s));
+                    bulk_load_1d(dst + A_BOX + B_BOX, img_lo + boff, B_BOX, xfull(s));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_tf32(TILE_M, NBLK, 0, 0);
+            int64_t g = 0;
+            int i = 0;
+            for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x, ++i) {
+                const int a = i & 1;
+                if (i >= 2) mbar_wait(accfree(a), (uint32_t)((i >> 1) - 1) & 1, &abort_flag, ctl);
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(a * NBLK);
+                for (int kb = 0; kb < KB; ++kb, ++g) {
+                    const int s = (int)(g % NS), l = (int)(g % NLO);
+                    mbar_wait(xsplit(s), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
+                    tc_fence_after();
+                    const uint32_t st = stage0 + (uint32_t)s * STAGE;
+                    const uint64_t da_hi = umma_desc_sw64(st), da_lo = umma_desc_sw64(lo0 + (uint32_t)l * A_BOX);
+                    const uint64_t db_hi = umma_desc_sw64(st + A_BOX), db_lo = umma_desc_sw64(st + A_BOX + B_BOX);
+                    // a k-step (8 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
+#pragma unroll
+                    for (int ks = 0; ks < KC / 8; ++ks)
+                        umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
+                                     (kb | ks) ? 1u : 0u);
+                    umma_commit(xfree(s));
+                    umma_commit(lofree(l));
+                }
+                umma_commit(accfull(a));
+            }
+        }
+    } else if (warp >= 2 + NEPI) {
+        // ------------------------------ split: X-hat box -> hi (in place), lo ------------------------------
+        const int st = threadIdx.x - (2 + NEPI) * 32;   // 0..127
+        int64_t g = 0;
+        for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x) {
+            for (int kb = 0; kb < KB; ++kb, ++g) {
+                const int s = (int)(g % NS), l = (int)(g % NLO);
+                mbar_wait(xfull(s), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
+                if (g >= NLO) mbar_wait(lofree(l), (uint32_t)((g / NLO) - 1) & 1, &abort_flag, ctl);
+                const uint32_t hi_a = stage0 + (uint32_t)s * STAGE, lo_a = lo0 + (uint32_t)l * A_BOX;
+                float4 xin[A_BOX / 16 / 128];
+#pragma unroll
+                for (int k = 0; k < A_BOX / 16 / 128; ++k) xin[k] = lds128(hi_a + (uint32_t)(k * 128 + st) * 16);
+#pragma unroll
+                for (int k = 0; k < A_BOX / 16 / 128; ++k) {
+                    const uint32_t off = (uint32_t)(k * 128 + st) * 16;
+                    const float4 x = xin[k];
+                    const float4 hi = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
+                    sts128(hi_a + off, hi);
+                    sts128(lo_a + off, make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w));
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(xsplit(s));
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (warps 2..9) ------------------------------
+        const int q = warp & 3;                           // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                 // columns 128 half .. 128 half + 127 of the item
+        const int rl = q * 32 + lane;
+        const int et = (warp - 2) * 32 + lane;            // 0..255 among the epilogue threads
+        // column held by this lane after colsum16 (within a 16-column group)
+        const int ccol = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+        int i = 0;
+        for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
+            const int a = i & 1;
+            const int64_t t = w / NCB;
+            const int cb = (int)(w % NCB);
+            const int64_t row = t * TILE_M + rl;
+            const bool valid = row < n;
+            const float nay = valid ? -alpha * ybar[row] : 0.f;
+            float* urow = U + (valid ? row : 0) * (int64_t)r;
+            float* my_tmp = stmp + (size_t)(a * 4 + q) * NBLK + half * 128;
+            mbar_wait(accfull(a), (uint32_t)(i >> 1) & 1, &abort_flag, ctl);
+            tc_fence_after();
+#pragma unroll 1
+            for (int jj = 0; jj < 8; ++jj) {
+                const int col0 = cb * NBLK + half * 128 + jj * 16;
+                float acc[16], wn[16];
+                float4 w4[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    w4[c] = (valid && col0 + 4 * c < r) ? __ldcs(reinterpret_cast<const float4*>(urow + col0 + 4 * c))
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NBLK + half * 128 + jj * 16), acc);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float4 p4 = *reinterpret_cast<const float4*>(sp + col0 + 4 * c);
+                    const float4 s4 = *reinterpret_cast<const float4*>(sas + col0 + 4 * c);
+                    const float wold[4] = {w4[c].x, w4[c].y, w4[c].z, w4[c].w};
+                    const float pj[4] = {p4.x, p4.y, p4.z, p4.w};
+                    const float sj[4] = {s4.x, s4.y, s4.z, s4.w};
+                    const bool live = valid && (col0 + 4 * c < r);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float u = live ? cf * wold[e] : 0.f;
+                        float v = fmaf(two_alpha, acc[4 * c + e], u);
+                        v = fmaf(nay, pj[e], v);
+                        v -= sj[e];
+                        const float wv = live ? fmaxf(v, 0.f) : 0.f;
+                        const double wd = (double)wv, ud = (double)u;
+                        sa = fma(wd, wd, sa);
+                        sb = fma(ud, ud, sb);
+                        sh = fma(wd, ud, sh);
+                        wn[4 * c + e] = wv;
+                    }
+                    if (live)
+                        *reinterpret_cast<float4*>(urow + col0 + 4 * c) = make_float4(wn[4 * c], wn[4 * c + 1], wn[4 * c + 2], wn[4 * c + 3]);
+                }
+                const float cs = colsum16(wn, lane);
+                if ((lane & 1) == 0) my_tmp[jj * 16 + ccol] = cs;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(accfree(a));
+            // the four quarters of a column, combined in fixed order by the thread that owns the column
+            named_bar_sync(1, NEPI * 32);
+            {
+                const float* t4 = stmp + (size_t)(a * 4) * NBLK + et;
+                const double v = (((double)t4[0] + (double)t4[NBLK]) + (double)t4[2 * NBLK]) + (double)t4[3 * NBLK];
+                scol[cb * NBLK + et] += v;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+
+    // ---- CTA partial: a, b, h and the column sums of W ----
+    const int PS = 4 + r;
+    sa = block_sum<NTHREADS>(sa, sred);
+    sb = block_sum<NTHREADS>(sb, sred);
+    sh = block_sum<NTHREADS>(sh, sred);
+    double* out = part + (size_t)blockIdx.x * PS;
+    if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; out[2] = sh; out[3] = 0.0; }
+    for (int j = threadIdx.x; j < r; j += NTHREADS) out[4 + j] = scol[j];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned prev = atomicAdd(&ctl->counter[1], 1u);
+        is_last = (prev == gridDim.x - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int G = gridDim.x;
+    double a = 0.0, b = 0.0, hh = 0.0;
+    for (int i = threadIdx.x; i < G; i += NTHREADS) {
+        a += __ldcg(part + (size_t)i * PS + 0);
+        b += __ldcg(part + (size_t)i * PS + 1);
+        hh += __ldcg(part + (size_t)i * PS + 2);
+    }
+    a = block_sum<NTHREADS>(a, sred);
+    b = block_sum<NTHREADS>(b, sred);
+    hh = block_sum<NTHREADS>(hh, sred);
+    if (threadIdx.x == 0) {
+        double c;
+        sok = fin2_scalars(ctl, a, b, hh, K, eps_d, &c) ? 1 : 0;
+        sc = c;
+        ctl->counter[1] = 0;
+    }
+    __syncthreads();
+    if (!sok) return;
+    for (int j = threadIdx.x; j < r; j += NTHREADS) {
+        double v = 0.0;
+        for (int i = 0; i < G; ++i) v += __ldcg(part + (size_t)i * PS + 4 + j);
+        p_out[j] = (float)(sc * v);
+    }
+}
+
+}  // namespace tcg
+
+bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
+{
+    const int d = pb.P.d, r = pb.P.r;
+    if (d % tcg::KC != 0 || r % 4 != 0 || r < 16 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
+    const int NCB = (r + tcg::NBLK - 1) / tcg::NBLK;
+    const int RP = NCB * tcg::NBLK;
+    if (RP > 2048) return false;
+    pl->NCB = NCB;
+    pl->smem2 = tcg::SMEM_RING + (size_t)RP * (4 + 4 + 8) + (size_t)2 * 4 * tcg::NBLK * 4 + 1024;
+    if (pl->smem2 > 227 * 1024 - 1024) return false;
+    pl->img_hi = img_storage;
+    pl->img_lo = img_storage + (size_t)d * RP;
+    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tcg::TILE_M, tcg::KC, false, 64)) return false;
+    const int64_t items = (pb.P.n + tcg::TILE_M - 1) / tcg::TILE_M * NCB;
+    pl->g2 = (int)(items < kSMs ? items : kSMs);
+    if (cudaFuncSetAttribute(tcg::k_pass2_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
+        return false;
+    return true;
+}
+
+void tcg_launch_second(const Problem& pb, const TcgPlan& pl)
+{
+    const int d = pb.P.d, r = pb.P.r;
+    tcg::k_theta_images64<<<kSMs * 4, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NCB, pb.ctl(), pl.img_hi, pl.img_lo);
+    tcg::k_pass2_tcg<<<pl.g2, tcg::NTHREADS, pl.smem2, pb.stream>>>(
+        pl.tmX, pl.img_hi, pl.img_lo, pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NCB,
+        pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
+    pb.count(2);
+}
+
+}  // namespace gemnlr

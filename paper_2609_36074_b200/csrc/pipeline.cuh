@@ -106,7 +106,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, float4 v)
 // atom32, 32-byte atoms: 32-byte chunk index XOR row mod 4 -- the layout MN-major TF32 UMMA operands
 // need), no swizzle otherwise.  Out-of-range elements read as zero.
 // Returns false if the driver entry point is missing or the encode fails.
-bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int cols, int box_rows,
-                        int box_cols, bool atom32 = false);
+bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int cols, int box_rows, int box_cols,
+                        bool atom32 = false, int swizzle_bytes = 0);
 
 }  // namespace gemnlr

@@ -41,3 +41,20 @@ bool tc1_plan(const Problem& pb, Tc1Plan* plan);
 void tc1_launch_first(const Problem& pb, const Tc1Plan& plan);
 
 }  // namespace gemnlr
+
+namespace gemnlr {
+
+// Tiled second product for wide problems (kernels_tcg.cu): d a multiple of 16, r a multiple of 4 up to
+// 2048; Theta^T images of 2 * d * (r rounded up to 256) floats.
+struct TcgPlan {
+    alignas(64) CUtensorMap tmX;   // X-hat boxes: 128 rows x 16 features, 64-byte swizzle
+    int NCB;                       // 256-column blocks
+    int g2;
+    size_t smem2;
+    float* img_hi;
+    float* img_lo;
+};
+bool tcg_plan(const Problem& pb, TcgPlan* plan, float* img_storage);
+void tcg_launch_second(const Problem& pb, const TcgPlan& plan);
+
+}  // namespace gemnlr

@@ -54,3 +54,41 @@ def test_tc_trajectory_matches_oracle_and_is_reproducible(n, d, K):
     Uo, _, infoo, _, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, hp["T_min"])
     assert u_err(outs[0][0], Uo) <= TOL_U
     assert rel(outs[0][1]["rho"], infoo["rho"]) <= 1e-4
+
+
+# ---- tiled tcgen05 second product (wide d and r: 256-column blocks, d streamed in 16-feature chunks) ----
+# one and several column blocks, r not a multiple of 16, ragged last row tile, more items than CTAs
+TCG_SHAPES = [(3000, 48, 300), (2049, 768, 1000), (5000, 64, 520), (21000, 32, 260)]
+
+
+@pytest.mark.parametrize("n,d,K", TCG_SHAPES)
+def test_tiled_tc_second_product_teacher_forced(n, d, K):
+    Xhat, U0 = _problem(n, d, K)
+    hp = synth.default_hparams(K)
+    s = make_solver(Xhat, U0, K, hp, precision=1)
+    assert "tf32x3.tiled" in s.path(), s.path()
+    s.destroy()
+    recs = teacher_forced_steps(Xhat, U0, K, hp, steps=2, tol_u=TOL_U, solver_kw=dict(precision=1))
+    for rec in recs:
+        assert rec["a"] <= 1e-6 and rec["b"] <= 1e-6 and rec["h"] <= 1e-6, rec
+        assert rec["c"] <= 2e-7 and rec["delta"] <= 1e-6, rec
+        assert rec["rho"] <= 1e-5 and rec["fhat"] <= TOL_F, rec
+        assert rec["dual"][0] == rec["dual"][1] and rec["stop"][0] == rec["stop"][1], rec
+
+
+def test_tiled_tc_trajectory_is_reproducible_and_matches_oracle():
+    n, d, K = 4000, 64, 300
+    Xhat, U0 = _problem(n, d, K)
+    hp = dict(synth.default_hparams(K), eps_d=0.2)
+    T = 12
+    outs = []
+    for _ in range(2):
+        s = make_solver(Xhat, U0, K, hp, T=T, precision=1)
+        rc, info, iters = s.run()
+        assert rc == gem.ITER_CAP and iters == T, (rc, s.last_error())
+        outs.append((s.U.cpu().numpy().copy(), info))
+        s.destroy()
+    assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    Uo, _, infoo, _, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, hp["T_min"])
+    assert u_err(outs[0][0], Uo) <= TOL_U
+    assert rel(outs[0][1]["rho"], infoo["rho"]) <= 1e-4
