@@ -52,7 +52,7 @@ Layout make_layout(const gem_nlr_params& P)
     L.ytilde = take(sizeof(float) * (size_t)n);
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families
-    size_t p1 = sizeof(double) * (size_t)L.g1x * d * r;
+    size_t p1 = sizeof(double) * (size_t)(L.g1x > 8 || r <= 256 ? L.g1x : 8) * d * r;   // r > 256: up to 8 row ranges of the tiled tcgen05 first product
     size_t p1_fast = ((size_t)d * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)d * r + r + 4) : 0;
     L.part1 = take(p1 > p1_fast ? p1 : p1_fast);
     L.part1v = take(sizeof(double) * (size_t)L.gv * (r + 2));
@@ -92,6 +92,8 @@ struct gem_nlr {
     TcPlan tc;
     Tc1Plan tc1;
     TcgPlan tcg;
+    Tcg1Plan tcg1;
+    bool use_tcg1;         // first product by the tiled tcgen05 kernel (vector pass separate)
     char err[256];
     int64_t launches;      // kernels launched by this handle
     int pi_iters;          // power iterations taken by the last setup
@@ -164,7 +166,8 @@ static void launch_iteration(gem_nlr_t* h)
         else ffma_launch_first(h->pb, h->ffma, 0);
     } else {
         launch_vector_pass(h->pb);
-        launch_generic_pass1(h->pb, 0);
+        if (h->use_tcg1) tcg_launch_first(h->pb, h->tcg1);
+        else launch_generic_pass1(h->pb, 0);
         launch_fin1(h->pb, 0);
     }
     if (prof) cudaEventRecord(e[1], h->pb.stream);
@@ -274,6 +277,10 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
         else if (tcg_plan(h->pb, &h->tcg, img)) {
             h->use_tcg = true;
             h->path = "generic+tf32x3.tiled";
+            if (tcg1_plan(h->pb, &h->tcg1)) {
+                h->use_tcg1 = true;
+                h->path = "tf32x3.tiled";
+            }
         }
     }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||

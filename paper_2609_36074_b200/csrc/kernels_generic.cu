@@ -647,6 +647,13 @@ void launch_generic_pass1(const Problem& pb, int ignore_stop)
     pb.count(2);
 }
 
+void launch_red1(const Problem& pb, int g, int ignore_stop)
+{
+    k_red1<<<pb.L.nred1, 256, 0, pb.stream>>>(pb.part1(), g, (int64_t)pb.P.d * pb.P.r, pb.ctl(), pb.theta(),
+                                             pb.red1(), ignore_stop);
+    pb.count(1);
+}
+
 void launch_generic_pass2_kernel(const Problem& pb)
 {
     const auto& P = pb.P;

@@ -354,6 +354,167 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
     }
 }
 
+
+// ================================================================================================
+// First product for the same wide problems:  Theta = X-hat^T (c_f W)  as Theta^T tiles.
+//
+// Work item (one CTA each, all resident at once) = (128 columns of U, up to 256 features, one of
+// NSPLIT contiguous row ranges).  The contraction runs over the data rows, so both operands are
+// MN-major: TMA boxes of 16 rows x 32 columns with the 128-byte swizzle of 32-byte atoms (A = 4 boxes
+// of U, B = up to 8 boxes of X-hat per stage).  Two teams of four warps take alternate stages and
+// rewrite the boxes as hi (in place; U scaled by the pending multiplier first) and lo (second ring);
+// the MMA issuer runs 2 k-steps x 3 products per stage into one of two TMEM accumulators, which is
+// handed to the epilogue every FLUSH stages and folded into the FP64 partial of this row range
+// (layout [feature][column] like the generic first product, so the same reduction kernel follows).
+// The row-local vector work cannot be fused here (a CTA sees 128 of the r columns): it runs as the
+// separate vector pass before this kernel.
+// ================================================================================================
+constexpr int TR1 = 16;                        // rows per stage (2 k-steps)
+constexpr int CH1 = TR1 * 128;                 // one box: 16 rows x 32 floats = 2 KB
+constexpr int NS1 = 4, NLO1 = 4;
+constexpr int FLUSH1 = 256;                    // stages per accumulation period (4096 rows)
+constexpr int NTH1 = 14 * 32;                  // producer, MMA, 4 epilogue, 8 split warps
+
+__global__ void __launch_bounds__(NTH1, 1)
+k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU, Ctl* __restrict__ ctl,
+            int64_t n, int d, int r, int NMT, int NNB, int NSPLIT, double* __restrict__ part)
+{
+    if (ctl->stopped) return;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t bars[3 * NS1 + NLO1 + 4];
+    __shared__ uint32_t abort_flag;
+    __shared__ uint32_t tmem_base_s;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // item of this CTA
+    const int mt = blockIdx.x % NMT, nb = (blockIdx.x / NMT) % NNB, sp = blockIdx.x / (NMT * NNB);
+    const int f0 = nb * 256;
+    const int Nb = (d - f0 < 256) ? d - f0 : 256;          // features of this item (multiple of 32)
+    const int NBX = Nb / 32;
+    const int STAGE1 = (4 + 8) * CH1;                       // U boxes then up to 8 X-hat boxes
+
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t raw0 = smem_base, lo0 = raw0 + (uint32_t)NS1 * STAGE1;
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto split = [&](int s) { return bar0 + 8u * (NS1 + s); };
+    auto rawfree = [&](int s) { return bar0 + 8u * (2 * NS1 + s); };
+    auto lofree = [&](int l) { return bar0 + 8u * (3 * NS1 + l); };
+    auto accfull = [&](int a) { return bar0 + 8u * (3 * NS1 + NLO1 + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (3 * NS1 + NLO1 + 2 + a); };
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS1; ++s) { mbar_init(full(s), 1); mbar_init(split(s), 4); mbar_init(rawfree(s), 1); }
+        for (int l = 0; l < NLO1; ++l) mbar_init(lofree(l), 1);
+        for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4); }
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_s;
+
+    // contiguous block of stages of this row range
+    const int64_t n_stages = (n + TR1 - 1) / TR1;
+    const int64_t base_cnt = n_stages / NSPLIT, rem_cnt = n_stages % NSPLIT;
+    const int64_t g_lo = (int64_t)sp * base_cnt + (sp < rem_cnt ? sp : rem_cnt);
+    const int my_stages = (int)(base_cnt + (sp < rem_cnt ? 1 : 0));
+    const int n_periods = (my_stages + FLUSH1 - 1) / FLUSH1;
+    const float cf = ctl->c_f;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int g = 0; g < my_stages && !abort_flag; ++g) {
+                const int s = g % NS1;
+                if (g >= NS1) mbar_wait(rawfree(s), ((g / NS1) - 1) & 1, &abort_flag, ctl);
+                const int row0 = (int)((g_lo + g) * TR1);
+                const uint32_t dst = raw0 + (uint32_t)s * STAGE1;
+                mbar_expect_tx(full(s), (uint32_t)(4 + NBX) * CH1);
+                for (int c = 0; c < 4; ++c) tma_load_2d(dst + c * CH1, &tmU, mt * 128 + c * 32, row0, full(s));
+                for (int b = 0; b < NBX; ++b) tma_load_2d(dst + (4 + b) * CH1, &tmX, f0 + b * 32, row0, full(s));
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_tf32(128, Nb, 1, 1);
+            for (int g = 0; g < my_stages && !abort_flag; ++g) {
+                const int s = g % NS1, l = g % NLO1;
+                const int period = g / FLUSH1, a = period & 1, in_period = g % FLUSH1;
+                if (in_period == 0 && period >= 2) mbar_wait(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
+                mbar_wait(split(s), (g / NS1) & 1, &abort_flag, ctl);
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(a * 256);
+                const uint32_t hi_s = raw0 + (uint32_t)s * STAGE1, lo_s = lo0 + (uint32_t)l * STAGE1;
+                // chunks are CH1 bytes apart (LBO); 4-row swizzle periods of 512 bytes along K (SBO); a k-step is 1 KB
+                const uint64_t da_hi = umma_desc_sw128_atom32(hi_s, CH1, 512), da_lo = umma_desc_sw128_atom32(lo_s, CH1, 512);
+                const uint64_t db_hi = umma_desc_sw128_atom32(hi_s + 4 * CH1, CH1, 512);
+                const uint64_t db_lo = umma_desc_sw128_atom32(lo_s + 4 * CH1, CH1, 512);
+#pragma unroll
+                for (int ks = 0; ks < TR1 / 8; ++ks)
+                    umma_tf32_x3(tacc, da_hi + 64 * ks, da_lo + 64 * ks, db_hi + 64 * ks, db_lo + 64 * ks, idesc,
+                                 (in_period | ks) ? 1u : 0u);
+                umma_commit(rawfree(s));
+                umma_commit(lofree(l));
+                if (in_period == FLUSH1 - 1 || g == my_stages - 1) umma_commit(accfull(a));
+            }
+        }
+    } else if (warp >= 6) {
+        // ------------------------------ split (two teams on alternate stages) ------------------------------
+        const int vw = warp - 6, team = vw >> 2;
+        const int tt = (vw & 3) * 32 + lane;               // 0..127 inside the team
+        const int nq = (4 + NBX) * (CH1 / 16) / 128;       // float4 per thread and stage (U boxes first)
+        for (int g = team; g < my_stages; g += 2) {
+            const int s = g % NS1, l = g % NLO1;
+            mbar_wait(full(s), (g / NS1) & 1, &abort_flag, ctl);
+            if (g >= NLO1) mbar_wait(lofree(l), ((g / NLO1) - 1) & 1, &abort_flag, ctl);
+            const uint32_t hi_s = raw0 + (uint32_t)s * STAGE1, lo_s = lo0 + (uint32_t)l * STAGE1;
+#pragma unroll 4
+            for (int k = 0; k < nq; ++k) {
+                const uint32_t off = (uint32_t)(k * 128 + tt) * 16;
+                float4 x = lds128(hi_s + off);
+                if (k < 4) { x.x *= cf; x.y *= cf; x.z *= cf; x.w *= cf; }      // the 4 U boxes: u = c_f w
+                const float4 h = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
+                sts128(hi_s + off, h);
+                sts128(lo_s + off, make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w));
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(split(s));
+        }
+    } else {
+        // ------------------------------ epilogue: FP64 fold of the accumulator ------------------------------
+        // thread = column j of U (TMEM lane); entry (feature f, column j) of this row range's partial
+        const int q4 = warp & 3;
+        const int j = mt * 128 + q4 * 32 + lane;
+        double* const out = part + (size_t)sp * ((size_t)d * r);
+        for (int period = 0; period < n_periods; ++period) {
+            const int a = period & 1;
+            mbar_wait(accfull(a), (period >> 1) & 1, &abort_flag, ctl);
+            tc_fence_after();
+            for (int c = 0; c * 16 < Nb; ++c) {
+                float v[16];
+                tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * 256 + c * 16), v);
+                if (j < r) {
+                    double* o = out + (size_t)(f0 + c * 16) * r + j;
+                    double prev[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) prev[k] = (period == 0) ? 0.0 : __ldcg(o + (size_t)k * r);
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) o[(size_t)k * r] = prev[k] + (double)v[k];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(accfree(a));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
 }  // namespace tcg
 
 bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
@@ -374,6 +535,33 @@ bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
     if (cudaFuncSetAttribute(tcg::k_pass2_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
         return false;
     return true;
+}
+
+bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
+{
+    const int d = pb.P.d, r = pb.P.r;
+    if (d % 32 != 0 || r % 4 != 0 || r < 16 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
+    pl->NMT = (r + 127) / 128;
+    pl->NNB = (d + 255) / 256;
+    const int tiles = pl->NMT * pl->NNB;
+    if (tiles > kSMs) return false;
+    pl->NSPLIT = kSMs / tiles;
+    if (pl->NSPLIT > 8) pl->NSPLIT = 8;                     // partial records are sized for 8 row ranges
+    pl->grid = tiles * pl->NSPLIT;
+    pl->smem = (size_t)(tcg::NS1 + tcg::NLO1) * 12 * tcg::CH1 + 1024;
+    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tcg::TR1, 32, true)) return false;
+    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tcg::TR1, 32, true)) return false;
+    if (cudaFuncSetAttribute(tcg::k_pass1_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess)
+        return false;
+    return true;
+}
+
+void tcg_launch_first(const Problem& pb, const Tcg1Plan& pl)
+{
+    tcg::k_pass1_tcg<<<pl.grid, tcg::NTH1, pl.smem, pb.stream>>>(pl.tmX, pl.tmU, pb.ctl(), pb.P.n, pb.P.d, pb.P.r,
+                                                                 pl.NMT, pl.NNB, pl.NSPLIT, pb.part1());
+    pb.count(1);
+    launch_red1(pb, pl.NSPLIT, 0);
 }
 
 void tcg_launch_second(const Problem& pb, const TcgPlan& pl)

@@ -55,6 +55,18 @@ struct TcgPlan {
     float* img_lo;
 };
 bool tcg_plan(const Problem& pb, TcgPlan* plan, float* img_storage);
+
+// Matching first product (Theta^T tiles of 128 columns x 256 features, split over row ranges): d a
+// multiple of 32, (r / 128) * (d / 256) tiles at most one per SM.  The vector pass runs separately.
+struct Tcg1Plan {
+    alignas(64) CUtensorMap tmX;   // X-hat boxes: 16 rows x 32 features, 128-byte swizzle with 32-byte atoms
+    alignas(64) CUtensorMap tmU;   // U boxes: 16 rows x 32 columns, same layout
+    int NMT, NNB, NSPLIT, grid;
+    size_t smem;
+};
+bool tcg1_plan(const Problem& pb, Tcg1Plan* plan);
+// Theta partials per row range + their reduction (Theta, ||Theta||^2 shares).
+void tcg_launch_first(const Problem& pb, const Tcg1Plan& plan);
 void tcg_launch_second(const Problem& pb, const TcgPlan& plan);
 
 }  // namespace gemnlr

@@ -58,7 +58,7 @@ def test_tc_trajectory_matches_oracle_and_is_reproducible(n, d, K):
 
 # ---- tiled tcgen05 second product (wide d and r: 256-column blocks, d streamed in 16-feature chunks) ----
 # one and several column blocks, r not a multiple of 16, ragged last row tile, more items than CTAs
-TCG_SHAPES = [(3000, 48, 300), (2049, 768, 1000), (5000, 64, 520), (21000, 32, 260)]
+TCG_SHAPES = [(3000, 48, 300), (2049, 768, 1000), (5000, 64, 520), (21000, 32, 260), (4200, 288, 600)]
 
 
 @pytest.mark.parametrize("n,d,K", TCG_SHAPES)
