@@ -75,6 +75,97 @@ k_rowvec(float* __restrict__ U, float* __restrict__ ytilde, float* __restrict__ 
     }
 }
 
+// Vector pass for wide factors (128 < r <= 1024, r a multiple of 4): one warp per row, all of the
+// row's 16-byte pieces requested at once (up to 8 per lane), s accumulated in FP32 over 16 rows and
+// then folded into per-warp FP64 sums.  Same outputs as k_rowvec.
+constexpr int RVW_WARPS = 8;
+template <bool MATERIALIZE>
+__global__ void __launch_bounds__(RVW_WARPS * 32)
+k_rowvec_wide(float* __restrict__ U, float* __restrict__ ytilde, float* __restrict__ ybar,
+              const Ctl* __restrict__ ctl, const float* __restrict__ p, int64_t n, int r, double gamma,
+              double* __restrict__ part, int ignore_stop)
+{
+    if (!ignore_stop && ctl->stopped) return;
+    extern __shared__ double sm_s[];              // [RVW_WARPS][r]
+    __shared__ double sm_red[2][RVW_WARPS];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float cf = ctl->c_f;
+    const int dual = ctl->dual_pending;
+    const int r4 = r >> 2;
+    double* my_s = sm_s + (size_t)warp * r;
+    for (int j = lane; j < r; j += 32) my_s[j] = 0.0;
+    float4 p4[8], sacc[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int c4 = lane + 32 * k;
+        p4[k] = (c4 < r4) ? reinterpret_cast<const float4*>(p)[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+        sacc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    auto flush = [&]() {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int c4 = lane + 32 * k;
+            if (c4 < r4) {
+                double* o = my_s + 4 * c4;
+                o[0] += (double)sacc[k].x; o[1] += (double)sacc[k].y; o[2] += (double)sacc[k].z; o[3] += (double)sacc[k].w;
+            }
+            sacc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    double qq = 0.0, yq = 0.0;
+    int since = 0;
+    const int64_t stride = (int64_t)gridDim.x * RVW_WARPS;
+    for (int64_t row = (int64_t)blockIdx.x * RVW_WARPS + warp; row < n; row += stride) {
+        float4* urow = reinterpret_cast<float4*>(U + row * r);
+        float4 u[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int c4 = lane + 32 * k;
+            u[k] = (c4 < r4) ? __ldcs(urow + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float yt = ytilde[row];
+        float acc = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            u[k].x *= cf; u[k].y *= cf; u[k].z *= cf; u[k].w *= cf;
+            acc = fmaf(u[k].x, p4[k].x, acc); acc = fmaf(u[k].y, p4[k].y, acc);
+            acc = fmaf(u[k].z, p4[k].z, acc); acc = fmaf(u[k].w, p4[k].w, acc);
+        }
+        acc = warp_sum(acc);
+        const float q = acc - 1.0f;
+        if (dual) yt = (float)((double)yt + gamma * (double)q);
+        const float yb = (float)((double)yt + gamma * (double)q);
+        if (lane == 0) {
+            if (dual) ytilde[row] = yt;
+            ybar[row] = yb;
+            qq += (double)q * (double)q;
+            yq += (double)yt * (double)q;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            sacc[k].x = fmaf(u[k].x, yb, sacc[k].x); sacc[k].y = fmaf(u[k].y, yb, sacc[k].y);
+            sacc[k].z = fmaf(u[k].z, yb, sacc[k].z); sacc[k].w = fmaf(u[k].w, yb, sacc[k].w);
+            if (MATERIALIZE && lane + 32 * k < r4) urow[lane + 32 * k] = u[k];
+        }
+        if (++since == 16) { flush(); since = 0; }
+    }
+    flush();
+    if (lane == 0) { sm_red[0][warp] = qq; sm_red[1][warp] = yq; }
+    __syncthreads();
+    double* out = part + (size_t)blockIdx.x * (r + 2);
+    for (int j = threadIdx.x; j < r; j += blockDim.x) {
+        double v = 0.0;
+        for (int w = 0; w < RVW_WARPS; ++w) v += sm_s[(size_t)w * r + j];
+        out[j] = v;
+    }
+    if (threadIdx.x == 0) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < RVW_WARPS; ++w) { a += sm_red[0][w]; b += sm_red[1][w]; }
+        out[r] = a;
+        out[r + 1] = b;
+    }
+}
+
 // Column sums of c_f * U (p = U^T 1 for a freshly loaded factor): part[blockIdx][0..r-1].
 __global__ void __launch_bounds__(RV_WARPS * 32)
 k_colsum(const float* __restrict__ U, const Ctl* __restrict__ ctl, int64_t n, int r,
@@ -558,6 +649,15 @@ static int small_grid(const Problem& pb)
     return (int)(g < 1 ? 1 : g);
 }
 
+static bool wide_r(int r) { return r > 128 && r <= 1024 && r % 4 == 0; }
+static int wide_grid(const Problem& pb)
+{
+    int64_t g = (pb.P.n + RVW_WARPS - 1) / RVW_WARPS;
+    const int cap = pb.L.gv < kSMs * 2 ? pb.L.gv : kSMs * 2;
+    if (g > cap) g = cap;
+    return (int)(g < 1 ? 1 : g);
+}
+
 template <bool MAT>
 static void launch_rowvec_small(const Problem& pb, int grid, int ignore_stop)
 {
@@ -576,6 +676,24 @@ static int launch_rowvec(const Problem& pb, bool materialize, int ignore_stop)
         const int grid = small_grid(pb);
         if (materialize) launch_rowvec_small<true>(pb, grid, ignore_stop);
         else launch_rowvec_small<false>(pb, grid, ignore_stop);
+        pb.count();
+        return grid;
+    }
+    if (wide_r(P.r)) {
+        const int grid = wide_grid(pb);
+        const size_t sm = sizeof(double) * RVW_WARPS * (size_t)P.r;
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaFuncSetAttribute(k_rowvec_wide<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * 8);
+            cudaFuncSetAttribute(k_rowvec_wide<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * 8);
+            attr_set = true;
+        }
+        if (materialize)
+            k_rowvec_wide<true><<<grid, RVW_WARPS * 32, sm, pb.stream>>>(
+                pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
+        else
+            k_rowvec_wide<false><<<grid, RVW_WARPS * 32, sm, pb.stream>>>(
+                pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
         pb.count();
         return grid;
     }
@@ -625,7 +743,7 @@ static void launch_fin1_g(const Problem& pb, int mode, int gv)
 
 void launch_fin1(const Problem& pb, int mode)
 {
-    launch_fin1_g(pb, mode, small_r(pb.P.r) ? small_grid(pb) : pb.L.gv);
+    launch_fin1_g(pb, mode, small_r(pb.P.r) ? small_grid(pb) : wide_r(pb.P.r) ? wide_grid(pb) : pb.L.gv);
 }
 
 void launch_fin2(const Problem& pb, int gx, int gy, int cols_per)

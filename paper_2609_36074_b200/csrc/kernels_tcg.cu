@@ -71,6 +71,20 @@ __global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, 
     }
 }
 
+// 16 TMEM lanes x 16 columns in the fragment layout of the warp-level MMA accumulators: thread t gets,
+// for column block b (8 columns), v[4b], v[4b+1] = (lane t/4, columns 8b + 2 (t%4), + 1) and v[4b+2], v[4b+3] =
+// the same columns of lane t/4 + 8.  Four threads hold 8 consecutive columns of a row: one 32-byte sector.
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, float* v)
+{
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Column sums of a 32-row x 16-column block held one row per lane (v[16]): after the exchange
 // lane l holds the sum of column 8 b4 + 4 b3 + 2 b2 + b1 (bits of l) over the 32 rows.
 __device__ __forceinline__ float colsum16(const float* v, int lane)
@@ -186,27 +200,31 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
+        // The wait for the next chunk (and, at an item boundary, for its accumulator) is placed between
+        // the two k-steps of the current chunk, so the tensor pipe has work queued while this thread polls.
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(TILE_M, NBLK, 0, 0);
             int64_t g = 0;
             int i = 0;
+            if ((int64_t)blockIdx.x < n_items) mbar_wait(xsplit(0), 0, &abort_flag, ctl);
             for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x, ++i) {
                 const int a = i & 1;
-                if (i >= 2) mbar_wait(accfree(a), (uint32_t)((i >> 1) - 1) & 1, &abort_flag, ctl);
-                tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * NBLK);
+                const bool more_items = w + gridDim.x < n_items;
                 for (int kb = 0; kb < KB; ++kb, ++g) {
                     const int s = (int)(g % NS), l = (int)(g % NLO);
-                    mbar_wait(xsplit(s), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
                     tc_fence_after();
                     const uint32_t st = stage0 + (uint32_t)s * STAGE;
                     const uint64_t da_hi = umma_desc_sw64(st), da_lo = umma_desc_sw64(lo0 + (uint32_t)l * A_BOX);
                     const uint64_t db_hi = umma_desc_sw64(st + A_BOX), db_lo = umma_desc_sw64(st + A_BOX + B_BOX);
                     // a k-step (8 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
-#pragma unroll
-                    for (int ks = 0; ks < KC / 8; ++ks)
-                        umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
-                                     (kb | ks) ? 1u : 0u);
+                    umma_tf32_x3(tacc, da_hi, da_lo, db_hi, db_lo, idesc, kb ? 1u : 0u);
+                    if (kb + 1 < KB || more_items) {
+                        if (kb + 1 == KB && i + 1 >= 2)
+                            mbar_wait(accfree((i + 1) & 1), (uint32_t)(((i + 1) >> 1) - 1) & 1, &abort_flag, ctl);
+                        mbar_wait(xsplit((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
+                    }
+                    umma_tf32_x3(tacc, da_hi + 2, da_lo + 2, db_hi + 2, db_lo + 2, idesc, 1u);
                     umma_commit(xfree(s));
                     umma_commit(lofree(l));
                 }
@@ -241,60 +259,84 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
         }
     } else {
         // ------------------------------ epilogue (warps 2..9) ------------------------------
-        const int q = warp & 3;                           // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;                 // columns 128 half .. 128 half + 127 of the item
-        const int rl = q * 32 + lane;
+        // Warp = (TMEM lane quarter q, column half).  Accumulators are read in the 16x256b fragment layout:
+        // a thread holds rows q*32 + g + {0, 8, 16, 24} (g = lane / 4) and, per 16-column group, the column
+        // pairs 8 b + 2 tq, + 1 (tq = lane % 4, b = 0, 1), so that the 4 lanes of a group read and write one
+        // full 32-byte sector of a row of U.
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int g4 = lane >> 2, tq = lane & 3;
         const int et = (warp - 2) * 32 + lane;            // 0..255 among the epilogue threads
-        // column held by this lane after colsum16 (within a 16-column group)
-        const int ccol = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
         int i = 0;
         for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
             const int a = i & 1;
             const int64_t t = w / NCB;
             const int cb = (int)(w % NCB);
-            const int64_t row = t * TILE_M + rl;
-            const bool valid = row < n;
-            const float nay = valid ? -alpha * ybar[row] : 0.f;
-            float* urow = U + (valid ? row : 0) * (int64_t)r;
+            bool valid[4];
+            float nay[4];
+            float* urow[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
+                valid[x] = row < n;
+                nay[x] = valid[x] ? -alpha * ybar[row] : 0.f;
+                urow[x] = U + (valid[x] ? row : 0) * (int64_t)r;
+            }
             float* my_tmp = stmp + (size_t)(a * 4 + q) * NBLK + half * 128;
             mbar_wait(accfull(a), (uint32_t)(i >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
 #pragma unroll 1
             for (int jj = 0; jj < 8; ++jj) {
                 const int col0 = cb * NBLK + half * 128 + jj * 16;
-                float acc[16], wn[16];
-                float4 w4[4];
+                // acc[x2][...]: x2 = 0: rows g4, g4 + 8; x2 = 1: rows g4 + 16, g4 + 24
+                float acc[2][8];
+                const uint32_t tcol = (uint32_t)(a * NBLK + half * 128 + jj * 16);
+                tmem_ld_16x256b_x2(tmem_base + ((uint32_t)(q * 32) << 16) + tcol, acc[0]);
+                tmem_ld_16x256b_x2(tmem_base + ((uint32_t)(q * 32 + 16) << 16) + tcol, acc[1]);
+                float2 wold[4][2];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    w4[c] = (valid && col0 + 4 * c < r) ? __ldcs(reinterpret_cast<const float4*>(urow + col0 + 4 * c))
-                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
-                tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * NBLK + half * 128 + jj * 16), acc);
+                for (int x = 0; x < 4; ++x)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const float4 p4 = *reinterpret_cast<const float4*>(sp + col0 + 4 * c);
-                    const float4 s4 = *reinterpret_cast<const float4*>(sas + col0 + 4 * c);
-                    const float wold[4] = {w4[c].x, w4[c].y, w4[c].z, w4[c].w};
-                    const float pj[4] = {p4.x, p4.y, p4.z, p4.w};
-                    const float sj[4] = {s4.x, s4.y, s4.z, s4.w};
-                    const bool live = valid && (col0 + 4 * c < r);
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float u = live ? cf * wold[e] : 0.f;
-                        float v = fmaf(two_alpha, acc[4 * c + e], u);
-                        v = fmaf(nay, pj[e], v);
-                        v -= sj[e];
-                        const float wv = live ? fmaxf(v, 0.f) : 0.f;
-                        const double wd = (double)wv, ud = (double)u;
-                        sa = fma(wd, wd, sa);
-                        sb = fma(ud, ud, sb);
-                        sh = fma(wd, ud, sh);
-                        wn[4 * c + e] = wv;
+                    for (int b = 0; b < 2; ++b) {
+                        const int c = col0 + 8 * b + 2 * tq;
+                        wold[x][b] = (valid[x] && c < r) ? __ldcs(reinterpret_cast<const float2*>(urow[x] + c))
+                                                         : make_float2(0.f, 0.f);
                     }
-                    if (live)
-                        *reinterpret_cast<float4*>(urow + col0 + 4 * c) = make_float4(wn[4 * c], wn[4 * c + 1], wn[4 * c + 2], wn[4 * c + 3]);
+                tmem_ld_wait();
+                float cs[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const int c = col0 + 8 * b + 2 * tq;
+                    const float2 p2 = *reinterpret_cast<const float2*>(sp + c);
+                    const float2 s2 = *reinterpret_cast<const float2*>(sas + c);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                        const bool live = valid[x] && c < r;
+                        // rows g4 + 8 x: x = 0, 1 from the first load (registers 4b + 0..1 / 4b + 2..3), x = 2, 3 from the second
+                        const float a0 = acc[x >> 1][4 * b + 2 * (x & 1)], a1 = acc[x >> 1][4 * b + 2 * (x & 1) + 1];
+                        const float u0 = live ? cf * wold[x][b].x : 0.f, u1 = live ? cf * wold[x][b].y : 0.f;
+                        float v0 = fmaf(two_alpha, a0, u0), v1 = fmaf(two_alpha, a1, u1);
+                        v0 = fmaf(nay[x], p2.x, v0); v1 = fmaf(nay[x], p2.y, v1);
+                        v0 -= s2.x; v1 -= s2.y;
+                        const float w0 = live ? fmaxf(v0, 0.f) : 0.f, w1 = live ? fmaxf(v1, 0.f) : 0.f;
+                        const double wd0 = (double)w0, ud0 = (double)u0, wd1 = (double)w1, ud1 = (double)u1;
+                        sa = fma(wd0, wd0, sa); sb = fma(ud0, ud0, sb); sh = fma(wd0, ud0, sh);
+                        sa = fma(wd1, wd1, sa); sb = fma(ud1, ud1, sb); sh = fma(wd1, ud1, sh);
+                        cs[b][0] += w0; cs[b][1] += w1;
+                        if (live) *reinterpret_cast<float2*>(urow[x] + c) = make_float2(w0, w1);
+                    }
                 }
-                const float cs = colsum16(wn, lane);
-                if ((lane & 1) == 0) my_tmp[jj * 16 + ccol] = cs;
+                // column sums over the 32 rows of the quarter: the 8 row groups g4 of the warp
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float v = cs[b][e];
+                        v += __shfl_xor_sync(0xffffffffu, v, 4);
+                        v += __shfl_xor_sync(0xffffffffu, v, 8);
+                        v += __shfl_xor_sync(0xffffffffu, v, 16);
+                        if (lane < 4) my_tmp[jj * 16 + 8 * b + 2 * tq + e] = v;
+                    }
             }
             tc_fence_before();
             __syncwarp();
@@ -439,11 +481,12 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(128, Nb, 1, 1);
+            // the wait for the next stage sits between the two k-steps of the current one
+            if (my_stages > 0) mbar_wait(split(0), 0, &abort_flag, ctl);
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int s = g % NS1, l = g % NLO1;
                 const int period = g / FLUSH1, a = period & 1, in_period = g % FLUSH1;
                 if (in_period == 0 && period >= 2) mbar_wait(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
-                mbar_wait(split(s), (g / NS1) & 1, &abort_flag, ctl);
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * 256);
                 const uint32_t hi_s = raw0 + (uint32_t)s * STAGE1, lo_s = lo0 + (uint32_t)l * STAGE1;
@@ -451,10 +494,9 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
                 const uint64_t da_hi = umma_desc_sw128_atom32(hi_s, CH1, 512), da_lo = umma_desc_sw128_atom32(lo_s, CH1, 512);
                 const uint64_t db_hi = umma_desc_sw128_atom32(hi_s + 4 * CH1, CH1, 512);
                 const uint64_t db_lo = umma_desc_sw128_atom32(lo_s + 4 * CH1, CH1, 512);
-#pragma unroll
-                for (int ks = 0; ks < TR1 / 8; ++ks)
-                    umma_tf32_x3(tacc, da_hi + 64 * ks, da_lo + 64 * ks, db_hi + 64 * ks, db_lo + 64 * ks, idesc,
-                                 (in_period | ks) ? 1u : 0u);
+                umma_tf32_x3(tacc, da_hi, da_lo, db_hi, db_lo, idesc, in_period ? 1u : 0u);
+                if (g + 1 < my_stages) mbar_wait(split((g + 1) % NS1), ((g + 1) / NS1) & 1, &abort_flag, ctl);
+                umma_tf32_x3(tacc, da_hi + 64, da_lo + 64, db_hi + 64, db_lo + 64, idesc, 1u);
                 umma_commit(rawfree(s));
                 umma_commit(lofree(l));
                 if (in_period == FLUSH1 - 1 || g == my_stages - 1) umma_commit(accfull(a));
