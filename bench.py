@@ -40,6 +40,32 @@ def _peaks():
         return 6650.0, "fallback"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the second-product kernel, from the ncu
+# captures summarised under profiles/ (config 2 captured at full size; configs 3, 4, 5 captured at
+# n = 2e6 / 131072 / 1.6e7 rows and scaled by n: every row is read and written once per launch).
+# Keyed by (n, d, r, kernel path); anything else reports null.
+NCU_TRAFFIC_BYTES = {
+    (1_000_000, 128, 16, "mma.tf32x3"): 640.0e6,
+    (10_000_000, 64, 100, "tf32x3"): 10.385e9,
+    (2_000_000, 768, 1000, "tf32x3.tiled"): 22.93e9,
+    (100_000_000, 32, 8, "ffma"): 19.49e9,
+}
+
+# nominal dense TF32 : bf16 tensor throughput on this part (1.1 : 2.25 PFLOP/s)
+TF32_OVER_BF16 = 1.1 / 2.25
+
+
+def _tensor_peak_tf32():
+    """TF32 tensor peak in TFLOP/s: the measured cuBLAS bf16 figure sustained under the power cap (the
+    kernels are timed inside a step of seconds) times the nominal TF32 : bf16 ratio."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            m = json.load(f)
+        return float(m["bf16_tflops_sustained"]) * TF32_OVER_BF16, "measured bf16 sustained x nominal tf32:bf16 ratio"
+    except Exception:
+        return 1400.0 * TF32_OVER_BF16, "fallback bf16 sustained x nominal tf32:bf16 ratio"
+
+
 class ClockSampler(threading.Thread):
     """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
 
@@ -254,14 +280,33 @@ def main():
     roofline = None
     if prof_iters > 0:
         p2_s = ms_p2 * 1e-3 / prof_iters
-        ach = second_product_bytes(n, d, r) / p2_s / 1e9
-        roofline = {"bound": "hbm", "kernel": "second product + fused epilogue", "achieved": ach, "peak": peak,
-                    "unit": "GB/s", "frac": ach / peak, "peak_kind": peak_kind + " copy bandwidth",
-                    "traffic": None, "ms_per_launch": p2_s * 1e3,
-                    "first_phase_ms_per_iteration": ms_p1 / prof_iters,
-                    "iteration": {"algorithmic_bytes": algorithmic_bytes(n, d, r),
-                                  "achieved_gbs": algorithmic_bytes(n, d, r) * world * args.steps * T / (ms * 1e-3) / 1e9 / world,
-                                  "frac_of_peak": algorithmic_bytes(n, d, r) * args.steps * T / (ms * 1e-3) / 1e9 / peak}}
+        it_s = ms * 1e-3 / (args.steps * T)
+        tpeak, tpeak_kind = _tensor_peak_tf32()
+        # MMA flops actually issued on the tensor-core paths: three TF32 products per useful product
+        mma_mult = 3 if "tf32" in path else 0
+        t_hbm2 = second_product_bytes(n, d, r) / (peak * 1e9)
+        t_tc2 = mma_mult * 2.0 * n * d * r / (tpeak * 1e12)
+        iteration = {"algorithmic_bytes": algorithmic_bytes(n, d, r),
+                     "achieved_gbs": algorithmic_bytes(n, d, r) / it_s / 1e9,
+                     "frac_of_peak": algorithmic_bytes(n, d, r) / it_s / 1e9 / peak,
+                     "mma_flops": mma_mult * 4.0 * n * d * r,
+                     "achieved_tflops": mma_mult * 4.0 * n * d * r / it_s / 1e12,
+                     "frac_of_tensor_peak": mma_mult * 4.0 * n * d * r / it_s / 1e12 / tpeak,
+                     "tensor_peak_tflops": tpeak}
+        if t_tc2 > t_hbm2:
+            ach = mma_mult * 2.0 * n * d * r / p2_s / 1e12
+            roofline = {"bound": "tensor", "kernel": "second product + fused epilogue", "achieved": ach, "peak": tpeak,
+                        "unit": "TFLOP/s", "frac": ach / tpeak, "peak_kind": tpeak_kind,
+                        "flops_per_launch": mma_mult * 2.0 * n * d * r,
+                        "flops_note": "3 TF32 MMA products (hi*hi, lo*hi, hi*lo) per FP32-accurate product, 2ndr each",
+                        "traffic": NCU_TRAFFIC_BYTES.get((n, d, r, path)), "ms_per_launch": p2_s * 1e3,
+                        "first_phase_ms_per_iteration": ms_p1 / prof_iters, "iteration": iteration}
+        else:
+            ach = second_product_bytes(n, d, r) / p2_s / 1e9
+            roofline = {"bound": "hbm", "kernel": "second product + fused epilogue", "achieved": ach, "peak": peak,
+                        "unit": "GB/s", "frac": ach / peak, "peak_kind": peak_kind + " copy bandwidth",
+                        "traffic": NCU_TRAFFIC_BYTES.get((n, d, r, path)), "ms_per_launch": p2_s * 1e3,
+                        "first_phase_ms_per_iteration": ms_p1 / prof_iters, "iteration": iteration}
 
     # ---- CPU oracle leg (rank 0, N = 1 only) ------------------------------------------------------
     cpu = None

@@ -274,13 +274,15 @@ k_pass1_generic(const float* __restrict__ X, const float* __restrict__ U,
     }
 }
 
-// Theta[e] = FP32(sum_g part[g][e]) in ascending g (four interleaved slices combined in order);
-// red[blockIdx] = this block's share of ||Theta||_F^2 (from the unrounded sums).
+// Theta[e] = FP32(scale * sum_g part[g][e]) in ascending g (four interleaved slices combined in order);
+// red[blockIdx] = this block's share of ||Theta||_F^2 (from the unrounded sums).  scale is the pending
+// multiplier c_f when the partials were formed from the unscaled factor (scale_cf), else 1.
 __global__ void __launch_bounds__(256)
 k_red1(const double* __restrict__ part, int g, int64_t dr, const Ctl* __restrict__ ctl,
-       float* __restrict__ theta, double* __restrict__ red, int ignore_stop)
+       float* __restrict__ theta, double* __restrict__ red, int ignore_stop, int scale_cf)
 {
     if (!ignore_stop && ctl->stopped) return;
+    const double scale = scale_cf ? (double)ctl->c_f : 1.0;
     __shared__ double sl[4][64];
     __shared__ double sred[32];
     const int e_local = threadIdx.x & 63, slice = threadIdx.x >> 6;
@@ -292,7 +294,7 @@ k_red1(const double* __restrict__ part, int g, int64_t dr, const Ctl* __restrict
     __syncthreads();
     double t2 = 0.0;
     if (slice == 0 && e < dr) {
-        double tot = ((sl[0][e_local] + sl[1][e_local]) + sl[2][e_local]) + sl[3][e_local];
+        const double tot = scale * (((sl[0][e_local] + sl[1][e_local]) + sl[2][e_local]) + sl[3][e_local]);
         theta[e] = (float)tot;
         t2 = tot * tot;
     }
@@ -761,14 +763,14 @@ void launch_generic_pass1(const Problem& pb, int ignore_stop)
     k_pass1_generic<<<g1, 256, 0, pb.stream>>>(pb.X, pb.U, pb.ctl(), P.n, P.d, P.r, L.g1y_r, pb.part1(),
                                                ignore_stop);
     k_red1<<<L.nred1, 256, 0, pb.stream>>>(pb.part1(), L.g1x, (int64_t)P.d * P.r, pb.ctl(), pb.theta(),
-                                            pb.red1(), ignore_stop);
+                                            pb.red1(), ignore_stop, 0);
     pb.count(2);
 }
 
-void launch_red1(const Problem& pb, int g, int ignore_stop)
+void launch_red1(const Problem& pb, int g, int ignore_stop, int scale_cf)
 {
     k_red1<<<pb.L.nred1, 256, 0, pb.stream>>>(pb.part1(), g, (int64_t)pb.P.d * pb.P.r, pb.ctl(), pb.theta(),
-                                             pb.red1(), ignore_stop);
+                                             pb.red1(), ignore_stop, scale_cf);
     pb.count(1);
 }
 

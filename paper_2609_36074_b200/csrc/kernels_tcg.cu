@@ -16,7 +16,9 @@
 //                time: tcgen05.ld, old U entries straight from global memory (each thread reads and
 //                writes whole 32-byte sectors of its row), FP64 statistics; column sums by a
 //                shuffle transpose-reduce, combined across the four quarters in fixed order
-//   warps 10-13  split of the X-hat box into hi (in place) and lo (second ring)
+//   warps 10-13  split: lo image of the X-hat box (second ring).  The raw box itself is the hi operand:
+//                kind::tf32 ignores the low 13 mantissa bits of an FP32 operand (checked: results are
+//                unchanged when the box is not rewritten), so hi = trunc(x) needs no storage
 // Every mbarrier wait is bounded (error status GEM_NLR_E_TIMEOUT, kernel runs to its end, TMEM freed).
 #include "nlr_common.cuh"
 #include "device_utils.cuh"
@@ -232,7 +234,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
             }
         }
     } else if (warp >= 2 + NEPI) {
-        // ------------------------------ split: X-hat box -> hi (in place), lo ------------------------------
+        // ------------------------------ split: lo image of the X-hat box ------------------------------
         const int st = threadIdx.x - (2 + NEPI) * 32;   // 0..127
         int64_t g = 0;
         for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x) {
@@ -249,7 +251,6 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
                     const uint32_t off = (uint32_t)(k * 128 + st) * 16;
                     const float4 x = xin[k];
                     const float4 hi = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
-                    sts128(hi_a + off, hi);
                     sts128(lo_a + off, make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w));
                 }
                 fence_proxy_async();
@@ -398,13 +399,15 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
 
 
 // ================================================================================================
-// First product for the same wide problems:  Theta = X-hat^T (c_f W)  as Theta^T tiles.
+// First product for the same wide problems:  Theta = c_f X-hat^T W  as Theta^T tiles.
 //
 // Work item (one CTA each, all resident at once) = (128 columns of U, up to 256 features, one of
 // NSPLIT contiguous row ranges).  The contraction runs over the data rows, so both operands are
 // MN-major: TMA boxes of 16 rows x 32 columns with the 128-byte swizzle of 32-byte atoms (A = 4 boxes
 // of U, B = up to 8 boxes of X-hat per stage).  Two teams of four warps take alternate stages and
-// rewrite the boxes as hi (in place; U scaled by the pending multiplier first) and lo (second ring);
+// write the lo images (x - trunc(x)) into a second ring; the raw boxes serve as the hi operands (the
+// tensor core ignores the low 13 mantissa bits) and the pending multiplier c_f is applied to the
+// reduced Theta instead of to every entry of U;
 // the MMA issuer runs 2 k-steps x 3 products per stage into one of two TMEM accumulators, which is
 // handed to the epilogue every FLUSH stages and folded into the FP64 partial of this row range
 // (layout [feature][column] like the generic first product, so the same reduction kernel follows).
@@ -413,7 +416,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
 // ================================================================================================
 constexpr int TR1 = 16;                        // rows per stage (2 k-steps)
 constexpr int CH1 = TR1 * 128;                 // one box: 16 rows x 32 floats = 2 KB
-constexpr int NS1 = 4, NLO1 = 4;
+constexpr int NS1 = 5, NLO1 = 3;               // a raw slot lives from the TMA issue to the last MMA, a lo slot from the split on
 constexpr int FLUSH1 = 256;                    // stages per accumulation period (4096 rows)
 constexpr int NTH1 = 14 * 32;                  // producer, MMA, 4 epilogue, 8 split warps
 
@@ -464,7 +467,6 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
     const int64_t g_lo = (int64_t)sp * base_cnt + (sp < rem_cnt ? sp : rem_cnt);
     const int my_stages = (int)(base_cnt + (sp < rem_cnt ? 1 : 0));
     const int n_periods = (my_stages + FLUSH1 - 1) / FLUSH1;
-    const float cf = ctl->c_f;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -512,15 +514,19 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
             mbar_wait(full(s), (g / NS1) & 1, &abort_flag, ctl);
             if (g >= NLO1) mbar_wait(lofree(l), ((g / NLO1) - 1) & 1, &abort_flag, ctl);
             const uint32_t hi_s = raw0 + (uint32_t)s * STAGE1, lo_s = lo0 + (uint32_t)l * STAGE1;
-#pragma unroll 4
-            for (int k = 0; k < nq; ++k) {
-                const uint32_t off = (uint32_t)(k * 128 + tt) * 16;
-                float4 x = lds128(hi_s + off);
-                if (k < 4) { x.x *= cf; x.y *= cf; x.z *= cf; x.w *= cf; }      // the 4 U boxes: u = c_f w
-                const float4 h = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
-                sts128(hi_s + off, h);
-                sts128(lo_s + off, make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w));
-            }
+            // lo = x - trunc(x) of every piece (12 per thread at most, all requested up front); the raw boxes
+            // are the hi operands as they are
+            float4 xin[12];
+#pragma unroll
+            for (int k = 0; k < 12; ++k)
+                if (k < nq) xin[k] = lds128(hi_s + (uint32_t)(k * 128 + tt) * 16);
+#pragma unroll
+            for (int k = 0; k < 12; ++k)
+                if (k < nq) {
+                    const float4 x = xin[k];
+                    sts128(lo_s + (uint32_t)(k * 128 + tt) * 16,
+                           make_float4(x.x - tf32_hi(x.x), x.y - tf32_hi(x.y), x.z - tf32_hi(x.z), x.w - tf32_hi(x.w)));
+                }
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(split(s));
@@ -603,7 +609,7 @@ void tcg_launch_first(const Problem& pb, const Tcg1Plan& pl)
     tcg::k_pass1_tcg<<<pl.grid, tcg::NTH1, pl.smem, pb.stream>>>(pl.tmX, pl.tmU, pb.ctl(), pb.P.n, pb.P.d, pb.P.r,
                                                                  pl.NMT, pl.NNB, pl.NSPLIT, pb.part1());
     pb.count(1);
-    launch_red1(pb, pl.NSPLIT, 0);
+    launch_red1(pb, pl.NSPLIT, 0, 1);
 }
 
 void tcg_launch_second(const Problem& pb, const TcgPlan& pl)

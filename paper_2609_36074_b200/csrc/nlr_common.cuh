@@ -78,7 +78,7 @@ void launch_generic_pass1(const Problem& pb, int ignore_stop);
 void launch_fin1(const Problem& pb, int mode);
 void launch_generic_pass2_kernel(const Problem& pb);
 // Reduction of g FP64 partials of Theta (layout [d][r] each) into Theta and the ||Theta||^2 shares.
-void launch_red1(const Problem& pb, int g, int ignore_stop);   // the fused second product alone
+void launch_red1(const Problem& pb, int g, int ignore_stop, int scale_cf);   // the fused second product alone
 void launch_fin2(const Problem& pb, int gx, int gy, int cols_per);
 void launch_tail(const Problem& pb);
 void launch_objective(const Problem& pb);                   // fills ctl->f_final for the current (U, y)
