@@ -11,7 +11,8 @@
 //   warp 0      producer: TMA loads of X-hat boxes (128 rows x 32 features, 128-byte swizzle = the
 //               K-major UMMA operand layout) and of U panels (128 rows x 32 columns); the pre-split
 //               Theta^T images are brought in once per CTA.
-//   warps 18-21 split: rewrite each box as hi (in place) and lo (second buffer).
+//   warps 18-21 split: lo image (x - trunc(x)) of each box in a second buffer; the raw box is the hi
+//               operand as it is (kind::tf32 ignores the low 13 mantissa bits).
 //   warp 1      MMA issuer: per box 4 k-steps x 3 tcgen05.mma (M = 128 rows, N = padded r);
 //               tcgen05.commit frees the stage and publishes the accumulator (two TMEM buffers).
 //   warps 2-17  epilogue, four groups taking the panels of a tile round-robin: thread = row;
@@ -207,7 +208,6 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     const uint32_t off = (uint32_t)(k * 128 + st) * 16;
                     const float4 x = xin[k];
                     const float4 hi = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
-                    sts128(hi_a + off, hi);
                     sts128(lo_a + off, make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w));
                 }
                 fence_proxy_async();

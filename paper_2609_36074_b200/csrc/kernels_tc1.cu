@@ -13,7 +13,8 @@
 // One persistent CTA per SM, 14 warps:
 //   warp 0       producer: per stage of TR = 32 rows, ceil(r/32) U boxes and d/32 X-hat boxes.
 //   warps 6-13   vector + split: one warp per row does the row-local vector work on the U boxes and
-//                rewrites them as hi (in place) and lo (separate ring); then the X-hat boxes are split.
+//                writes their lo image (x - trunc(x)) into a separate ring, then those of the X-hat boxes.
+//                The raw boxes are the hi operands (kind::tf32 ignores the low 13 mantissa bits).
 //   warp 1       MMA issuer.  Every FLUSH stages the accumulator is handed to the epilogue and the
 //                other TMEM buffer is started from zero, so FP32 accumulation chains stay short.
 //   warps 2-5    epilogue: add each handed-over accumulator into this CTA's FP64 partial of Theta^T
@@ -176,7 +177,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             for (int half = 0; half < 2; ++half) {
                 // four independent rows at a time: loads first, reductions interleaved, then scalars and stores
                 uint32_t off[4];
-                float4 u4[4];
+                float4 u4[4], w4[4];
                 float dot[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
@@ -184,7 +185,6 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     off[k] = (uint32_t)(box * CHUNK_BYTES + rl * 128) + (uint32_t)((((c >> 1) ^ (rl & 3)) << 5) | ((c & 1) << 4));
                 }
                 {
-                    float4 w4[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k) w4[k] = lds128(hi_s + off[k]);
 #pragma unroll
@@ -216,9 +216,10 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     const float yb = __shfl_sync(0xffffffffu, yb_l, half * 4 + k);
                     s_acc[0] = fmaf(u4[k].x, yb, s_acc[0]); s_acc[1] = fmaf(u4[k].y, yb, s_acc[1]);   // rows beyond n: u = 0
                     s_acc[2] = fmaf(u4[k].z, yb, s_acc[2]); s_acc[3] = fmaf(u4[k].w, yb, s_acc[3]);
-                    const float4 hi = make_float4(tf32_hi(u4[k].x), tf32_hi(u4[k].y), tf32_hi(u4[k].z), tf32_hi(u4[k].w));
-                    sts128(hi_s + off[k], hi);
-                    sts128(lo_s + off[k], make_float4(u4[k].x - hi.x, u4[k].y - hi.y, u4[k].z - hi.z, u4[k].w - hi.w));
+                    // the raw box (unscaled w) is the hi operand as it is: the tensor core ignores the low 13
+                    // mantissa bits; c_f is applied when the accumulator is folded into the FP64 partial
+                    sts128(lo_s + off[k], make_float4(w4[k].x - tf32_hi(w4[k].x), w4[k].y - tf32_hi(w4[k].y),
+                                                      w4[k].z - tf32_hi(w4[k].z), w4[k].w - tf32_hi(w4[k].w)));
                 }
             }
             if (lane < 8 && myrow < n) {
@@ -231,8 +232,6 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 const float4 x0 = lds128(hi_s + o0), x1 = lds128(hi_s + o1);
                 const float4 h0 = make_float4(tf32_hi(x0.x), tf32_hi(x0.y), tf32_hi(x0.z), tf32_hi(x0.w));
                 const float4 h1 = make_float4(tf32_hi(x1.x), tf32_hi(x1.y), tf32_hi(x1.z), tf32_hi(x1.w));
-                sts128(hi_s + o0, h0);
-                sts128(hi_s + o1, h1);
                 sts128(lo_s + o0, make_float4(x0.x - h0.x, x0.y - h0.y, x0.z - h0.z, x0.w - h0.w));
                 sts128(lo_s + o1, make_float4(x1.x - h1.x, x1.y - h1.y, x1.z - h1.z, x1.w - h1.w));
             }
@@ -251,6 +250,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         // out[f * r + j]; every thread owns its addresses, lanes are contiguous in j).
         const int q4 = warp & 3;                          // TMEM lane quarter
         const int j = q4 * 32 + lane;                     // column of U
+        const double cfd = (double)cf;                    // Theta = c_f X-hat^T W: the MMAs run on the unscaled factor
         for (int period = 0; period < n_periods; ++period) {
             const int a = period & 1;
             mbar_wait(accfull(a), (period >> 1) & 1, &abort_flag, ctl);
@@ -263,7 +263,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const double prev = (period == 0) ? 0.0 : o[(size_t)k * r];
-                        o[(size_t)k * r] = prev + (double)v[k];
+                        o[(size_t)k * r] = prev + cfd * (double)v[k];
                     }
                 }
             }
