@@ -163,15 +163,18 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(TILE_M, NP, 0, 0);
             mbar_wait(thfull, 0, &abort_flag, ctl);
+            // Inside a tile the wait for the next box sits in the middle of the current box's k-steps, so the
+            // tensor pipe has MMAs queued while this thread polls.
             int i = 0;
             for (int64_t t = blockIdx.x; t < n_tiles && !abort_flag; t += gridDim.x, ++i) {
                 const int a = i & 1;
+                // tile boundary: the accumulator hand-over of the previous tile is already committed, so the
+                // epilogue runs while this thread waits for a free accumulator and the first box
                 if (i >= 2) mbar_wait(accfree(a), ((i >> 1) - 1) & 1, &abort_flag, ctl);
-                tc_fence_after();
+                mbar_wait(xsplit((i * NB) % NSB), ((i * NB) / NSB) & 1, &abort_flag, ctl);
                 const uint32_t tacc = tmem_base + (uint32_t)(a * ACC_COLS);
                 for (int b = 0; b < NB; ++b) {
                     const int g = i * NB + b, s = g % NSB, l = g % NLO;
-                    mbar_wait(xsplit(s), (g / NSB) & 1, &abort_flag, ctl);
                     tc_fence_after();
                     const uint32_t a_hi = stage0 + (uint32_t)s * BOX_BYTES, a_lo = lo0 + (uint32_t)l * BOX_BYTES;
                     const uint32_t b_hi = th_hi_s + (uint32_t)b * NP * 128, b_lo = th_lo_s + (uint32_t)b * NP * 128;
@@ -180,9 +183,11 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     const uint64_t da_hi = umma_desc_sw128(a_hi, 16, 1024), da_lo = umma_desc_sw128(a_lo, 16, 1024);
                     const uint64_t db_hi = umma_desc_sw128(b_hi, 16, 1024), db_lo = umma_desc_sw128(b_lo, 16, 1024);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
+                    for (int ks = 0; ks < 4; ++ks) {
+                        if (ks == 2 && b + 1 < NB) mbar_wait(xsplit((g + 1) % NSB), ((g + 1) / NSB) & 1, &abort_flag, ctl);
                         umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
                                      (b | ks) ? 1u : 0u);
+                    }
                     umma_commit(xfree(s));
                     umma_commit(lofree(l));
                 }

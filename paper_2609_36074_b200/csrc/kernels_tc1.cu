@@ -122,11 +122,13 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(128, d, 1, 1);
+            // The wait for the next stage sits in the middle of the current stage's k-steps, so the tensor
+            // pipe has MMAs queued while this thread polls.
+            if (my_stages > 0) mbar_wait(split(0), 0, &abort_flag, ctl);
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int s = g % NSR, l = g % NLO;
                 const int period = g / FLUSH, a = period & 1, in_period = g % FLUSH;
                 if (in_period == 0 && period >= 2) mbar_wait(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
-                mbar_wait(split(s), (g / NSR) & 1, &abort_flag, ctl);
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * d);
                 const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, lo_s = lo0 + (uint32_t)l * STAGE;
@@ -136,9 +138,12 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 const uint64_t db_hi = umma_desc_sw128_atom32(hi_s + 4 * CHUNK_BYTES, CHUNK_BYTES, 512);
                 const uint64_t db_lo = umma_desc_sw128_atom32(lo_s + 4 * CHUNK_BYTES, CHUNK_BYTES, 512);
 #pragma unroll
-                for (int ks = 0; ks < TR / 8; ++ks)
+                for (int ks = 0; ks < TR / 8; ++ks) {
+                    if (ks == TR / 16 && g + 1 < my_stages)
+                        mbar_wait(split((g + 1) % NSR), ((g + 1) / NSR) & 1, &abort_flag, ctl);
                     umma_tf32_x3(tacc, da_hi + 64 * ks, da_lo + 64 * ks, db_hi + 64 * ks, db_lo + 64 * ks, idesc,
                                  (in_period | ks) ? 1u : 0u);
+                }
                 umma_commit(rawfree(s));
                 umma_commit(lofree(l));
                 if (in_period == FLUSH - 1 || g == my_stages - 1) umma_commit(accfull(a));

@@ -202,17 +202,19 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
-        // The wait for the next chunk (and, at an item boundary, for its accumulator) is placed between
-        // the two k-steps of the current chunk, so the tensor pipe has work queued while this thread polls.
+        // Inside an item the wait for the next chunk is placed between the two k-steps of the current chunk,
+        // so the tensor pipe has work queued while this thread polls.
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_tf32(TILE_M, NBLK, 0, 0);
             int64_t g = 0;
             int i = 0;
-            if ((int64_t)blockIdx.x < n_items) mbar_wait(xsplit(0), 0, &abort_flag, ctl);
             for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x, ++i) {
                 const int a = i & 1;
+                // item boundary: the previous accumulator is already handed over; wait for a free one and for
+                // the first chunk
+                if (i >= 2) mbar_wait(accfree(a), (uint32_t)((i >> 1) - 1) & 1, &abort_flag, ctl);
+                mbar_wait(xsplit((int)(g % NS)), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
                 const uint32_t tacc = tmem_base + (uint32_t)(a * NBLK);
-                const bool more_items = w + gridDim.x < n_items;
                 for (int kb = 0; kb < KB; ++kb, ++g) {
                     const int s = (int)(g % NS), l = (int)(g % NLO);
                     tc_fence_after();
@@ -221,11 +223,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
                     const uint64_t db_hi = umma_desc_sw64(st + A_BOX), db_lo = umma_desc_sw64(st + A_BOX + B_BOX);
                     // a k-step (8 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
                     umma_tf32_x3(tacc, da_hi, da_lo, db_hi, db_lo, idesc, kb ? 1u : 0u);
-                    if (kb + 1 < KB || more_items) {
-                        if (kb + 1 == KB && i + 1 >= 2)
-                            mbar_wait(accfree((i + 1) & 1), (uint32_t)(((i + 1) >> 1) - 1) & 1, &abort_flag, ctl);
-                        mbar_wait(xsplit((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
-                    }
+                    if (kb + 1 < KB) mbar_wait(xsplit((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
                     umma_tf32_x3(tacc, da_hi + 2, da_lo + 2, db_hi + 2, db_lo + 2, idesc, 1u);
                     umma_commit(xfree(s));
                     umma_commit(lofree(l));
