@@ -73,52 +73,6 @@ __global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, 
     }
 }
 
-// 16 TMEM lanes x 16 columns in the fragment layout of the warp-level MMA accumulators: thread t gets,
-// for column block b (8 columns), v[4b], v[4b+1] = (lane t/4, columns 8b + 2 (t%4), + 1) and v[4b+2], v[4b+3] =
-// the same columns of lane t/4 + 8.  Four threads hold 8 consecutive columns of a row: one 32-byte sector.
-__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, float* v)
-{
-    uint32_t r[8];
-    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr));
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Column sums of a 32-row x 16-column block held one row per lane (v[16]): after the exchange
-// lane l holds the sum of column 8 b4 + 4 b3 + 2 b2 + b1 (bits of l) over the 32 rows.
-__device__ __forceinline__ float colsum16(const float* v, int lane)
-{
-    float a8[8], a4[4], a2[2], a1;
-    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float send = h16 ? v[i] : v[i + 8];
-        const float keep = h16 ? v[i + 8] : v[i];
-        a8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float send = h8 ? a8[i] : a8[i + 4];
-        const float keep = h8 ? a8[i + 4] : a8[i];
-        a4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-    }
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const float send = h4 ? a4[i] : a4[i + 2];
-        const float keep = h4 ? a4[i + 2] : a4[i];
-        a2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-    }
-    {
-        const float send = h2 ? a2[0] : a2[1];
-        const float keep = h2 ? a2[1] : a2[0];
-        a1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-    }
-    return a1 + __shfl_xor_sync(0xffffffffu, a1, 1);
-}
-
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ img_hi,
             const float* __restrict__ img_lo, float* __restrict__ U, const float* __restrict__ ybar,

@@ -126,6 +126,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v)
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 16 TMEM lanes x 16 columns in the fragment layout of the warp-level MMA accumulators: thread t gets,
+// for column block b (8 columns), v[4b], v[4b+1] = (lane t/4, columns 8b + 2 (t%4), + 1) and v[4b+2], v[4b+3] =
+// the same columns of lane t/4 + 8.  Four threads hold 8 consecutive columns of a row: one 32-byte sector.
+// Completion must be awaited with tmem_ld_wait() before the values are used.
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, float* v)
+{
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // TMA tile store shared -> global (clipped at the tensor bounds), bulk-group completion.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, int x, int y, uint32_t src)
 {
