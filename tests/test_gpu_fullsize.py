@@ -100,3 +100,49 @@ def test_embedding_shape_reduced_n_twin():
     """Config 4's d = 768, K = 1000 and unit-sphere data at n = 20,000 (generic kernel family)."""
     out = _run(dataclasses.replace(synth.config(4), n=20_000, name="embedding-n20000"))
     print(f"config 4 twin: a={out['a']:.6g} U err={out['err']:.2e} label ties={out['label_ties']}")
+
+
+def test_embedding_shape_full_size_every_entry():
+    """Config 4 at its full n = 2e6 (d = 768, K = 1000), tiled tcgen05 kernels as bench.py runs them: one
+    iteration from the seeded start against the row-chunked FP64 numpy restatement of the iteration
+    (itself pinned to the C oracle by the CPU tests), on every entry of U and all statistics."""
+    from oracle import np_iteration
+    spec = synth.config(4)
+    n, d, K = spec.n, spec.d, spec.K
+    need = 4 * n * d + 3 * 4 * n * K + (4 << 30)
+    if psutil.virtual_memory().available < need:
+        pytest.skip(f"needs about {need / 2**30:.0f} GiB of host memory")
+    if torch.cuda.mem_get_info()[0] < 4 * n * (d + K + 8) + (2 << 30):
+        pytest.skip("not enough device memory")
+    hp = synth.default_hparams(K)
+    X, _, _ = synth.make_mixture(spec)
+    U0 = synth.make_u0(n, K, K)
+    Xd = torch.from_numpy(X).cuda()
+    del X
+    Ud = torch.from_numpy(U0).cuda()
+    s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"],
+                   T=spec.iters, T_min=spec.iters)
+    assert s.path() == "tf32x3.tiled", s.path()
+    s.spectral_norm()
+    Xhat = Xd.cpu().numpy()                      # both sides work on the library's X-hat
+    rc, info = s.step()
+    assert rc >= 0, (rc, s.last_error())
+    Ug = s.U.cpu().numpy()
+    lab_g = s.labels().cpu().numpy()
+    s.destroy()
+    del Xd, Ud
+    Uref, _, ref = np_iteration.iteration(Xhat, U0, np.zeros(n, np.float32), K, hp["alpha"], hp["beta"], hp["eps_d"])
+    scale = float(np.abs(Uref).max())
+    err = _chunked_max_abs_diff(Ug, Uref.astype(np.float64)) / scale
+    print(f"config 4 full size: U err={err:.2e}")
+    assert err <= TOL_U, err
+    assert _rel(info["a"], ref["a"]) <= 1e-6 and _rel(info["b"], ref["b"]) <= 1e-6 and _rel(info["h"], ref["h"]) <= 1e-6
+    assert _rel(info["c"], ref["c"]) <= 2e-7 and abs(info["delta_hat"] - ref["delta_hat"]) <= 1e-6
+    assert _rel(info["fhat"], ref["fhat"]) <= TOL_F and info["dual_applied"] == ref["dual"]
+    lab_o = oracle.labels(Uref)
+    diff = np.nonzero(lab_g != lab_o)[0]
+    if diff.size:
+        top_o = Uref[diff, lab_o[diff]].astype(np.float64)
+        alt_o = Uref[diff, lab_g[diff]].astype(np.float64)
+        assert ((top_o - alt_o) <= 2 * TOL_U * scale).all()
+    assert diff.size <= 1e-4 * n

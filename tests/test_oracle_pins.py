@@ -327,3 +327,27 @@ def test_run_equals_repeated_steps():
     assert iters == 25 and rc == 0
     assert np.array_equal(U, st.U) and np.array_equal(yt, st.ytilde)
     assert last["delta_hat"] == info["delta_hat"] and last["rho"] == info["rho"]
+
+
+def test_numpy_iteration_matches_the_c_oracle():
+    """The row-chunked numpy restatement used for the largest shape agrees with the C oracle entry by
+    entry (two consecutive iterations, the second with a pending dual step)."""
+    from oracle import np_iteration
+    n, d, K = 3001, 24, 7
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 3)
+    X, _, _ = synth.make_mixture(spec)
+    Xhat, _, _ = oracle.normalize(X)
+    U0 = synth.make_u0(n, K, K, seed=3)
+    hp = dict(synth.default_hparams(K), eps_d=10.0)           # gate always open: the dual step is exercised
+    st = oracle.State(Xhat, U0)
+    U, yt, dual = U0, np.zeros(n, np.float32), False
+    for _ in range(2):
+        ref = st.step(K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], 100)
+        U, yt, info = np_iteration.iteration(Xhat, U, yt, K, hp["alpha"], hp["beta"], hp["eps_d"], dual_pending=dual,
+                                             rows=1000)
+        dual = bool(info["dual"])
+        assert np.abs(U.astype(np.float64) - st.U).max() <= 2e-7 * np.abs(st.U).max()
+        for k in ("a", "b", "h", "fhat"):
+            assert abs(info[k] - ref[k]) <= (1e-7 if k == "fhat" else 1e-9) * max(abs(ref[k]), 1e-3), (k, info[k], ref[k])
+        assert abs(info["c"] - ref["c"]) <= 1e-7 * ref["c"] and abs(info["delta_hat"] - ref["delta_hat"]) <= 1e-9
+        assert info["dual"] == ref["dual"] == 1
