@@ -166,9 +166,8 @@ def main():
     import paper_2609_36074_b200 as gem
     from paper_2609_36074_b200.binding import make_params
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2609_36074_b200 import replicas
+    rank, world, local = replicas.rank_world_local()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -179,8 +178,7 @@ def main():
     n, d, K = spec.n, spec.d, spec.K
     r = K
     # every rank holds its own replica, seeded by rank
-    import dataclasses
-    rspec = dataclasses.replace(spec, seed=spec.seed + rank)
+    rspec = replicas.replica_spec(spec, rank)
     X_host = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
     synth.make_mixture(rspec, out=X_host.numpy())
     U0_host = torch.empty((n, r), dtype=torch.float32, pin_memory=True)
@@ -213,8 +211,7 @@ def main():
     solver.profile(True)
     launches0 = solver.launch_count()
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
+    replicas.barrier()
     sampler = ClockSampler(local)
     sampler.start()
     ev[2].record()
@@ -222,18 +219,14 @@ def main():
         info = one_step()
     ev[3].record()
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
+    replicas.barrier()
     clocks = sampler.finish()
     ms = ev[2].elapsed_time(ev[3])
     launches = solver.launch_count() - launches0
     ms_p1, ms_p2, prof_iters = solver.profile_read()
     solver.profile(False)
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * args.steps * T / (ms * 1e-3)
+    ms = replicas.max_over_ranks(ms, dev)
+    value = replicas.whole_job_rate(world, args.steps, T, ms)
 
     # labels (S7) timed on their own
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -266,11 +259,8 @@ def main():
             if i > 0:
                 tot += e0.elapsed_time(e1)
         e2e_ms = tot / reps
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e = {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * n * (d + r),
+        e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
+        e2e = {"value": replicas.whole_job_rate(world, 1, T, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": 4 * n * (d + r),
                "d2h_bytes_per_step": 4 * n * (r + 1), "ms_per_job": e2e_ms,
                "includes": "H2D of X and U0, mean + power iteration + normalization, T iterations, labels, D2H of U and labels"}
         del buf
