@@ -81,7 +81,6 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     const int NPAN = (r + PW - 1) / PW;            // PW-column panels of U per tile (PW = 16 or 32)
     const int ACC_COLS = (NPAN * PW + 31) / 32 * 32;   // TMEM columns per accumulator buffer
     const int PAN_BYTES = TILE_M * PW * 4;
-    const int CS_ROWS = PW / 2;                    // rows per thread in the column-sum sweep
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * ACC_COLS) tmem_cols <<= 1;
     const uint32_t th_bytes = (uint32_t)NB * NP * 128;
@@ -131,9 +130,8 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     const float cf = ctl->c_f;
     const float two_alpha = 2.0f * alpha;
     double sa = 0.0, sb = 0.0, sh = 0.0;
-    double csum[8];                      // epilogue thread (col, quarter): running column sums, one per panel
-#pragma unroll
-    for (int i = 0; i < 8; ++i) csum[i] = 0.0;
+    double csum[2][2];                   // epilogue thread: running sums of its column (after the transpose-reduce) per
+    csum[0][0] = csum[0][1] = csum[1][0] = csum[1][1] = 0.0;   // (panel of the group, 16-column half); over this quarter's rows
 
     if (warp == 0) {
         // ------------------------------ producer ------------------------------
@@ -230,9 +228,9 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         const int q = warp & 3;                           // TMEM lane quarter of this warp
         const int grp = (warp - 2) >> 2;                  // epilogue group
         const int rl = q * 32 + lane;                     // row of the tile owned by this thread
-        const int gt = (q * 32 + lane);                   // 0..127 inside the group (any bijection works)
-        const int cs_col = gt % PW, cs_o = gt / PW;       // column-sum sweep: column, row group
-        const int CS_ROWS_G = TILE_M / (GROUP_THREADS / PW);
+        const int gt = (q * 32 + lane);                   // 0..127 inside the group
+        // column (within a 16-column half) whose sum this lane holds after colsum16
+        const int ccol = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
         int i = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
             const int a = i & 1;
@@ -248,8 +246,11 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 mbar_wait(ufull(sl), (h / NUP) & 1, &abort_flag, ctl);
 #pragma unroll 1
                 for (int hf = 0; hf < PW / 16; ++hf) {
-                    float acc[16];
+                    float acc[16], wn[16];
                     tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * ACC_COLS + pn * PW + hf * 16), acc);
+                    // Statistics of these 16 entries in FP32 (w >= 0, u >= 0: no cancellation), folded into the
+                    // FP64 running sums once per group: the FP32 -> FP64 conversion unit is the scarce resource.
+                    float a32 = 0.f, b32 = 0.f, h32 = 0.f;
 #pragma unroll
                     for (int cc = 0; cc < 4; ++cc) {
                         const int c = hf * 4 + cc;
@@ -262,23 +263,27 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                         const float wold[4] = {w4.x, w4.y, w4.z, w4.w};
                         const float pj[4] = {p4.x, p4.y, p4.z, p4.w};
                         const float sj[4] = {s4.x, s4.y, s4.z, s4.w};
-                        float wn[4];
+                        const bool live = valid && (col0 < r);           // r is a multiple of 4
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const bool live = valid && (col0 + e < r);
                             const float u = live ? cf * wold[e] : 0.f;
                             float v = fmaf(two_alpha, acc[4 * cc + e], u);
                             v = fmaf(nay, pj[e], v);
                             v -= sj[e];
                             const float w = live ? fmaxf(v, 0.f) : 0.f;
-                            const double wd = (double)w, ud = (double)u;
-                            sa = fma(wd, wd, sa);
-                            sb = fma(ud, ud, sb);
-                            sh = fma(wd, ud, sh);
-                            wn[e] = w;
+                            a32 = fmaf(w, w, a32);
+                            b32 = fmaf(u, u, b32);
+                            h32 = fmaf(w, u, h32);
+                            wn[4 * cc + e] = w;
                         }
-                        sts128(addr, make_float4(wn[0], wn[1], wn[2], wn[3]));
+                        sts128(addr, make_float4(wn[4 * cc], wn[4 * cc + 1], wn[4 * cc + 2], wn[4 * cc + 3]));
                     }
+                    sa += (double)a32;
+                    sb += (double)b32;
+                    sh += (double)h32;
+                    // column sums over this warp's 32 rows (transpose-reduce), FP64 across tiles
+                    const float cs = colsum16(wn, lane);
+                    csum[(pn / NGROUPS) & 1][hf & 1] += (double)cs;
                 }
                 fence_proxy_async();
                 named_bar_sync(1 + grp, GROUP_THREADS);
@@ -286,26 +291,12 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     tma_store_2d(&tmU, pn * PW, (int)(t * TILE_M), pan);
                     bulk_commit();
                 }
-                // column sums of this panel: thread (column, row group) adds its rows
-                {
-                    float cs = 0.f;
-#pragma unroll 8
-                    for (int rr = 0; rr < CS_ROWS_G; ++rr) {
-                        const int row_l = cs_o * CS_ROWS_G + rr;
-                        const uint32_t addr = (PW == 32)
-                            ? pan + (uint32_t)row_l * 128 + (uint32_t)((((cs_col >> 2) ^ (row_l & 7)) << 4) + (cs_col & 3) * 4)
-                            : pan + (uint32_t)row_l * 64 + (uint32_t)(cs_col * 4);
-                        float v;
-                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-                        cs += v;
-                    }
-                    csum[(pn / NGROUPS) & 7] += (double)cs;
+                // the slot goes back to the producer as soon as the store has read it (every thread of the group
+                // passed the barrier above after its last access)
+                if (gt == 0) {
+                    bulk_wait_read<0>();
+                    mbar_arrive(ufree(sl));
                 }
-                // the store has read the panel (its wait overlapped the sweep above) and every thread of
-                // the group is done with it: hand the slot back to the producer
-                if (gt == 0) bulk_wait_read<0>();
-                named_bar_sync(1 + grp, GROUP_THREADS);
-                if (gt == 0) mbar_arrive(ufree(sl));
             }
             tc_fence_before();
             __syncwarp();
@@ -322,20 +313,19 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     sa = block_sum<NTHREADS>(sa, sred);
     sb = block_sum<NTHREADS>(sb, sred);
     sh = block_sum<NTHREADS>(sh, sred);
-    double* scol = reinterpret_cast<double*>(smem);        // [128 / PW row groups][ACC_COLS]
-    if (warp >= 2 && warp < 2 + 4 * NGROUPS) {
-        const int grp = (warp - 2) >> 2, gt = (warp & 3) * 32 + lane;
+    double* scol = reinterpret_cast<double*>(smem);        // [4 lane quarters][ACC_COLS]
+    if (warp >= 2 && warp < 2 + 4 * NGROUPS && (lane & 1) == 0) {
+        const int grp = (warp - 2) >> 2, q = warp & 3;
+        const int ccol = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
         for (int pn = grp; pn < NPAN; pn += NGROUPS)
-            scol[(size_t)(gt / PW) * ACC_COLS + pn * PW + (gt % PW)] = csum[(pn / NGROUPS) & 7];
+            for (int hf = 0; hf < PW / 16; ++hf)
+                scol[(size_t)q * ACC_COLS + pn * PW + hf * 16 + ccol] = csum[(pn / NGROUPS) & 1][hf & 1];
     }
     __syncthreads();
     double* out = part + (size_t)blockIdx.x * PS;
     if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; out[2] = sh; out[3] = 0.0; }
-    for (int j = threadIdx.x; j < r; j += NTHREADS) {
-        double v = 0.0;
-        for (int o = 0; o < GROUP_THREADS / PW; ++o) v += scol[(size_t)o * ACC_COLS + j];
-        out[4 + j] = v;
-    }
+    for (int j = threadIdx.x; j < r; j += NTHREADS)
+        out[4 + j] = ((scol[j] + scol[(size_t)ACC_COLS + j]) + scol[(size_t)2 * ACC_COLS + j]) + scol[(size_t)3 * ACC_COLS + j];
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {

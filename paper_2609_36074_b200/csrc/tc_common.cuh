@@ -141,6 +141,39 @@ __device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, float* v)
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Column sums of a 32-row x 16-column block held one row per lane (v[16]): after the exchange
+// lane l holds the sum of column 8 b4 + 4 b3 + 2 b2 + b1 (bits of l) over the 32 rows (both lanes of a
+// pair hold the same value).  31 adds and 16 shuffles instead of 80 of each for 16 butterfly sums.
+__device__ __forceinline__ float colsum16(const float* v, int lane)
+{
+    float a8[8], a4[4], a2[2], a1;
+    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float send = h16 ? v[i] : v[i + 8];
+        const float keep = h16 ? v[i + 8] : v[i];
+        a8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float send = h8 ? a8[i] : a8[i + 4];
+        const float keep = h8 ? a8[i + 4] : a8[i];
+        a4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float send = h4 ? a4[i] : a4[i + 2];
+        const float keep = h4 ? a4[i + 2] : a4[i];
+        a2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    {
+        const float send = h2 ? a2[0] : a2[1];
+        const float keep = h2 ? a2[1] : a2[0];
+        a1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    return a1 + __shfl_xor_sync(0xffffffffu, a1, 1);
+}
+
 // TMA tile store shared -> global (clipped at the tensor bounds), bulk-group completion.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, int x, int y, uint32_t src)
 {
