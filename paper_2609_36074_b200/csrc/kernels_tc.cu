@@ -35,7 +35,7 @@ namespace tc {
 constexpr int TILE_M = 128;
 constexpr int BOX_BYTES = TILE_M * 128;       // 128 rows x 32 floats
 constexpr int NGROUPS = 4;               // epilogue warp groups; group g owns panels pn = g (mod 4)
-constexpr int NTHREADS = (2 + 4 * NGROUPS + 4) * 32;   // producer, MMA, 16 epilogue, 4 split warps
+constexpr int NTHREADS = (2 + 4 * NGROUPS + 4 + 1) * 32;   // X producer, MMA, 16 epilogue, 4 split, U-panel producer warps
 constexpr int GROUP_THREADS = 128;
 constexpr int MAX_RING = 8;
 
@@ -60,7 +60,7 @@ __global__ void k_theta_images(const float* __restrict__ theta, int d, int r, in
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU,
-           const float* __restrict__ img_hi, const float* __restrict__ img_lo,
+           const float* __restrict__ U, const float* __restrict__ img_hi, const float* __restrict__ img_lo,
            const float* __restrict__ ybar, const float* __restrict__ p, const float* __restrict__ alpha_s,
            Ctl* __restrict__ ctl, int64_t n, int d, int r, int NP, int PW, int NSB, int NLO, int NUP, float alpha, int K,
            double eps_d, double* __restrict__ part, float* __restrict__ p_out)
@@ -148,6 +148,28 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     mbar_expect_tx(xfull(s), BOX_BYTES);
                     tma_load_2d(stage0 + (uint32_t)s * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
                 }
+            }
+        }
+    } else if (warp == 2 + 4 * NGROUPS + 4) {
+        // ------------------------------ U-panel producer ------------------------------
+        // Its own thread, so that waiting for a free panel slot (the epilogue of the previous tile) never
+        // holds back the X-hat loads of the next tile.  The U rows of the tile after next (one contiguous
+        // block) are asked into L2 ahead of time: a slot is refilled only once its group has stored the
+        // previous panel, and the refill should then not pay DRAM latency.
+        if (lane == 0) {
+            int i = 0;
+            for (int64_t t = blockIdx.x; t < n_tiles && !abort_flag; t += gridDim.x, ++i) {
+                const int row0 = (int)(t * TILE_M);
+                {
+                    const int64_t tn = t + gridDim.x;
+                    if (tn < n_tiles) {
+                        const int64_t r0 = tn * TILE_M, r1 = (r0 + TILE_M < n) ? r0 + TILE_M : n;
+                        const char* src = reinterpret_cast<const char*>(U + r0 * (int64_t)r);
+                        const int64_t bytes = (r1 - r0) * (int64_t)r * 4;        // multiple of 16: r is a multiple of 4
+                        for (int64_t o = 0; o < bytes; o += 16384)
+                            bulk_prefetch_l2(src + o, (uint32_t)(bytes - o < 16384 ? bytes - o : 16384));
+                    }
+                }
                 for (int pn = 0; pn < NPAN; ++pn) {
                     const int h = i * NPAN + pn, sl = h % NUP;
                     if (h >= NUP) mbar_wait(ufree(sl), ((h / NUP) - 1) & 1, &abort_flag, ctl);
@@ -192,7 +214,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 umma_commit(accfull(a));
             }
         }
-    } else if (warp >= 2 + 4 * NGROUPS) {
+    } else if (warp >= 2 + 4 * NGROUPS && warp < 2 + 4 * NGROUPS + 4) {
         // ------------------------------ split: box -> hi (in place), lo ------------------------------
         const int st = threadIdx.x - (2 + 4 * NGROUPS) * 32;   // 0..127
         int i = 0;
@@ -407,7 +429,7 @@ void tc_launch_second(const Problem& pb, const TcPlan& pl)
     const int total = d * pl.NP;
     tc::k_theta_images<<<(total + 255) / 256, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NP, pb.ctl(), pl.img_hi, pl.img_lo);
     tc::k_pass2_tc<<<pl.g2, tc::NTHREADS, pl.smem2, pb.stream>>>(
-        pl.tmX, pl.tmU, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NP,
+        pl.tmX, pl.tmU, pb.U, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NP,
         pl.PW, pl.NSB, pl.NLO, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
     pb.count(2);
 }
