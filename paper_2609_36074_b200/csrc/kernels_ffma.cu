@@ -41,7 +41,8 @@ bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int c
     cuuint32_t estr[2] = {1, 1};
     CUresult rc = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, (void*)base, gdim, gstride, box, estr,
                          CU_TENSOR_MAP_INTERLEAVE_NONE,
-                         (swizzle_bytes == 64 && box_cols * sizeof(float) == 64) ? CU_TENSOR_MAP_SWIZZLE_64B
+                         swizzle_bytes == 1 ? CU_TENSOR_MAP_SWIZZLE_NONE
+                         : (swizzle_bytes == 64 && box_cols * sizeof(float) == 64) ? CU_TENSOR_MAP_SWIZZLE_64B
                          : box_cols * sizeof(float) != 128 ? CU_TENSOR_MAP_SWIZZLE_NONE
                              : (atom32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B),
                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
