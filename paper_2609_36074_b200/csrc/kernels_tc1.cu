@@ -7,7 +7,7 @@
 // x 2^k = h1 + h2 with h1 = fp16(x 2^k), h2 = fp16(x 2^k - h1) (22 significant bits), and the product is
 // accumulated in FP32 as h1 h1' + h2 h1' + h1 h2' (three MMAs with K = 16); the dropped h2 h2' term is
 // below 2^-22 relative.  The scales cannot overflow: |x-hat_ij| <= ||X-hat||_2 = 1 (scale 2^15) and
-// |w_ij| <= ||W||_F = sqrt(K) / c_f (scale the largest power of two with |w| 2^k <= 2^14).  Against the
+// |u_ij| <= ||U||_F = sqrt(K) (scale the largest power of two with |u| 2^k <= 2^14).  Against the
 // 3xTF32 split of the other kernels this halves the number of MMA instructions per row (K = 16 instead
 // of 8), and an MMA instruction costs the same ~130-180 cycles whatever K is: at N = d = 64 the TF32
 // version of this kernel was bound by exactly that instruction rate.
@@ -20,7 +20,7 @@
 //
 // One persistent CTA per SM, 14 warps:
 //   warp 0       producer: per stage ceil(r/32) U boxes and d/32 X-hat boxes (plain FP32 rows).
-//   warps 6-13   vector + split, two teams on alternate stages: one warp per row does the row-local
+//   warps 6-17   vector + split, three teams taking stages round-robin: one warp per row does the row-local
 //                vector work on the U boxes, then both operands are converted into the image ring;
 //                the raw stage goes back to the producer as soon as the team has read it.
 //   warp 1       MMA issuer (2 k-steps x 3 products per stage).  Every FLUSH stages the accumulator is
@@ -41,7 +41,8 @@ namespace tc1 {
 
 constexpr int TR = 32;                         // data rows per stage (4 k-steps)
 constexpr int CHUNK_BYTES = TR * 128;          // one box: TR rows x 32 floats
-constexpr int NTHREADS = 14 * 32;
+constexpr int NTEAMS = 3;                      // vector / split teams of four warps, taking stages round-robin
+constexpr int NTHREADS = (6 + 4 * NTEAMS) * 32;
 constexpr int MAX_RING = 8;
 constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
 constexpr int ATOM_BYTES = TR * 128;           // one MN atom of an image: 64 columns (128 bytes) x TR rows
@@ -117,7 +118,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t tmem_base_s;
     __shared__ __align__(16) float sp[128];
-    __shared__ double sq[2][8];
+    __shared__ double sq[2][4 * NTEAMS];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NBX = d / 32;                        // X-hat boxes per stage
@@ -164,15 +165,15 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
 
     const float cf = ctl->c_f;
     const int dual = ctl->dual_pending;
-    // power-of-two operand scales (see the header): x-hat 2^15, w 2^eW with |w| 2^eW <= 2^14
-    int eW;
+    // power-of-two operand scales (see the header): x-hat 2^15, u 2^eU with |u| 2^eU <= 2^14
+    int eU;
     {
         int e;
-        frexpf(sqrtf((float)K) / cf, &e);              // sqrt(K) / c_f <= 2^e
-        eW = 14 - e;
+        frexpf(sqrtf((float)K), &e);                   // |u_ij| <= ||U||_F = sqrt(K) <= 2^e
+        eU = 14 - e;
     }
-    const float sW = ldexpf(1.0f, eW), sX = 32768.0f;
-    const double unscale = (double)cf * ldexp(1.0, -15 - eW);
+    const float sU = ldexpf(1.0f, eU), sX = 32768.0f;
+    const double unscale = ldexp(1.0, -15 - eU);
     double qq = 0.0, yq = 0.0;
     float s_acc[4] = {0.f, 0.f, 0.f, 0.f};         // vector warps: s partial of this lane's 4 columns
     double* const out = part + (size_t)blockIdx.x * ((size_t)d * r + r + 2);
@@ -224,9 +225,10 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         // ------------------------------ vector pass + split ------------------------------
         // One warp per row at a time: lane = (U chunk, 16-byte piece), i.e. the 32 lanes read the 4 x 8
         // pieces of one row -- every quarter-warp covers one full 128-byte line, no bank conflicts.
-        // Two teams of four warps take alternate stages, so the fixed latencies of a stage (barrier
-        // wake-ups, fence, hand-over to the MMA issuer) of one team overlap the work of the other.
-        const int vw = warp - 6;                           // 0..7
+        // NTEAMS teams of four warps take the stages round-robin: a stage costs a team about 3,400 cycles of
+        // mostly dependent latency (reductions, FP64 row scalars, conversions) against a budget of ~900, so
+        // several stages have to be in flight.
+        const int vw = warp - 6;                           // 0 .. 4 NTEAMS - 1
         const int team = vw >> 2, tw = vw & 3;             // team; rows tw + 4 k (k = 0..7) of the team's stages
         const int tt = (vw & 3) * 32 + lane;               // 0..127 inside the team
         const int box = lane >> 3, c = lane & 7;           // U chunk (32 columns) and logical 16-byte piece inside it
@@ -239,12 +241,12 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             const int64_t row_f = (g_lo + team) * TR + tw + 4 * (lane & 7);
             if (lane < 8 && row_f < n) yt_next = ytilde[row_f];
         }
-        for (int g = team; g < my_stages; g += 2) {
+        for (int g = team; g < my_stages; g += NTEAMS) {
             const int s = g % NSR, l = g % NLO;
             const int64_t srow0 = (g_lo + g) * TR;
             const int64_t myrow = srow0 + tw + 4 * (lane & 7);
             float yt_l = yt_next;
-            yt_next = (g + 2 < my_stages && lane < 8 && myrow + 2 * TR < n) ? ytilde[myrow + 2 * TR] : 0.f;
+            yt_next = (g + NTEAMS < my_stages && lane < 8 && myrow + NTEAMS * TR < n) ? ytilde[myrow + NTEAMS * TR] : 0.f;
             float yb_l = 0.f;
             mbar_wait(full(s), (g / NSR) & 1, &abort_flag, ctl);
             if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
@@ -253,7 +255,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             for (int half = 0; half < 2; ++half) {
                 // four independent rows at a time: loads first, reductions interleaved, then scalars and stores
                 uint32_t off[4];
-                float4 u4[4], w4[4];
+                float4 u4[4];
                 float dot[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
@@ -261,6 +263,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     off[k] = (uint32_t)(box * CHUNK_BYTES + rl * 128 + c * 16);
                 }
                 {
+                    float4 w4[4];
 #pragma unroll
                     for (int k = 0; k < 4; ++k)      // boxes beyond r are never loaded: their columns are zero
                         w4[k] = (box < NBU) ? lds128(hi_s + off[k]) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -293,9 +296,9 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     const float yb = __shfl_sync(0xffffffffu, yb_l, half * 4 + k);
                     s_acc[0] = fmaf(u4[k].x, yb, s_acc[0]); s_acc[1] = fmaf(u4[k].y, yb, s_acc[1]);   // rows beyond n: u = 0
                     s_acc[2] = fmaf(u4[k].z, yb, s_acc[2]); s_acc[3] = fmaf(u4[k].w, yb, s_acc[3]);
-                    // image of the unscaled factor entries w 2^eW; c_f is applied when the accumulator is folded
+                    // image of u 2^eU (u = c_f w rounded to FP32, as the plain definition has it)
                     uint2 h1, h2;
-                    split_h4(make_float4(w4[k].x * sW, w4[k].y * sW, w4[k].z * sW, w4[k].w * sW), h1, h2);
+                    split_h4(make_float4(u4[k].x * sU, u4[k].y * sU, u4[k].z * sU, u4[k].w * sU), h1, h2);
                     const uint32_t io = img_off(tw + 4 * (half * 4 + k), col0);
                     sts64(im + io, h1);
                     sts64(im + 2 * ATOM_BYTES + io, h2);
@@ -361,7 +364,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
-    float* sscr = reinterpret_cast<float*>(smem);             // [8 vector warps][128 columns]
+    float* sscr = reinterpret_cast<float*>(smem);             // [vector warps][128 columns]
     if (warp >= 6) {
         const int col0 = (lane >> 3) * 32 + 4 * (lane & 7);
 #pragma unroll
@@ -370,12 +373,12 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     __syncthreads();
     if (threadIdx.x < r) {
         double v = 0.0;
-        for (int k = 0; k < 8; ++k) v += (double)sscr[k * 128 + threadIdx.x];
+        for (int k = 0; k < 4 * NTEAMS; ++k) v += (double)sscr[k * 128 + threadIdx.x];
         out[(size_t)d * r + threadIdx.x] = v;
     }
     if (threadIdx.x == 0) {
         double a0 = 0.0, a1 = 0.0;
-        for (int w = 0; w < 8; ++w) { a0 += sq[0][w]; a1 += sq[1][w]; }
+        for (int w = 0; w < 4 * NTEAMS; ++w) { a0 += sq[0][w]; a1 += sq[1][w]; }
         out[(size_t)d * r + r] = a0;
         out[(size_t)d * r + r + 1] = a1;
     }
