@@ -12,9 +12,13 @@
 // of 8), and an MMA instruction costs the same ~130-180 cycles whatever K is: at N = d = 64 the TF32
 // version of this kernel was bound by exactly that instruction rate.
 //
-// The contraction runs over the data rows, so both operands are MN-major: per stage of TR = 32 rows the
-// split warps write fp16 images in the canonical MN-major 128-byte-swizzle layout (atoms of 64 columns
-// x 8 rows = 8 x 128 bytes, 16-byte chunk index XOR row mod 8; K atoms 1 KB apart, MN atoms 4 KB apart).
+// The contraction runs over the data rows, which is the slow (MN-major) operand orientation of the
+// tensor core: MN-major operands are fetched at about 9 elements per clock whatever their type.  The
+// split warps touch every entry anyway, so they write the fp16 images transposed, K-major: one 64-byte
+// row (the 32 data rows of a stage) per column of U / feature of X-hat, 64-byte swizzle (16-byte chunk
+// index XOR (row >> 1) mod 4).  A lane owns columns lane + 32 j and a warp eight consecutive data rows, so
+// a lane holds the 8 K-values of a chunk and writes it with one conflict-free 16-byte store.  With
+// K-major operands an M = 128, N = d MMA costs about 130 cycles: 6 per stage, under the HBM budget.
 // The accumulator is Theta^T: TMEM lane = column j of U (M = 128, columns beyond r are zero), TMEM
 // column = feature f (N = d).
 //
@@ -45,19 +49,18 @@ constexpr int NTEAMS = 3;                      // vector / split teams of four w
 constexpr int NTHREADS = (6 + 4 * NTEAMS) * 32;
 constexpr int MAX_RING = 8;
 constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
-constexpr int ATOM_BYTES = TR * 128;           // one MN atom of an image: 64 columns (128 bytes) x TR rows
+constexpr int UIMG = 128 * 64;                 // one fp16 image of the U operand: 128 columns x 32 data rows
 
-// Shared-memory matrix descriptor of an MN-major fp16 operand in the 128-byte-swizzle layout:
-// leading byte offset = distance between MN atoms (64 columns), stride byte offset = distance between
-// K atoms (8 rows).
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+// Shared-memory matrix descriptor, K-major operand with the 64-byte swizzle: 64-byte rows, groups
+// of 8 rows 512 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k_sw64(uint32_t smem_addr)
 {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)(16u >> 4) << 16;
+    d |= (uint64_t)(512u >> 4) << 32;
     d |= (uint64_t)1 << 46;          // version
-    d |= (uint64_t)2 << 61;          // SWIZZLE_128B
+    d |= (uint64_t)4 << 61;          // SWIZZLE_64B
     return d;
 }
 
@@ -83,26 +86,38 @@ __device__ __forceinline__ void umma_f16_x3(uint32_t tmem_d, uint64_t a1, uint64
         : "memory");
 }
 
-// v (already scaled) -> (h1, h2) packed for 4 consecutive entries: 8 bytes each.
-__device__ __forceinline__ void split_h4(const float4 v, uint2& h1, uint2& h2)
+// Eight scaled values (consecutive data rows of one column) -> the two fp16 chunks h1, h2 (16 bytes each).
+__device__ __forceinline__ void split_h8(const float* v, uint4& h1, uint4& h2)
 {
-    const __half2 a01 = __floats2half2_rn(v.x, v.y), a23 = __floats2half2_rn(v.z, v.w);
-    const float2 f01 = __half22float2(a01), f23 = __half22float2(a23);
-    const __half2 b01 = __floats2half2_rn(v.x - f01.x, v.y - f01.y), b23 = __floats2half2_rn(v.z - f23.x, v.w - f23.y);
-    h1 = make_uint2(*reinterpret_cast<const uint32_t*>(&a01), *reinterpret_cast<const uint32_t*>(&a23));
-    h2 = make_uint2(*reinterpret_cast<const uint32_t*>(&b01), *reinterpret_cast<const uint32_t*>(&b23));
+    uint32_t a[4], b[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __half2 hi = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
+        const float2 f = __half22float2(hi);
+        const __half2 lo = __floats2half2_rn(v[2 * i] - f.x, v[2 * i + 1] - f.y);
+        a[i] = *reinterpret_cast<const uint32_t*>(&hi);
+        b[i] = *reinterpret_cast<const uint32_t*>(&lo);
+    }
+    h1 = make_uint4(a[0], a[1], a[2], a[3]);
+    h2 = make_uint4(b[0], b[1], b[2], b[3]);
 }
 
-__device__ __forceinline__ void sts64(uint32_t addr, uint2 v)
+__device__ __forceinline__ void sts128u(uint32_t addr, uint4 v)
 {
-    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(v.x), "r"(v.y) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// Byte offset of 4 consecutive columns starting at column c (multiple of 4) of row rl inside an image
-// (MN atoms of 64 columns ATOM_BYTES apart, 128-byte rows, 16-byte chunk index XOR row mod 8).
-__device__ __forceinline__ uint32_t img_off(int rl, int c)
+__device__ __forceinline__ float lds32f(uint32_t addr)
 {
-    return (uint32_t)((c >> 6) * ATOM_BYTES + rl * 128 + ((((c & 63) >> 3) ^ (rl & 7)) << 4) + (c & 7) * 2);
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
+// Byte offset inside a K-major image of the 16-byte chunk holding data rows 8 kg .. 8 kg + 7 of MN row m.
+__device__ __forceinline__ uint32_t kimg_off(int m, int kg)
+{
+    return (uint32_t)(m * 64 + ((kg ^ ((m >> 1) & 3)) << 4));
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -124,8 +139,8 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     const int NBX = d / 32;                        // X-hat boxes per stage
     const int NBU = (r + 31) / 32;                 // U boxes per stage (M = 128 reads 4; missing ones are never written: see below)
     const int STAGE = (4 + NBX) * CHUNK_BYTES;     // raw stage: 4 U boxes then the X-hat boxes (FP32 rows of 128 bytes)
-    const int NXA = (d + 63) / 64;                 // MN atoms of an X-hat image
-    const int IMG = (2 * 2 + 2 * NXA) * ATOM_BYTES;   // image stage: U h1 (2 atoms), U h2, X h1, X h2
+    const int XIMG = d * 64;                       // one fp16 image of the X-hat operand: d features x 32 data rows
+    const int IMG = 2 * UIMG + 2 * XIMG;           // image stage: U h1, U h2, X h1, X h2
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * d) tmem_cols <<= 1;
 
@@ -194,7 +209,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f16(128, d, 1, 1);
+            const uint32_t idesc = umma_idesc_f16(128, d, 0, 0);
             // The wait for the next stage sits between the two k-steps of the current one, so the tensor pipe
             // has MMAs queued while this thread polls.
             if (my_stages > 0) mbar_wait(split(0), 0, &abort_flag, ctl);
@@ -205,16 +220,15 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * d);
                 const uint32_t im = img0 + (uint32_t)l * IMG;
-                // A = U images (M = 128: 2 MN atoms), B = X-hat images (N = d); MN atoms ATOM_BYTES apart (LBO),
-                // K atoms of 8 rows 1 KB apart (SBO); a k-step of 16 rows advances the start address by 2 KB
-                const uint64_t da1 = umma_desc_mn_sw128(im, ATOM_BYTES, 1024), da2 = umma_desc_mn_sw128(im + 2 * ATOM_BYTES, ATOM_BYTES, 1024);
-                const uint64_t db1 = umma_desc_mn_sw128(im + 4 * ATOM_BYTES, ATOM_BYTES, 1024);
-                const uint64_t db2 = umma_desc_mn_sw128(im + (4 + NXA) * ATOM_BYTES, ATOM_BYTES, 1024);
+                // A = U images (M = 128 columns), B = X-hat images (N = d features), K-major; a k-step of 16 data
+                // rows (32 bytes inside the 64-byte swizzled row) advances the start address by 2
+                const uint64_t da1 = umma_desc_k_sw64(im), da2 = umma_desc_k_sw64(im + UIMG);
+                const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG), db2 = umma_desc_k_sw64(im + 2 * UIMG + XIMG);
 #pragma unroll
                 for (int ks = 0; ks < TR / 16; ++ks) {
                     if (ks == 1 && g + 1 < my_stages)
                         mbar_wait(split((g + 1) % NLO), ((g + 1) / NLO) & 1, &abort_flag, ctl);
-                    umma_f16_x3(tacc, da1 + 128 * ks, da2 + 128 * ks, db1 + 128 * ks, db2 + 128 * ks, idesc,
+                    umma_f16_x3(tacc, da1 + 2 * ks, da2 + 2 * ks, db1 + 2 * ks, db2 + 2 * ks, idesc,
                                 (in_period | ks) ? 1u : 0u);
                 }
                 umma_commit(lofree(l));
@@ -223,103 +237,96 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         }
     } else if (warp >= 6) {
         // ------------------------------ vector pass + split ------------------------------
-        // One warp per row at a time: lane = (U chunk, 16-byte piece), i.e. the 32 lanes read the 4 x 8
-        // pieces of one row -- every quarter-warp covers one full 128-byte line, no bank conflicts.
-        // NTEAMS teams of four warps take the stages round-robin: a stage costs a team about 3,400 cycles of
-        // mostly dependent latency (reductions, FP64 row scalars, conversions) against a budget of ~900, so
-        // several stages have to be in flight.
+        // A warp takes 8 consecutive data rows of a stage, a lane the columns lane + 32 j of U (scalar loads
+        // from the plain FP32 rows: consecutive lanes, consecutive words).  NTEAMS teams of four warps take
+        // the stages round-robin: a stage costs a team a few thousand cycles of mostly dependent latency
+        // (reductions, FP64 row scalars, conversions) against a budget of ~900, so several are in flight.
         const int vw = warp - 6;                           // 0 .. 4 NTEAMS - 1
-        const int team = vw >> 2, tw = vw & 3;             // team; rows tw + 4 k (k = 0..7) of the team's stages
-        const int tt = (vw & 3) * 32 + lane;               // 0..127 inside the team
-        const int box = lane >> 3, c = lane & 7;           // U chunk (32 columns) and logical 16-byte piece inside it
-        const int col0 = box * 32 + 4 * c;                 // first of this lane's 4 columns of u
-        const float4 p4 = *reinterpret_cast<const float4*>(sp + col0);
-        // ytilde of this warp's eight rows (lane k < 8 holds row tw + 4 k) is requested one of the team's
+        const int team = vw >> 2, tw = vw & 3;             // team; data rows 8 tw .. 8 tw + 7 of the team's stages
+        const int tt = tw * 32 + lane;                     // 0..127 inside the team
+        float p1[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) p1[j] = sp[lane + 32 * j];
+        // ytilde of this warp's eight rows (lane k < 8 holds row 8 tw + k) is requested one of the team's
         // stages ahead, so its DRAM latency is not paid inside the stage
         float yt_next = 0.f;
         if (team < my_stages) {
-            const int64_t row_f = (g_lo + team) * TR + tw + 4 * (lane & 7);
+            const int64_t row_f = (g_lo + team) * TR + 8 * tw + (lane & 7);
             if (lane < 8 && row_f < n) yt_next = ytilde[row_f];
         }
         for (int g = team; g < my_stages; g += NTEAMS) {
             const int s = g % NSR, l = g % NLO;
             const int64_t srow0 = (g_lo + g) * TR;
-            const int64_t myrow = srow0 + tw + 4 * (lane & 7);
+            const int64_t myrow = srow0 + 8 * tw + (lane & 7);
             float yt_l = yt_next;
             yt_next = (g + NTEAMS < my_stages && lane < 8 && myrow + NTEAMS * TR < n) ? ytilde[myrow + NTEAMS * TR] : 0.f;
             float yb_l = 0.f;
             mbar_wait(full(s), (g / NSR) & 1, &abort_flag, ctl);
             if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
             const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, im = img0 + (uint32_t)l * IMG;
+            float u[8][4], dot[8];
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                // four independent rows at a time: loads first, reductions interleaved, then scalars and stores
-                uint32_t off[4];
-                float4 u4[4];
-                float dot[4];
+            for (int k = 0; k < 8; ++k) {
+                dot[k] = 0.f;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int rl = tw + 4 * (half * 4 + k);
-                    off[k] = (uint32_t)(box * CHUNK_BYTES + rl * 128 + c * 16);
+                for (int j = 0; j < 4; ++j) {        // boxes beyond r are never loaded: their columns are zero
+                    const float w = (j < NBU) ? lds32f(hi_s + (uint32_t)(j * CHUNK_BYTES + (8 * tw + k) * 128 + lane * 4)) : 0.f;
+                    u[k][j] = cf * w;
+                    dot[k] = fmaf(u[k][j], p1[j], dot[k]);
                 }
-                {
-                    float4 w4[4];
+            }
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)      // boxes beyond r are never loaded: their columns are zero
-                        w4[k] = (box < NBU) ? lds128(hi_s + off[k]) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        u4[k] = make_float4(cf * w4[k].x, cf * w4[k].y, cf * w4[k].z, cf * w4[k].w);
-                        dot[k] = fmaf(u4[k].x, p4.x, fmaf(u4[k].y, p4.y, fmaf(u4[k].z, p4.z, u4[k].w * p4.w)));
+                for (int k = 0; k < 8; ++k) dot[k] += __shfl_xor_sync(0xffffffffu, dot[k], o);
+            // row scalars: lane k < 8 owns row 8 tw + k (dot[] is the same in every lane)
+            {
+                float q = dot[0];
+#pragma unroll
+                for (int k = 1; k < 8; ++k) q = ((lane & 7) == k) ? dot[k] : q;
+                const float qm1 = q - 1.0f;
+                if (lane < 8) {
+                    if (dual) yt_l = (float)((double)yt_l + gamma * (double)qm1);
+                    yb_l = (float)((double)yt_l + gamma * (double)qm1);
+                    if (myrow < n) {
+                        qq = fma((double)qm1, (double)qm1, qq);
+                        yq = fma((double)yt_l, (double)qm1, yq);
                     }
                 }
+            }
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1)
+            for (int k = 0; k < 8; ++k) {
+                const float yb = __shfl_sync(0xffffffffu, yb_l, k);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) dot[k] += __shfl_xor_sync(0xffffffffu, dot[k], o);
-                // row scalars: lane 4 half + k owns row tw + 4 (4 half + k) (dot[] is the same in every lane)
-                {
-                    const int kk = lane & 3;
-                    const float q = (kk == 0) ? dot[0] : (kk == 1) ? dot[1] : (kk == 2) ? dot[2] : dot[3];
-                    const float qm1 = q - 1.0f;
-                    if ((lane >> 2) == half) {
-                        if (dual) yt_l = (float)((double)yt_l + gamma * (double)qm1);
-                        yb_l = (float)((double)yt_l + gamma * (double)qm1);
-                        if (myrow < n) {
-                            qq = fma((double)qm1, (double)qm1, qq);
-                            yq = fma((double)yt_l, (double)qm1, yq);
-                        }
-                    }
-                }
+                for (int j = 0; j < 4; ++j) s_acc[j] = fmaf(u[k][j], yb, s_acc[j]);     // rows beyond n: u = 0
+            }
+            // images of u 2^eU (u = c_f w rounded to FP32, as the plain definition has it): one chunk per column
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float yb = __shfl_sync(0xffffffffu, yb_l, half * 4 + k);
-                    s_acc[0] = fmaf(u4[k].x, yb, s_acc[0]); s_acc[1] = fmaf(u4[k].y, yb, s_acc[1]);   // rows beyond n: u = 0
-                    s_acc[2] = fmaf(u4[k].z, yb, s_acc[2]); s_acc[3] = fmaf(u4[k].w, yb, s_acc[3]);
-                    // image of u 2^eU (u = c_f w rounded to FP32, as the plain definition has it)
-                    uint2 h1, h2;
-                    split_h4(make_float4(u4[k].x * sU, u4[k].y * sU, u4[k].z * sU, u4[k].w * sU), h1, h2);
-                    const uint32_t io = img_off(tw + 4 * (half * 4 + k), col0);
-                    sts64(im + io, h1);
-                    sts64(im + 2 * ATOM_BYTES + io, h2);
-                }
+            for (int j = 0; j < 4; ++j) {
+                float v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[k] = u[k][j] * sU;
+                uint4 h1, h2;
+                split_h8(v, h1, h2);
+                const uint32_t io = kimg_off(lane + 32 * j, tw);
+                sts128u(im + io, h1);
+                sts128u(im + UIMG + io, h2);
             }
             if (lane < 8 && myrow < n) {
                 if (dual) ytilde[myrow] = yt_l;
                 ybar[myrow] = yb_l;
             }
-            // ---- X-hat boxes -> fp16 images: 256 float4 per box, two per thread of the team ----
+            // ---- X-hat boxes -> fp16 images: thread = (feature tt & 31, data rows 8 (tt >> 5) .. + 7) of a box ----
             for (int b = 0; b < NBX; ++b) {
+                float v[8];
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int idx = tt + 128 * hh, rr = idx >> 3, f0 = b * 32 + 4 * (idx & 7);
-                    const float4 x = lds128(hi_s + (uint32_t)((4 + b) * CHUNK_BYTES) + (uint32_t)idx * 16);
-                    uint2 h1, h2;
-                    split_h4(make_float4(x.x * sX, x.y * sX, x.z * sX, x.w * sX), h1, h2);
-                    const uint32_t io = img_off(rr, f0);
-                    sts64(im + 4 * ATOM_BYTES + io, h1);
-                    sts64(im + (4 + NXA) * ATOM_BYTES + io, h2);
-                }
+                for (int k = 0; k < 8; ++k)
+                    v[k] = sX * lds32f(hi_s + (uint32_t)((4 + b) * CHUNK_BYTES + (8 * tw + k) * 128 + lane * 4));
+                uint4 h1, h2;
+                split_h8(v, h1, h2);
+                const uint32_t io = kimg_off(b * 32 + lane, tw);
+                sts128u(im + 2 * UIMG + io, h1);
+                sts128u(im + 2 * UIMG + XIMG + io, h2);
             }
             fence_proxy_async();
             __syncwarp();
@@ -366,9 +373,8 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
     float* sscr = reinterpret_cast<float*>(smem);             // [vector warps][128 columns]
     if (warp >= 6) {
-        const int col0 = (lane >> 3) * 32 + 4 * (lane & 7);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + col0 + k] = s_acc[k];
+        for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + lane + 32 * k] = s_acc[k];
     }
     __syncthreads();
     if (threadIdx.x < r) {
@@ -391,9 +397,9 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     const int d = pb.P.d, r = pb.P.r;
     if (d % 32 != 0 || d > 256 || r % 4 != 0 || r < 8 || r > 128 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
     if ((size_t)d * r > 16384) return false;          // partial records of the shared reduction kernel
-    const int NBX = d / 32, NXA = (d + 63) / 64;
+    const int NBX = d / 32;
     const size_t stage = (size_t)(4 + NBX) * tc1::CHUNK_BYTES;
-    const size_t img = (size_t)(4 + 2 * NXA) * tc1::ATOM_BYTES;
+    const size_t img = (size_t)2 * tc1::UIMG + (size_t)2 * d * 64;
     const size_t limit = 227 * 1024 - 2048;
     int NLO = 0, NSR = 0;
     for (int nlo = 4; nlo >= 2 && !NSR; --nlo)
