@@ -66,6 +66,31 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     ctl->stopped = 1;
 }
 
+// Same bounded wait for roles that are not on the critical path of the tensor pipe: the hardware may
+// suspend the thread for up to ~1 us per attempt instead of letting it poll, so that waiting warps do not
+// take issue slots from the single thread that issues the MMAs on the same scheduler.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ void mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                  Ctl* ctl)
+{
+    if (*abort_flag) return;
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait_suspend(bar, parity, 1000u)) return;
+    *abort_flag = 1u;
+    ctl->status = GEM_NLR_E_TIMEOUT;
+    ctl->stopped = 1;
+}
+
 // Tile load: box of the tensor map at element coordinates (x = column, y = row).  x * 4 bytes
 // must be a multiple of 16.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar)
