@@ -198,7 +198,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int s = g % NSR;
-                if (g >= NSR) mbar_wait_relaxed(rawfree(s), ((g / NSR) - 1) & 1, &abort_flag, ctl);
+                if (g >= NSR) mbar_wait_spin(rawfree(s), ((g / NSR) - 1) & 1, &abort_flag, ctl);
                 const int row0 = (int)((g_lo + g) * TR);
                 const uint32_t dst = raw0 + (uint32_t)s * STAGE;
                 mbar_expect_tx(full(s), (uint32_t)(NBU + NBX) * CHUNK_BYTES);
@@ -212,12 +212,12 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             const uint32_t idesc = umma_idesc_f16(128, d, 0, 0);
             // The wait for the next stage sits between the two k-steps of the current one, so the tensor pipe
             // has MMAs queued while this thread polls.
-            if (my_stages > 0) mbar_wait(split(0), 0, &abort_flag, ctl);
+            if (my_stages > 0) mbar_wait_spin(split(0), 0, &abort_flag, ctl);
             // image slot l and its phase, accumulator a and position in the accumulation period: kept
             // incrementally (this thread's instruction stream is the critical path of the kernel)
             int l = 0, lph = 0, a = 0, in_period = 0, period = 0;
             for (int g = 0; g < my_stages; ++g) {
-                if (in_period == 0 && period >= 2) mbar_wait(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
+                if (in_period == 0 && period >= 2) mbar_wait_spin(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * d);
                 const uint32_t im = img0 + (uint32_t)l * IMG;
@@ -228,7 +228,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
                 int ln = l + 1, lphn = lph;
                 if (ln == NLO) { ln = 0; lphn ^= 1; }
-                if (g + 1 < my_stages) mbar_wait(split(ln), (uint32_t)lphn, &abort_flag, ctl);
+                if (g + 1 < my_stages) mbar_wait_spin(split(ln), (uint32_t)lphn, &abort_flag, ctl);
                 umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
                 umma_commit(lofree(l));
                 if (in_period == FLUSH - 1 || g == my_stages - 1) umma_commit(accfull(a));
@@ -263,8 +263,8 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             float yt_l = yt_next;
             yt_next = (g + NTEAMS < my_stages && lane < 8 && myrow + NTEAMS * TR < n) ? ytilde[myrow + NTEAMS * TR] : 0.f;
             float yb_l = 0.f;
-            mbar_wait_relaxed(full(s), (g / NSR) & 1, &abort_flag, ctl);
-            if (g >= NLO) mbar_wait_relaxed(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+            mbar_wait_spin(full(s), (g / NSR) & 1, &abort_flag, ctl);
+            if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
             const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, im = img0 + (uint32_t)l * IMG;
             float u[8][4], dot[8];
 #pragma unroll

@@ -66,6 +66,27 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     ctl->stopped = 1;
 }
 
+// Bounded wait by polling (mbarrier.test_wait never suspends the thread): for the hand-overs on the critical
+// path of a pipeline, where the suspension period of try_wait (of the order of a microsecond) would be
+// paid on every stage.
+__device__ __forceinline__ void mbar_wait_spin(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               Ctl* ctl)
+{
+    if (*abort_flag) return;
+    for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return;
+    }
+    *abort_flag = 1u;
+    ctl->status = GEM_NLR_E_TIMEOUT;
+    ctl->stopped = 1;
+}
+
 // Same bounded wait for roles that are not on the critical path of the tensor pipe: the hardware may
 // suspend the thread for up to ~1 us per attempt instead of letting it poll, so that waiting warps do not
 // take issue slots from the single thread that issues the MMAs on the same scheduler.
