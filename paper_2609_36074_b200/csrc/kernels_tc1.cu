@@ -23,7 +23,8 @@
 // column = feature f (N = d).
 //
 // One persistent CTA per SM, 14 warps:
-//   warp 0       producer: per stage ceil(r/32) U boxes and d/32 X-hat boxes (plain FP32 rows).
+//   warp 0       producer: per stage one bulk copy of the TR rows of U and one of X-hat (contiguous in
+//                global memory).
 //   warps 6-17   vector + split, three teams taking stages round-robin: one warp per row does the row-local
 //                vector work on the U boxes, then both operands are converted into the image ring;
 //                the raw stage goes back to the producer as soon as the team has read it.
@@ -121,7 +122,7 @@ __device__ __forceinline__ uint32_t kimg_off(int m, int kg)
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU,
+k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
            float* __restrict__ ytilde, float* __restrict__ ybar, Ctl* __restrict__ ctl,
            const float* __restrict__ p, int64_t n, int d, int r, int K, int NSR, int NLO, double gamma,
            double* __restrict__ part)
@@ -138,7 +139,10 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NBX = d / 32;                        // X-hat boxes per stage
     const int NBU = (r + 31) / 32;                 // U boxes per stage (M = 128 reads 4; missing ones are never written: see below)
-    const int STAGE = (4 + NBX) * CHUNK_BYTES;     // raw stage: 4 U boxes then the X-hat boxes (FP32 rows of 128 bytes)
+    // raw stage: the TR rows of U then those of X-hat exactly as they lie in global memory (row pitch r and
+    // d floats): the rows of a stage are contiguous there, so each operand arrives with one bulk copy
+    const int URAW = (TR * r * 4 + 127) / 128 * 128;
+    const int STAGE = (URAW + TR * d * 4 + 1023) / 1024 * 1024;
     const int XIMG = d * 64;                       // one fp16 image of the X-hat operand: d features x 32 data rows
     const int IMG = 2 * UIMG + 2 * XIMG;           // image stage: U h1, U h2, X h1, X h2
     uint32_t tmem_cols = 32;
@@ -199,11 +203,12 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int s = g % NSR;
                 if (g >= NSR) mbar_wait_spin(rawfree(s), ((g / NSR) - 1) & 1, &abort_flag, ctl);
-                const int row0 = (int)((g_lo + g) * TR);
+                const int64_t row0 = (g_lo + g) * TR;
+                const int rows = (n - row0 < TR) ? (int)(n - row0) : TR;
                 const uint32_t dst = raw0 + (uint32_t)s * STAGE;
-                mbar_expect_tx(full(s), (uint32_t)(NBU + NBX) * CHUNK_BYTES);
-                for (int c = 0; c < NBU; ++c) tma_load_2d(dst + c * CHUNK_BYTES, &tmU, c * 32, row0, full(s));
-                for (int b = 0; b < NBX; ++b) tma_load_2d(dst + (4 + b) * CHUNK_BYTES, &tmX, b * 32, row0, full(s));
+                mbar_expect_tx(full(s), (uint32_t)(rows * (r + d) * 4));
+                bulk_load_1d(dst, U + row0 * r, (uint32_t)(rows * r * 4), full(s));
+                bulk_load_1d(dst + URAW, X + row0 * d, (uint32_t)(rows * d * 4), full(s));
             }
         }
     } else if (warp == 1) {
@@ -266,13 +271,15 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             mbar_wait_spin(full(s), (g / NSR) & 1, &abort_flag, ctl);
             if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
             const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, im = img0 + (uint32_t)l * IMG;
+            const int rows_here = (n - srow0 < TR) ? (int)(n - srow0) : TR;
             float u[8][4], dot[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 dot[k] = 0.f;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {        // boxes beyond r are never loaded: their columns are zero
-                    const float w = (j < NBU) ? lds32f(hi_s + (uint32_t)(j * CHUNK_BYTES + (8 * tw + k) * 128 + lane * 4)) : 0.f;
+                for (int j = 0; j < 4; ++j) {        // columns beyond r and rows beyond n are zero
+                    const float w = (lane + 32 * j < r && 8 * tw + k < rows_here)
+                                        ? lds32f(hi_s + (uint32_t)(((8 * tw + k) * r + lane + 32 * j) * 4)) : 0.f;
                     u[k][j] = cf * w;
                     dot[k] = fmaf(u[k][j], p1[j], dot[k]);
                 }
@@ -323,7 +330,7 @@ k_pass1_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 float v[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    v[k] = sX * lds32f(hi_s + (uint32_t)((4 + b) * CHUNK_BYTES + (8 * tw + k) * 128 + lane * 4));
+                    v[k] = (8 * tw + k < rows_here) ? sX * lds32f(hi_s + (uint32_t)(URAW + ((8 * tw + k) * d + b * 32 + lane) * 4)) : 0.f;
                 uint4 h1, h2;
                 split_h8(v, h1, h2);
                 const uint32_t io = kimg_off(b * 32 + lane, tw);
@@ -400,7 +407,7 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     if (d % 32 != 0 || d > 256 || r % 4 != 0 || r < 8 || r > 128 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
     if ((size_t)d * r > 16384) return false;          // partial records of the shared reduction kernel
     const int NBX = d / 32;
-    const size_t stage = (size_t)(4 + NBX) * tc1::CHUNK_BYTES;
+    const size_t stage = (((size_t)tc1::TR * r * 4 + 127) / 128 * 128 + (size_t)tc1::TR * d * 4 + 1023) / 1024 * 1024;
     const size_t img = (size_t)2 * tc1::UIMG + (size_t)2 * d * 64;
     const size_t limit = 227 * 1024 - 2048;
     int NLO = 0, NSR = 0;
@@ -411,8 +418,6 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     pl->NSR = NSR; pl->NLO = NLO;
     pl->smem = (size_t)NSR * stage + (size_t)NLO * img + 1024;
     if (pl->smem < (size_t)8 * 128 * 4 + 1024) pl->smem = (size_t)8 * 128 * 4 + 1024;     // s scratch of the tail
-    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc1::TR, 32, false, 1)) return false;      // plain rows
-    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tc1::TR, 32, false, 1)) return false;
     const int64_t stages = (pb.P.n + tc1::TR - 1) / tc1::TR;
     pl->grid = (int)(stages < kSMs ? stages : kSMs);
     if (cudaFuncSetAttribute(tc1::k_pass1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess)
@@ -423,7 +428,7 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
 void tc1_launch_first(const Problem& pb, const Tc1Plan& pl)
 {
     tc1::k_pass1_tc<<<pl.grid, tc1::NTHREADS, pl.smem, pb.stream>>>(
-        pl.tmX, pl.tmU, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.P.d, pb.P.r, pb.P.K, pl.NSR, pl.NLO, pb.gamma,
+        pb.X, pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.P.d, pb.P.r, pb.P.K, pl.NSR, pl.NLO, pb.gamma,
         pb.part1());
     pb.count(1);
 }
