@@ -39,7 +39,6 @@
 #include "pipeline.cuh"
 #include "tc_common.cuh"
 #include "tc_family.cuh"
-#include <cuda_fp16.h>
 
 namespace gemnlr {
 namespace tc1 {
@@ -51,75 +50,6 @@ constexpr int NTHREADS = (6 + 4 * NTEAMS) * 32;
 constexpr int MAX_RING = 8;
 constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
 constexpr int UIMG = 128 * 64;                 // one fp16 image of the U operand: 128 columns x 32 data rows
-
-// Shared-memory matrix descriptor, K-major operand with the 64-byte swizzle: 64-byte rows, groups
-// of 8 rows 512 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_k_sw64(uint32_t smem_addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
-    d |= (uint64_t)(16u >> 4) << 16;
-    d |= (uint64_t)(512u >> 4) << 32;
-    d |= (uint64_t)1 << 46;          // version
-    d |= (uint64_t)4 << 61;          // SWIZZLE_64B
-    return d;
-}
-
-// Instruction descriptor for kind::f16 with fp16 operands, FP32 accumulate, M x N tile.
-__host__ __device__ constexpr uint32_t umma_idesc_f16(int M, int N, int a_mn, int b_mn)
-{
-    return (1u << 4) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
-}
-
-// D (+)= A1 B1 + A2 B1 + A1 B2 (one k-step of 16 of the two-term fp16 split).
-__device__ __forceinline__ void umma_f16_x3(uint32_t tmem_d, uint64_t a1, uint64_t a2, uint64_t b1, uint64_t b2,
-                                            uint32_t idesc, uint32_t accumulate_first)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, t;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "setp.eq.b32 t, %7, %7;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %3, %5, {%7, %7, %7, %7}, p;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %3, %5, {%7, %7, %7, %7}, t;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %4, %5, {%7, %7, %7, %7}, t;\n\t}"
-        ::"r"(tmem_d), "l"(a1), "l"(a2), "l"(b1), "l"(b2), "r"(idesc), "r"(accumulate_first), "r"(0u)
-        : "memory");
-}
-
-// Eight scaled values (consecutive data rows of one column) -> the two fp16 chunks h1, h2 (16 bytes each).
-__device__ __forceinline__ void split_h8(const float* v, uint4& h1, uint4& h2)
-{
-    uint32_t a[4], b[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const __half2 hi = __floats2half2_rn(v[2 * i], v[2 * i + 1]);
-        const float2 f = __half22float2(hi);
-        const __half2 lo = __floats2half2_rn(v[2 * i] - f.x, v[2 * i + 1] - f.y);
-        a[i] = *reinterpret_cast<const uint32_t*>(&hi);
-        b[i] = *reinterpret_cast<const uint32_t*>(&lo);
-    }
-    h1 = make_uint4(a[0], a[1], a[2], a[3]);
-    h2 = make_uint4(b[0], b[1], b[2], b[3]);
-}
-
-__device__ __forceinline__ void sts128u(uint32_t addr, uint4 v)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-__device__ __forceinline__ float lds32f(uint32_t addr)
-{
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
-}
-
-// Byte offset inside a K-major image of the 16-byte chunk holding data rows 8 kg .. 8 kg + 7 of MN row m.
-__device__ __forceinline__ uint32_t kimg_off(int m, int kg)
-{
-    return (uint32_t)(m * 64 + ((kg ^ ((m >> 1) & 3)) << 4));
-}
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
