@@ -47,7 +47,6 @@ def _peaks():
 NCU_TRAFFIC_BYTES = {
     (1_000_000, 128, 16, "mma.tf32x3"): 640.0e6,
     (10_000_000, 64, 100, "tf32x3"): 10.385e9,
-    (2_000_000, 768, 1000, "tf32x3.tiled"): 22.93e9,
     (100_000_000, 32, 8, "ffma"): 19.49e9,
 }
 
@@ -271,9 +270,14 @@ def main():
     if prof_iters > 0:
         p2_s = ms_p2 * 1e-3 / prof_iters
         it_s = ms * 1e-3 / (args.steps * T)
-        tpeak, tpeak_kind = _tensor_peak_tf32()
-        # MMA flops actually issued on the tensor-core paths: three TF32 products per useful product
-        mma_mult = 3 if "tf32" in path else 0
+        # MMA flops actually issued on the tensor-core paths: three products per useful product; the fp16 split
+        # runs on the f16 pipe (peak = the measured bf16 figure), the TF32 split on the TF32 pipe
+        if "f16x3" in path:
+            tpeak, tpeak_kind = _tensor_peak_tf32()
+            tpeak, tpeak_kind = tpeak / TF32_OVER_BF16, "measured bf16 sustained (f16 pipe)"
+        else:
+            tpeak, tpeak_kind = _tensor_peak_tf32()
+        mma_mult = 3 if ("tf32" in path or "f16x3" in path) else 0
         t_hbm2 = second_product_bytes(n, d, r) / (peak * 1e9)
         t_tc2 = mma_mult * 2.0 * n * d * r / (tpeak * 1e12)
         iteration = {"algorithmic_bytes": algorithmic_bytes(n, d, r),
@@ -288,7 +292,7 @@ def main():
             roofline = {"bound": "tensor", "kernel": "second product + fused epilogue", "achieved": ach, "peak": tpeak,
                         "unit": "TFLOP/s", "frac": ach / tpeak, "peak_kind": tpeak_kind,
                         "flops_per_launch": mma_mult * 2.0 * n * d * r,
-                        "flops_note": "3 TF32 MMA products (hi*hi, lo*hi, hi*lo) per FP32-accurate product, 2ndr each",
+                        "flops_note": "3 tensor-core products (two-term operand split) per FP32-accurate product, 2ndr each",
                         "traffic": NCU_TRAFFIC_BYTES.get((n, d, r, path)), "ms_per_launch": p2_s * 1e3,
                         "first_phase_ms_per_iteration": ms_p1 / prof_iters, "iteration": iteration}
         else:

@@ -64,6 +64,12 @@ Layout make_layout(const gem_nlr_params& P)
     L.setup = take(sizeof(double) * (3 * (size_t)d + 4 + (size_t)L.gs * d));
     L.hist = take(P.history ? sizeof(gem_nlr_iter_info) * (size_t)(P.T > 0 ? P.T : 1) : 0);
     L.xhat = take(P.x_inplace ? 0 : sizeof(float) * (size_t)n * d);
+    // Wide tensor-core shapes (the tiled tcgen05 pair): X-hat is static, so its two-term fp16 split is built
+    // once, row-major (second product) and transposed (first product): 2 x 2 x n x d halves.
+    L.n_pad = (n + 63) / 64 * 64;
+    const bool wide_tc = (P.precision == -1 || P.precision == 1) && r > 256 && d % 32 == 0 && n >= 4096;
+    L.ximg = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)n * d : 0);
+    L.ximgT = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)d * L.n_pad : 0);
     L.total = off;
     return L;
 }
@@ -276,10 +282,10 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
         }
         else if (tcg_plan(h->pb, &h->tcg, img)) {
             h->use_tcg = true;
-            h->path = "generic+tf32x3.tiled";
+            h->path = "generic+f16x3.tiled";
             if (tcg1_plan(h->pb, &h->tcg1)) {
                 h->use_tcg1 = true;
-                h->path = "tf32x3.tiled";
+                h->path = "f16x3.tiled";
             }
         }
     }
@@ -317,6 +323,10 @@ int gem_nlr_spectral_norm(gem_nlr_t* h, double* a_out)
     CK(h, cudaStreamSynchronize(h->pb.stream));
     h->a = a;
     h->normalized = true;
+    if (h->use_tcg) {                                    // static fp16 images of X-hat for the tiled tensor-core kernels
+        tcg_prepare(h->pb);
+        CK(h, cudaStreamSynchronize(h->pb.stream));
+    }
     if (a_out) *a_out = a;
     return GEM_NLR_OK;
 }
@@ -327,6 +337,10 @@ int gem_nlr_set_normalized(gem_nlr_t* h, double a)
     if (!h->pb.P.x_inplace) return GEM_NLR_E_INVALID;  // X-hat must be in the caller's buffer
     h->a = a;
     h->normalized = true;
+    if (h->use_tcg) {
+        tcg_prepare(h->pb);
+        CK(h, cudaStreamSynchronize(h->pb.stream));
+    }
     return GEM_NLR_OK;
 }
 

@@ -49,6 +49,29 @@ bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int c
     return rc == CUDA_SUCCESS;
 }
 
+// 2D tensor map over a row-major fp16 matrix (rows x cols halves, row pitch pitch_halves), box of
+// box_rows x box_cols; box_cols * 2 bytes must be 64 (64-byte swizzle) or 128 (128-byte swizzle).
+bool make_tensor_map_2d_f16(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t pitch_halves,
+                            int box_rows, int box_cols)
+{
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn)
+        return false;
+    auto encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)pitch_halves * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapSwizzle sw = box_cols * 2 == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                : box_cols * 2 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE;
+    CUresult rc = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
 namespace ffma {
 
 constexpr int NCW = 8;                    // consumer warps

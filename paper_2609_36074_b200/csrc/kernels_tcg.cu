@@ -1,24 +1,27 @@
-// Tiled 3xTF32 tcgen05 second product for wide problems (d and r too large for the resident-Theta
-// kernel: the embedding-sized shape d = 768, r = 1000):
+// Tiled tensor-core kernels (tcgen05 + TMEM) for wide problems (d and r too large for the resident-Theta
+// kernels: the embedding-sized shape d = 768, r = 1000).  Second product:
 //   acc = X-hat Theta ;  W = [U + 2 alpha acc - alpha (ybar p^T + 1 s^T)]_+ in place ;  FP64 a, b, h ;
 //   column sums of W                                               (Eq. "entrywise-fusion", Algorithm 2 call 4)
 //
-// Work item = (128-row tile, 256-column block).  The K loop streams d in chunks of 16 features:
-// a stage holds the X-hat box (128 rows x 64 bytes, TMA with the 64-byte swizzle = K-major UMMA
-// operand) and the matching boxes of the pre-split Theta^T images (256 columns x 64 bytes, hi and
-// lo, already swizzled in global memory, one bulk copy each).  With M = 128, N = 256 a TF32
-// tcgen05.mma runs at the tensor pipe's full rate, and the accumulator (256 TMEM columns) is
+// FP32 accuracy from FP16 tensor cores: x 2^k = h1 + h2 with h1 = fp16(x 2^k), h2 = fp16(x 2^k - h1)
+// (22 significant bits), product accumulated in FP32 as h1 h1' + h2 h1' + h1 h2' (three K = 16 MMAs).
+// The scales are powers of two that cannot overflow: |x-hat_ij| <= ||X-hat||_2 = 1 (2^15) and
+// |Theta_jk| <= ||X-hat||_2 ||U||_F = sqrt(K).  X-hat is static, so its images are built once at setup
+// (k_ximg_build: row-major for this kernel, transposed for the first product) and arrive by TMA already
+// in the K-major 64-byte-swizzle layout; nothing is split inside this kernel.
+//
+// Work item = (128-row tile, 256-column block).  The K loop streams d in chunks of 32 features: a
+// stage holds the two X-hat image boxes (128 rows x 64 bytes) and the matching boxes of the Theta^T
+// images (256 columns x 64 bytes, pre-swizzled in global memory, one bulk copy each).  With M = 128,
+// N = 256 an MMA runs at the tensor pipe's full rate, and the accumulator (256 TMEM columns) is
 // double-buffered, so the epilogue of one item overlaps the MMAs of the next.
 //
 //   warp 0       producer (TMA / bulk copies, 4-stage ring)
 //   warp 1       MMA issuer: per chunk 2 k-steps x 3 products; commits free the stage
-//   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); thread = row; 16 columns at a
-//                time: tcgen05.ld, old U entries straight from global memory (each thread reads and
-//                writes whole 32-byte sectors of its row), FP64 statistics; column sums by a
-//                shuffle transpose-reduce, combined across the four quarters in fixed order
-//   warps 10-13  split: lo image of the X-hat box (second ring).  The raw box itself is the hi operand:
-//                kind::tf32 ignores the low 13 mantissa bits of an FP32 operand (checked: results are
-//                unchanged when the box is not rewritten), so hi = trunc(x) needs no storage
+//   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); accumulators read in the 16x256b
+//                fragment layout, old U entries straight from global memory (every 4-lane group reads and
+//                writes one 32-byte sector of a row), FP64 statistics; column sums by warp shuffles,
+//                combined across the four quarters in fixed order
 // Every mbarrier wait is bounded (error status GEM_NLR_E_TIMEOUT, kernel runs to its end, TMEM freed).
 #include "nlr_common.cuh"
 #include "device_utils.cuh"
@@ -32,57 +35,77 @@ namespace tcg {
 
 constexpr int TILE_M = 128;
 constexpr int NBLK = 256;                     // columns per item = MMA N
-constexpr int KC = 16;                        // features per chunk (64-byte rows)
-constexpr int A_BOX = TILE_M * KC * 4;        // 8 KB
-constexpr int B_BOX = NBLK * KC * 4;          // 16 KB
-constexpr int STAGE = A_BOX + 2 * B_BOX;      // 40 KB: X-hat raw/hi, Theta^T hi, Theta^T lo
-constexpr int NS = 4, NLO = 3;
+constexpr int KC = 32;                        // features per chunk (64-byte fp16 rows)
+constexpr int A_BOX = TILE_M * KC * 2;        // 8 KB
+constexpr int B_BOX = NBLK * KC * 2;          // 16 KB
+constexpr int STAGE = 2 * A_BOX + 2 * B_BOX;  // 48 KB: X-hat h1, h2, Theta^T h1, h2
+constexpr int NS = 4;
 constexpr int NEPI = 8;                       // epilogue warps
-constexpr int NTHREADS = (2 + NEPI + 4) * 32;
-constexpr size_t SMEM_RING = (size_t)NS * STAGE + (size_t)NLO * A_BOX;
+constexpr int NTHREADS = (2 + NEPI) * 32;
+constexpr size_t SMEM_RING = (size_t)NS * STAGE;
 
-// Shared-memory matrix descriptor, K-major operand with the 64-byte swizzle: 64-byte rows, groups
-// of 8 rows 512 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw64(uint32_t smem_addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
-    d |= (uint64_t)(16u >> 4) << 16;
-    d |= (uint64_t)(512u >> 4) << 32;
-    d |= (uint64_t)1 << 46;          // version
-    d |= (uint64_t)4 << 61;          // SWIZZLE_64B
-    return d;
-}
-
-// Theta (d x r, FP32 row-major) -> hi / lo images of Theta^T as K-major 64-byte-swizzled boxes:
-// box (kb, cb) = features 16 kb .. 16 kb + 15 of columns 256 cb .. 256 cb + 255 (zero beyond r).
-__global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, int NCB, const Ctl* __restrict__ ctl,
-                                 float* __restrict__ img_hi, float* __restrict__ img_lo)
+// Theta (d x r, FP32 row-major) -> fp16 images h1, h2 of Theta^T 2^eT as K-major 64-byte-swizzled boxes:
+// box (kb, cb) = features 32 kb .. 32 kb + 31 of columns 256 cb .. 256 cb + 255 (zero beyond r).
+__global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, int NCB, int eT, const Ctl* __restrict__ ctl,
+                                 __half* __restrict__ img_h1, __half* __restrict__ img_h2)
 {
     if (ctl->stopped) return;
+    const float sT = ldexpf(1.0f, eT);
     const int64_t total = (int64_t)d * NCB * NBLK;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int j = (int)(e / (NCB * NBLK)), k = (int)(e % (NCB * NBLK));     // feature, column
-        const float v = (k < r) ? theta[(size_t)j * r + k] : 0.f;
-        const float hi = tf32_hi(v);
-        const int kb = j >> 4, jj = j & 15, c = jj >> 2, w = jj & 3;
+        const float v = (k < r) ? theta[(size_t)j * r + k] * sT : 0.f;
+        const __half h1 = __float2half_rn(v);
+        const __half h2 = __float2half_rn(v - __half2float(h1));
+        const int kb = j >> 5, jj = j & 31, c = jj >> 3, w = jj & 7;
         const int cb = k >> 8, kr = k & 255;
-        const size_t off = ((size_t)(kb * NCB + cb) * NBLK + kr) * KC + (size_t)(((c ^ ((kr >> 1) & 3)) << 2) + w);
-        img_hi[off] = hi;
-        img_lo[off] = v - hi;
+        const size_t off = ((size_t)(kb * NCB + cb) * NBLK + kr) * KC + (size_t)(((c ^ ((kr >> 1) & 3)) << 3) + w);
+        img_h1[off] = h1;
+        img_h2[off] = h2;
+    }
+}
+
+// X-hat (n x d FP32) -> its fp16 split images x 2^15 = h1 + h2, row-major (n x d) and transposed
+// (d x n_pad, zero beyond n).  One block per 32 x 32 tile; the transposition goes through shared memory.
+__global__ void __launch_bounds__(256)
+k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, __half* __restrict__ h1, __half* __restrict__ h2,
+             __half* __restrict__ h1T, __half* __restrict__ h2T)
+{
+    __shared__ __half t1[32][33], t2[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;            // 32 x 8
+    const int64_t row0 = (int64_t)blockIdx.x * 32;
+    const int f0 = blockIdx.y * 32;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t row = row0 + ty + 8 * i;
+        const int f = f0 + tx;
+        const float v = (row < n && f < d) ? X[row * d + f] * 32768.0f : 0.f;
+        const __half a = __float2half_rn(v);
+        const __half b = __float2half_rn(v - __half2float(a));
+        if (row < n && f < d) { h1[row * d + f] = a; h2[row * d + f] = b; }
+        t1[ty + 8 * i][tx] = a;
+        t2[ty + 8 * i][tx] = b;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int f = f0 + ty + 8 * i;
+        const int64_t row = row0 + tx;
+        if (f < d && row < n_pad) { h1T[(size_t)f * n_pad + row] = t1[tx][ty + 8 * i]; h2T[(size_t)f * n_pad + row] = t2[tx][ty + 8 * i]; }
     }
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ img_hi,
-            const float* __restrict__ img_lo, float* __restrict__ U, const float* __restrict__ ybar,
-            const float* __restrict__ p, const float* __restrict__ alpha_s, Ctl* __restrict__ ctl, int64_t n, int d,
-            int r, int NCB, float alpha, int K, double eps_d, double* __restrict__ part, float* __restrict__ p_out)
+k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
+            const __half* __restrict__ img_h1, const __half* __restrict__ img_h2, float* __restrict__ U,
+            const float* __restrict__ ybar, const float* __restrict__ p, const float* __restrict__ alpha_s,
+            Ctl* __restrict__ ctl, int64_t n, int d, int r, int NCB, int eT, float alpha, int K, double eps_d,
+            double* __restrict__ part, float* __restrict__ p_out)
 {
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[3 * NS + NLO + 4];
+    __shared__ __align__(8) uint64_t bars[2 * NS + 4];
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t tmem_base_s;
     __shared__ double sred[32];
@@ -95,7 +118,6 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
     const int RP = NCB * NBLK;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t stage0 = smem_base;
-    const uint32_t lo0 = stage0 + (uint32_t)NS * STAGE;
     unsigned char* tail = smem + SMEM_RING;
     float* sp = reinterpret_cast<float*>(tail);                         // [RP] p
     float* sas = sp + RP;                                               // [RP] alpha s
@@ -104,15 +126,12 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
 
     const uint32_t bar0 = smem_u32(bars);
     auto xfull = [&](int s) { return bar0 + 8u * s; };
-    auto xsplit = [&](int s) { return bar0 + 8u * (NS + s); };
-    auto xfree = [&](int s) { return bar0 + 8u * (2 * NS + s); };
-    auto lofree = [&](int l) { return bar0 + 8u * (3 * NS + l); };
-    auto accfull = [&](int a) { return bar0 + 8u * (3 * NS + NLO + a); };
-    auto accfree = [&](int a) { return bar0 + 8u * (3 * NS + NLO + 2 + a); };
+    auto xfree = [&](int s) { return bar0 + 8u * (NS + s); };
+    auto accfull = [&](int a) { return bar0 + 8u * (2 * NS + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (2 * NS + 2 + a); };
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(xfull(s), 1); mbar_init(xsplit(s), 4); mbar_init(xfree(s), 1); }
-        for (int l = 0; l < NLO; ++l) mbar_init(lofree(l), 1);
+        for (int s = 0; s < NS; ++s) { mbar_init(xfull(s), 1); mbar_init(xfree(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), NEPI); }
         abort_flag = 0;
         fence_barrier_init();
@@ -131,7 +150,8 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
     const int64_t n_tiles = (n + TILE_M - 1) / TILE_M;
     const int64_t n_items = n_tiles * NCB;
     const float cf = ctl->c_f;
-    const float two_alpha = 2.0f * alpha;
+    // the accumulator holds (x-hat 2^15) (Theta 2^eT) sums: fold the scales into the 2 alpha factor
+    const float two_alpha = 2.0f * alpha * ldexpf(1.0f, -15 - eT);
     double sa = 0.0, sb = 0.0, sh = 0.0;
 
     if (warp == 0) {
@@ -144,13 +164,14 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
                 const int row0 = (int)(t * TILE_M);
                 for (int kb = 0; kb < KB; ++kb, ++g) {
                     const int s = (int)(g % NS);
-                    if (g >= NS) mbar_wait(xfree(s), (uint32_t)((g / NS) - 1) & 1, &abort_flag, ctl);
+                    if (g >= NS) mbar_wait_spin(xfree(s), (uint32_t)((g / NS) - 1) & 1, &abort_flag, ctl);
                     const uint32_t dst = stage0 + (uint32_t)s * STAGE;
                     const size_t boff = ((size_t)(kb * NCB + cb) * NBLK) * KC;
                     mbar_expect_tx(xfull(s), STAGE);
-                    tma_load_2d(dst, &tmX, kb * KC, row0, xfull(s));
-                    bulk_load_1d(dst + A_BOX, img_hi + boff, B_BOX, xfull(s));
-                    bulk_load_1d(dst + A_BOX + B_BOX, img_lo + boff, B_BOX, xfull(s));
+                    tma_load_2d(dst, &tmX1, kb * KC, row0, xfull(s));
+                    tma_load_2d(dst + A_BOX, &tmX2, kb * KC, row0, xfull(s));
+                    bulk_load_1d(dst + 2 * A_BOX, img_h1 + boff, B_BOX, xfull(s));
+                    bulk_load_1d(dst + 2 * A_BOX + B_BOX, img_h2 + boff, B_BOX, xfull(s));
                 }
             }
         }
@@ -159,55 +180,29 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
         // Inside an item the wait for the next chunk is placed between the two k-steps of the current chunk,
         // so the tensor pipe has work queued while this thread polls.
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_tf32(TILE_M, NBLK, 0, 0);
+            const uint32_t idesc = umma_idesc_f16(TILE_M, NBLK, 0, 0);
             int64_t g = 0;
             int i = 0;
             for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x, ++i) {
                 const int a = i & 1;
                 // item boundary: the previous accumulator is already handed over; wait for a free one and for
                 // the first chunk
-                if (i >= 2) mbar_wait(accfree(a), (uint32_t)((i >> 1) - 1) & 1, &abort_flag, ctl);
-                mbar_wait(xsplit((int)(g % NS)), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
+                if (i >= 2) mbar_wait_spin(accfree(a), (uint32_t)((i >> 1) - 1) & 1, &abort_flag, ctl);
+                mbar_wait_spin(xfull((int)(g % NS)), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
                 const uint32_t tacc = tmem_base + (uint32_t)(a * NBLK);
                 for (int kb = 0; kb < KB; ++kb, ++g) {
-                    const int s = (int)(g % NS), l = (int)(g % NLO);
+                    const int s = (int)(g % NS);
                     tc_fence_after();
                     const uint32_t st = stage0 + (uint32_t)s * STAGE;
-                    const uint64_t da_hi = umma_desc_sw64(st), da_lo = umma_desc_sw64(lo0 + (uint32_t)l * A_BOX);
-                    const uint64_t db_hi = umma_desc_sw64(st + A_BOX), db_lo = umma_desc_sw64(st + A_BOX + B_BOX);
-                    // a k-step (8 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
-                    umma_tf32_x3(tacc, da_hi, da_lo, db_hi, db_lo, idesc, kb ? 1u : 0u);
-                    if (kb + 1 < KB) mbar_wait(xsplit((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
-                    umma_tf32_x3(tacc, da_hi + 2, da_lo + 2, db_hi + 2, db_lo + 2, idesc, 1u);
+                    const uint64_t da1 = umma_desc_k_sw64(st), da2 = umma_desc_k_sw64(st + A_BOX);
+                    const uint64_t db1 = umma_desc_k_sw64(st + 2 * A_BOX), db2 = umma_desc_k_sw64(st + 2 * A_BOX + B_BOX);
+                    // a k-step (16 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
+                    umma_f16_x3(tacc, da1, da2, db1, db2, idesc, kb ? 1u : 0u);
+                    if (kb + 1 < KB) mbar_wait_spin(xfull((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
+                    umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
                     umma_commit(xfree(s));
-                    umma_commit(lofree(l));
                 }
                 umma_commit(accfull(a));
-            }
-        }
-    } else if (warp >= 2 + NEPI) {
-        // ------------------------------ split: lo image of the X-hat box ------------------------------
-        const int st = threadIdx.x - (2 + NEPI) * 32;   // 0..127
-        int64_t g = 0;
-        for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x) {
-            for (int kb = 0; kb < KB; ++kb, ++g) {
-                const int s = (int)(g % NS), l = (int)(g % NLO);
-                mbar_wait(xfull(s), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
-                if (g >= NLO) mbar_wait(lofree(l), (uint32_t)((g / NLO) - 1) & 1, &abort_flag, ctl);
-                const uint32_t hi_a = stage0 + (uint32_t)s * STAGE, lo_a = lo0 + (uint32_t)l * A_BOX;
-                float4 xin[A_BOX / 16 / 128];
-#pragma unroll
-                for (int k = 0; k < A_BOX / 16 / 128; ++k) xin[k] = lds128(hi_a + (uint32_t)(k * 128 + st) * 16);
-#pragma unroll
-                for (int k = 0; k < A_BOX / 16 / 128; ++k) {
-                    const uint32_t off = (uint32_t)(k * 128 + st) * 16;
-                    const float4 x = xin[k];
-                    const float4 hi = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
-                    sts128(lo_a + off, make_float4(x.x - hi.x, x.y - hi.y, x.z - hi.z, x.w - hi.w));
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(xsplit(s));
             }
         }
     } else {
@@ -236,7 +231,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ i
                 urow[x] = U + (valid[x] ? row : 0) * (int64_t)r;
             }
             float* my_tmp = stmp + (size_t)(a * 4 + q) * NBLK + half * 128;
-            mbar_wait(accfull(a), (uint32_t)(i >> 1) & 1, &abort_flag, ctl);
+            mbar_wait_relaxed(accfull(a), (uint32_t)(i >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
 #pragma unroll 1
             for (int jj = 0; jj < 8; ++jj) {
@@ -520,21 +515,36 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
 bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
 {
     const int d = pb.P.d, r = pb.P.r;
-    if (d % tcg::KC != 0 || r % 4 != 0 || r < 16 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
+    if (!pb.has_ximg() || d % tcg::KC != 0 || r % 4 != 0 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
     const int NCB = (r + tcg::NBLK - 1) / tcg::NBLK;
     const int RP = NCB * tcg::NBLK;
     if (RP > 2048) return false;
     pl->NCB = NCB;
+    {
+        int e;
+        frexpf(sqrtf((float)pb.P.K), &e);                  // |Theta_jk| <= ||X-hat||_2 ||U||_F = sqrt(K) <= 2^e
+        pl->eT = 14 - e;
+    }
     pl->smem2 = tcg::SMEM_RING + (size_t)RP * (4 + 4 + 8) + (size_t)2 * 4 * tcg::NBLK * 4 + 1024;
     if (pl->smem2 > 227 * 1024 - 1024) return false;
-    pl->img_hi = img_storage;
-    pl->img_lo = img_storage + (size_t)d * RP;
-    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tcg::TILE_M, tcg::KC, false, 64)) return false;
+    pl->img_h1 = img_storage;
+    pl->img_h2 = reinterpret_cast<uint16_t*>(img_storage) + (size_t)d * RP;
+    if (!make_tensor_map_2d_f16(&pl->tmX1, pb.ximg(0), pb.P.n, d, d, tcg::TILE_M, tcg::KC)) return false;
+    if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, d, tcg::TILE_M, tcg::KC)) return false;
     const int64_t items = (pb.P.n + tcg::TILE_M - 1) / tcg::TILE_M * NCB;
     pl->g2 = (int)(items < kSMs ? items : kSMs);
     if (cudaFuncSetAttribute(tcg::k_pass2_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
         return false;
     return true;
+}
+
+void tcg_prepare(const Problem& pb)
+{
+    const dim3 grid((unsigned)((pb.L.n_pad + 31) / 32), (unsigned)((pb.P.d + 31) / 32));
+    tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.P.d, pb.L.n_pad,
+                                                   reinterpret_cast<__half*>(pb.ximg(0)), reinterpret_cast<__half*>(pb.ximg(1)),
+                                                   reinterpret_cast<__half*>(pb.ximgT(0)), reinterpret_cast<__half*>(pb.ximgT(1)));
+    pb.count(1);
 }
 
 bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
@@ -567,9 +577,11 @@ void tcg_launch_first(const Problem& pb, const Tcg1Plan& pl)
 void tcg_launch_second(const Problem& pb, const TcgPlan& pl)
 {
     const int d = pb.P.d, r = pb.P.r;
-    tcg::k_theta_images64<<<kSMs * 4, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NCB, pb.ctl(), pl.img_hi, pl.img_lo);
+    __half* i1 = reinterpret_cast<__half*>(pl.img_h1);
+    __half* i2 = reinterpret_cast<__half*>(pl.img_h2);
+    tcg::k_theta_images64<<<kSMs * 4, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NCB, pl.eT, pb.ctl(), i1, i2);
     tcg::k_pass2_tcg<<<pl.g2, tcg::NTHREADS, pl.smem2, pb.stream>>>(
-        pl.tmX, pl.img_hi, pl.img_lo, pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NCB,
+        pl.tmX1, pl.tmX2, i1, i2, pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NCB, pl.eT,
         pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
     pb.count(2);
 }

@@ -29,6 +29,8 @@ struct Ctl {
 
 struct Layout {
     size_t ctl, p, s, alpha_s, theta, thimg, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
+    size_t ximg, ximgT;      // fp16 split images of X-hat (row-major and transposed), wide tensor-core shapes only (else 0 bytes)
+    int64_t n_pad;           // row count of the transposed images' rows, n rounded up to 64
     int g1x, g1y_d, g1y_r;   // generic pass-1 grid: row chunks, d tiles, r tiles
     int gv;                  // vector kernel CTAs
     int g2x, g2y;            // generic pass-2 grid: row-tile CTAs, column tiles
@@ -58,6 +60,10 @@ struct Problem {
     float* s() const { return reinterpret_cast<float*>(ws + L.s); }
     float* alpha_s() const { return reinterpret_cast<float*>(ws + L.alpha_s); }
     float* theta() const { return reinterpret_cast<float*>(ws + L.theta); }
+    // fp16 split images of X-hat (wide tensor-core shapes): h1 then h2, row-major n x d; transposed d x n_pad
+    uint16_t* ximg(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximg) + (size_t)which * P.n * P.d; }
+    uint16_t* ximgT(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximgT) + (size_t)which * P.d * L.n_pad; }
+    bool has_ximg() const { return L.ximgT > L.ximg; }
     float* ytilde() const { return reinterpret_cast<float*>(ws + L.ytilde); }
     float* ybar() const { return reinterpret_cast<float*>(ws + L.ybar); }
     double* part1() const { return reinterpret_cast<double*>(ws + L.part1); }

@@ -160,5 +160,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, float4 v)
 // Returns false if the driver entry point is missing or the encode fails.
 bool make_tensor_map_2d(CUtensorMap* out, const float* base, int64_t rows, int cols, int box_rows, int box_cols,
                         bool atom32 = false, int swizzle_bytes = 0);
+bool make_tensor_map_2d_f16(CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int64_t pitch_halves,
+                            int box_rows, int box_cols);
 
 }  // namespace gemnlr

@@ -47,14 +47,18 @@ namespace gemnlr {
 // Tiled second product for wide problems (kernels_tcg.cu): d a multiple of 16, r a multiple of 4 up to
 // 2048; Theta^T images of 2 * d * (r rounded up to 256) floats.
 struct TcgPlan {
-    alignas(64) CUtensorMap tmX;   // X-hat boxes: 128 rows x 16 features, 64-byte swizzle
+    alignas(64) CUtensorMap tmX1;  // X-hat image h1 (n x d fp16): boxes of 128 rows x 32 features, 64-byte swizzle
+    alignas(64) CUtensorMap tmX2;  // X-hat image h2
     int NCB;                       // 256-column blocks
+    int eT;                        // Theta is scaled by 2^eT before its fp16 split
     int g2;
     size_t smem2;
-    float* img_hi;
-    float* img_lo;
+    void* img_h1;                  // Theta^T images (fp16), rebuilt every iteration
+    void* img_h2;
 };
 bool tcg_plan(const Problem& pb, TcgPlan* plan, float* img_storage);
+// Builds the static fp16 images of X-hat (row-major and transposed); call whenever X-hat has become valid.
+void tcg_prepare(const Problem& pb);
 
 // Matching first product (Theta^T tiles of 128 columns x 256 features, split over row ranges): d a
 // multiple of 32, (r / 128) * (d / 256) tiles at most one per SM.  The vector pass runs separately.

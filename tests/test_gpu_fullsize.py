@@ -122,7 +122,7 @@ def test_embedding_shape_full_size_every_entry():
     Ud = torch.from_numpy(U0).cuda()
     s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"],
                    T=spec.iters, T_min=spec.iters)
-    assert s.path() == "tf32x3.tiled", s.path()
+    assert s.path() == "f16x3.tiled", s.path()
     s.spectral_norm()
     Xhat = Xd.cpu().numpy()                      # both sides work on the library's X-hat
     rc, info = s.step()
