@@ -69,7 +69,7 @@ Layout make_layout(const gem_nlr_params& P)
     L.n_pad = (n + 63) / 64 * 64;
     const bool wide_tc = (P.precision == -1 || P.precision == 1) && r > 256 && d % 32 == 0 && n >= 4096;
     L.ximg = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)n * d : 0);
-    L.ximgT = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)d * L.n_pad : 0);
+    L.ximgT = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)(L.n_pad / 32) * ((d + 255) / 256) * 256 * 32 : 0);
     L.total = off;
     return L;
 }

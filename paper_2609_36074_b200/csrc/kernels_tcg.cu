@@ -65,8 +65,11 @@ __global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, 
     }
 }
 
-// X-hat (n x d FP32) -> its fp16 split images x 2^15 = h1 + h2, row-major (n x d) and transposed
-// (d x n_pad, zero beyond n).  One block per 32 x 32 tile; the transposition goes through shared memory.
+// X-hat (n x d FP32) -> its fp16 split images x 2^15 = h1 + h2: row-major (n x d), and transposed in the
+// exact shared-memory form the first product consumes: for every stage of 32 data rows and block of 256
+// features one contiguous 16 KB box [feature][32 rows] with the 64-byte swizzle already applied (zero
+// beyond n and d), so that a box arrives with one bulk copy.  One block per 32 x 32 tile; the
+// transposition goes through shared memory.
 __global__ void __launch_bounds__(256)
 k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, __half* __restrict__ h1, __half* __restrict__ h2,
              __half* __restrict__ h1T, __half* __restrict__ h2T)
@@ -91,7 +94,11 @@ k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, __hal
     for (int i = 0; i < 4; ++i) {
         const int f = f0 + ty + 8 * i;
         const int64_t row = row0 + tx;
-        if (f < d && row < n_pad) { h1T[(size_t)f * n_pad + row] = t1[tx][ty + 8 * i]; h2T[(size_t)f * n_pad + row] = t2[tx][ty + 8 * i]; }
+        if (row < n_pad) {                                 // features d .. 256 NNB - 1 of the last block stay zero (memset)
+            const int nnb = (d + 255) / 256, nbk = f >> 8, m = f & 255, kk = tx;       // kk = row inside the stage
+            const size_t off = (((size_t)blockIdx.x * nnb + nbk) * 256 + m) * 32 + (size_t)((((kk >> 3) ^ ((m >> 1) & 3)) << 3) + (kk & 7));
+            if (f < d) { h1T[off] = t1[tx][ty + 8 * i]; h2T[off] = t2[tx][ty + 8 * i]; }
+        }
     }
 }
 
@@ -346,58 +353,61 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
 
 
 // ================================================================================================
-// First product for the same wide problems:  Theta = c_f X-hat^T W  as Theta^T tiles.
+// First product for the same wide problems:  Theta = X-hat^T U  as Theta^T tiles, u = c_f w.
 //
 // Work item (one CTA each, all resident at once) = (128 columns of U, up to 256 features, one of
-// NSPLIT contiguous row ranges).  The contraction runs over the data rows, so both operands are
-// MN-major: TMA boxes of 16 rows x 32 columns with the 128-byte swizzle of 32-byte atoms (A = 4 boxes
-// of U, B = up to 8 boxes of X-hat per stage).  Two teams of four warps take alternate stages and
-// write the lo images (x - trunc(x)) into a second ring; the raw boxes serve as the hi operands (the
-// tensor core ignores the low 13 mantissa bits) and the pending multiplier c_f is applied to the
-// reduced Theta instead of to every entry of U;
-// the MMA issuer runs 2 k-steps x 3 products per stage into one of two TMEM accumulators, which is
-// handed to the epilogue every FLUSH stages and folded into the FP64 partial of this row range
-// (layout [feature][column] like the generic first product, so the same reduction kernel follows).
-// The row-local vector work cannot be fused here (a CTA sees 128 of the r columns): it runs as the
-// separate vector pass before this kernel.
+// NSPLIT contiguous row ranges).  The contraction runs over the data rows, the slow (MN-major)
+// operand orientation of the tensor core, so both operands are presented K-major instead: the X-hat
+// side comes from the transposed fp16 images built at setup (one contiguous, pre-swizzled 16 KB box per
+// stage and 256-feature block, bulk-copied straight into the image stage); the U side is transposed on the fly: TMA brings
+// the 32 x 128 FP32 slice of the stage, a team of four warps (thread = column) scales by c_f and a power
+// of two, splits u 2^k = h1 + h2 in fp16 and writes one 16-byte chunk per (column, 8 rows).  The MMA
+// issuer runs 2 k-steps (K = 16) x 3 products per stage with M = 128, N = 256 into one of two TMEM
+// accumulators, which is handed to the epilogue every FLUSH1 stages and folded, rescaled, into the FP64
+// partial of this row range (layout [feature][column] like the generic first product, so the same
+// reduction kernel follows).  The row-local vector work cannot be fused here (a CTA sees 128 of the r
+// columns): it runs as the separate vector pass before this kernel.
 // ================================================================================================
-constexpr int TR1 = 16;                        // rows per stage (2 k-steps)
-constexpr int CH1 = TR1 * 128;                 // one box: 16 rows x 32 floats = 2 KB
-constexpr int NS1 = 5, NLO1 = 3;               // a raw slot lives from the TMA issue to the last MMA, a lo slot from the split on
-constexpr int FLUSH1 = 256;                    // stages per accumulation period (4096 rows)
-constexpr int NTH1 = 14 * 32;                  // producer, MMA, 4 epilogue, 8 split warps
+constexpr int TR1 = 32;                        // data rows per stage (2 k-steps of 16)
+constexpr int NT1 = 2;                         // teams of four warps on alternate stages
+constexpr int NIM1 = 3, NRAW1 = 3;             // image stages, raw U stages
+constexpr int URAW1 = TR1 * 128 * 4;           // raw U slice: 32 rows x 128 columns FP32 = 16 KB
+constexpr int UIMG1 = 128 * 64;                // fp16 image of the U operand: 128 columns x 32 data rows
+constexpr int XIMG1 = 256 * 64;                // fp16 image of the X-hat operand: 256 features x 32 data rows
+constexpr int IMG1 = 2 * UIMG1 + 2 * XIMG1;    // U h1, U h2, X h1, X h2: 48 KB
+constexpr int FLUSH1 = 128;                    // stages per accumulation period (4096 rows)
+constexpr int NTH1 = (2 + 4 + 4 * NT1) * 32;   // producer, MMA issuer, 4 epilogue, 4 NT1 team warps
 
 __global__ void __launch_bounds__(NTH1, 1)
-k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU, Ctl* __restrict__ ctl,
-            int64_t n, int d, int r, int NMT, int NNB, int NSPLIT, double* __restrict__ part)
+k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ xT1,
+            const __half* __restrict__ xT2, Ctl* __restrict__ ctl, int64_t n, int d, int r, int K,
+            int NMT, int NNB, int NSPLIT, double* __restrict__ part)
 {
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[3 * NS1 + NLO1 + 4];
+    __shared__ __align__(8) uint64_t bars[2 * NIM1 + 2 * NRAW1 + 4];
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t tmem_base_s;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // item of this CTA
     const int mt = blockIdx.x % NMT, nb = (blockIdx.x / NMT) % NNB, sp = blockIdx.x / (NMT * NNB);
+    const int c0 = mt * 128;                               // first column of U of this item
     const int f0 = nb * 256;
     const int Nb = (d - f0 < 256) ? d - f0 : 256;          // features of this item (multiple of 32)
-    const int NBX = Nb / 32;
-    const int STAGE1 = (4 + 8) * CH1;                       // U boxes then up to 8 X-hat boxes
 
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t raw0 = smem_base, lo0 = raw0 + (uint32_t)NS1 * STAGE1;
+    const uint32_t img0 = smem_u32(smem);
+    const uint32_t raw0 = img0 + (uint32_t)NIM1 * IMG1;
     const uint32_t bar0 = smem_u32(bars);
-    auto full = [&](int s) { return bar0 + 8u * s; };
-    auto split = [&](int s) { return bar0 + 8u * (NS1 + s); };
-    auto rawfree = [&](int s) { return bar0 + 8u * (2 * NS1 + s); };
-    auto lofree = [&](int l) { return bar0 + 8u * (3 * NS1 + l); };
-    auto accfull = [&](int a) { return bar0 + 8u * (3 * NS1 + NLO1 + a); };
-    auto accfree = [&](int a) { return bar0 + 8u * (3 * NS1 + NLO1 + 2 + a); };
+    auto imgfull = [&](int l) { return bar0 + 8u * l; };
+    auto imgfree = [&](int l) { return bar0 + 8u * (NIM1 + l); };
+    auto ufull = [&](int s) { return bar0 + 8u * (2 * NIM1 + s); };
+    auto ufree = [&](int s) { return bar0 + 8u * (2 * NIM1 + NRAW1 + s); };
+    auto accfull = [&](int a) { return bar0 + 8u * (2 * NIM1 + 2 * NRAW1 + a); };
+    auto accfree = [&](int a) { return bar0 + 8u * (2 * NIM1 + 2 * NRAW1 + 2 + a); };
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS1; ++s) { mbar_init(full(s), 1); mbar_init(split(s), 4); mbar_init(rawfree(s), 1); }
-        for (int l = 0; l < NLO1; ++l) mbar_init(lofree(l), 1);
+        for (int l = 0; l < NIM1; ++l) { mbar_init(imgfull(l), 4 + 1); mbar_init(imgfree(l), 1); }   // team warps + X-hat boxes
+        for (int s = 0; s < NRAW1; ++s) { mbar_init(ufull(s), 1); mbar_init(ufree(s), 4); }
         for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4); }
         abort_flag = 0;
         fence_barrier_init();
@@ -414,79 +424,103 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
     const int64_t g_lo = (int64_t)sp * base_cnt + (sp < rem_cnt ? sp : rem_cnt);
     const int my_stages = (int)(base_cnt + (sp < rem_cnt ? 1 : 0));
     const int n_periods = (my_stages + FLUSH1 - 1) / FLUSH1;
+    const float cf = ctl->c_f;
+    // power-of-two operand scales: x-hat 2^15 (in the images), u 2^eU with |u| 2^eU <= 2^14
+    int eU;
+    {
+        int e;
+        frexpf(sqrtf((float)K), &e);                       // |u_ij| <= ||U||_F = sqrt(K) <= 2^e
+        eU = 14 - e;
+    }
+    const float sU = ldexpf(1.0f, eU);
+    const double unscale = ldexp(1.0, -15 - eU);
 
     if (warp == 0) {
+        // ------------------------------ producer ------------------------------
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
-                const int s = g % NS1;
-                if (g >= NS1) mbar_wait(rawfree(s), ((g / NS1) - 1) & 1, &abort_flag, ctl);
+                const int s = g % NRAW1, l = g % NIM1;
                 const int row0 = (int)((g_lo + g) * TR1);
-                const uint32_t dst = raw0 + (uint32_t)s * STAGE1;
-                mbar_expect_tx(full(s), (uint32_t)(4 + NBX) * CH1);
-                for (int c = 0; c < 4; ++c) tma_load_2d(dst + c * CH1, &tmU, mt * 128 + c * 32, row0, full(s));
-                for (int b = 0; b < NBX; ++b) tma_load_2d(dst + (4 + b) * CH1, &tmX, f0 + b * 32, row0, full(s));
+                if (g >= NRAW1) mbar_wait_spin(ufree(s), ((g / NRAW1) - 1) & 1, &abort_flag, ctl);
+                mbar_expect_tx(ufull(s), URAW1);
+                tma_load_2d(raw0 + (uint32_t)s * URAW1, &tmU, c0, row0, ufull(s));
+                if (g >= NIM1) mbar_wait_spin(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
+                const uint32_t im = img0 + (uint32_t)l * IMG1;
+                const size_t xoff = ((size_t)(g_lo + g) * NNB + nb) * (256 * 32);      // this stage's box of the feature block
+                mbar_expect_tx(imgfull(l), 2 * XIMG1);
+                bulk_load_1d(im + 2 * UIMG1, xT1 + xoff, XIMG1, imgfull(l));
+                bulk_load_1d(im + 2 * UIMG1 + XIMG1, xT2 + xoff, XIMG1, imgfull(l));
             }
         }
     } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_tf32(128, Nb, 1, 1);
-            // the wait for the next stage sits between the two k-steps of the current one
-            if (my_stages > 0) mbar_wait(split(0), 0, &abort_flag, ctl);
-            for (int g = 0; g < my_stages && !abort_flag; ++g) {
-                const int s = g % NS1, l = g % NLO1;
-                const int period = g / FLUSH1, a = period & 1, in_period = g % FLUSH1;
-                if (in_period == 0 && period >= 2) mbar_wait(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
+            const uint32_t idesc = umma_idesc_f16(128, Nb, 0, 0);
+            if (my_stages > 0) mbar_wait_spin(imgfull(0), 0, &abort_flag, ctl);
+            int l = 0, lph = 0, a = 0, in_period = 0, period = 0;
+            for (int g = 0; g < my_stages; ++g) {
+                if (in_period == 0 && period >= 2) mbar_wait_spin(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * 256);
-                const uint32_t hi_s = raw0 + (uint32_t)s * STAGE1, lo_s = lo0 + (uint32_t)l * STAGE1;
-                // chunks are CH1 bytes apart (LBO); 4-row swizzle periods of 512 bytes along K (SBO); a k-step is 1 KB
-                const uint64_t da_hi = umma_desc_sw128_atom32(hi_s, CH1, 512), da_lo = umma_desc_sw128_atom32(lo_s, CH1, 512);
-                const uint64_t db_hi = umma_desc_sw128_atom32(hi_s + 4 * CH1, CH1, 512);
-                const uint64_t db_lo = umma_desc_sw128_atom32(lo_s + 4 * CH1, CH1, 512);
-                umma_tf32_x3(tacc, da_hi, da_lo, db_hi, db_lo, idesc, in_period ? 1u : 0u);
-                if (g + 1 < my_stages) mbar_wait(split((g + 1) % NS1), ((g + 1) / NS1) & 1, &abort_flag, ctl);
-                umma_tf32_x3(tacc, da_hi + 64, da_lo + 64, db_hi + 64, db_lo + 64, idesc, 1u);
-                umma_commit(rawfree(s));
-                umma_commit(lofree(l));
+                const uint32_t im = img0 + (uint32_t)l * IMG1;
+                // K-major images; a k-step of 16 data rows (32 bytes inside the 64-byte swizzled row) advances
+                // the start address by 2
+                const uint64_t da1 = umma_desc_k_sw64(im), da2 = umma_desc_k_sw64(im + UIMG1);
+                const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG1), db2 = umma_desc_k_sw64(im + 2 * UIMG1 + XIMG1);
+                umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
+                int ln = l + 1, lphn = lph;
+                if (ln == NIM1) { ln = 0; lphn ^= 1; }
+                if (g + 1 < my_stages) mbar_wait_spin(imgfull(ln), (uint32_t)lphn, &abort_flag, ctl);
+                umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
+                umma_commit(imgfree(l));
                 if (in_period == FLUSH1 - 1 || g == my_stages - 1) umma_commit(accfull(a));
+                l = ln; lph = lphn;
+                if (++in_period == FLUSH1) { in_period = 0; ++period; a ^= 1; }
+                if (abort_flag) break;
             }
         }
     } else if (warp >= 6) {
-        // ------------------------------ split (two teams on alternate stages) ------------------------------
-        const int vw = warp - 6, team = vw >> 2;
-        const int tt = (vw & 3) * 32 + lane;               // 0..127 inside the team
-        const int nq = (4 + NBX) * (CH1 / 16) / 128;       // float4 per thread and stage (U boxes first)
-        for (int g = team; g < my_stages; g += 2) {
-            const int s = g % NS1, l = g % NLO1;
-            mbar_wait(full(s), (g / NS1) & 1, &abort_flag, ctl);
-            if (g >= NLO1) mbar_wait(lofree(l), ((g / NLO1) - 1) & 1, &abort_flag, ctl);
-            const uint32_t hi_s = raw0 + (uint32_t)s * STAGE1, lo_s = lo0 + (uint32_t)l * STAGE1;
-            // lo = x - trunc(x) of every piece (12 per thread at most, all requested up front); the raw boxes
-            // are the hi operands as they are
-            float4 xin[12];
+        // ------------------------------ U teams: FP32 slice -> K-major fp16 images ------------------------------
+        const int vw = warp - 6, team = vw >> 2, tw = vw & 3;
+        const int tt = tw * 32 + lane;                     // column of the slice
+        for (int g = team; g < my_stages; g += NT1) {
+            const int s = g % NRAW1, l = g % NIM1;
+            mbar_wait_spin(ufull(s), (g / NRAW1) & 1, &abort_flag, ctl);
+            const uint32_t rs = raw0 + (uint32_t)s * URAW1;
+            float uv[4][8];
 #pragma unroll
-            for (int k = 0; k < 12; ++k)
-                if (k < nq) xin[k] = lds128(hi_s + (uint32_t)(k * 128 + tt) * 16);
+            for (int kg = 0; kg < 4; ++kg)
 #pragma unroll
-            for (int k = 0; k < 12; ++k)
-                if (k < nq) {
-                    const float4 x = xin[k];
-                    sts128(lo_s + (uint32_t)(k * 128 + tt) * 16,
-                           make_float4(x.x - tf32_hi(x.x), x.y - tf32_hi(x.y), x.z - tf32_hi(x.z), x.w - tf32_hi(x.w)));
-                }
+                for (int k = 0; k < 8; ++k) uv[kg][k] = lds32f(rs + (uint32_t)(((8 * kg + k) * 128 + tt) * 4));
+            if (g >= NIM1) mbar_wait_spin(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
+            const uint32_t im = img0 + (uint32_t)l * IMG1;
+#pragma unroll
+            for (int kg = 0; kg < 4; ++kg) {
+                float v[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[k] = (cf * uv[kg][k]) * sU;      // u = c_f w rounded to FP32, then scaled
+                uint4 h1, h2;
+                split_h8(v, h1, h2);
+                const uint32_t io = kimg_off(tt, kg);
+                sts128u(im + io, h1);
+                sts128u(im + UIMG1 + io, h2);
+            }
             fence_proxy_async();
             __syncwarp();
-            if (lane == 0) mbar_arrive(split(s));
+            if (lane == 0) {
+                mbar_arrive(imgfull(l));
+                mbar_arrive(ufree(s));
+            }
         }
     } else {
-        // ------------------------------ epilogue: FP64 fold of the accumulator ------------------------------
+        // ------------------------------ epilogue: FP64 fold of the accumulator (warps 2-5) ------------------------------
         // thread = column j of U (TMEM lane); entry (feature f, column j) of this row range's partial
         const int q4 = warp & 3;
-        const int j = mt * 128 + q4 * 32 + lane;
+        const int j = c0 + q4 * 32 + lane;
         double* const out = part + (size_t)sp * ((size_t)d * r);
         for (int period = 0; period < n_periods; ++period) {
             const int a = period & 1;
-            mbar_wait(accfull(a), (period >> 1) & 1, &abort_flag, ctl);
+            mbar_wait_relaxed(accfull(a), (period >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
             for (int c = 0; c * 16 < Nb; ++c) {
                 float v[16];
@@ -497,7 +531,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUt
 #pragma unroll
                     for (int k = 0; k < 16; ++k) prev[k] = (period == 0) ? 0.0 : __ldcg(o + (size_t)k * r);
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) o[(size_t)k * r] = prev[k] + (double)v[k];
+                    for (int k = 0; k < 16; ++k) o[(size_t)k * r] = prev[k] + unscale * (double)v[k];
                 }
             }
             tc_fence_before();
@@ -540,6 +574,7 @@ bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
 
 void tcg_prepare(const Problem& pb)
 {
+    cudaMemsetAsync(pb.ximgT(0), 0, sizeof(uint16_t) * 2 * pb.ximgT_halves(), pb.stream);
     const dim3 grid((unsigned)((pb.L.n_pad + 31) / 32), (unsigned)((pb.P.d + 31) / 32));
     tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.P.d, pb.L.n_pad,
                                                    reinterpret_cast<__half*>(pb.ximg(0)), reinterpret_cast<__half*>(pb.ximg(1)),
@@ -550,7 +585,7 @@ void tcg_prepare(const Problem& pb)
 bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
 {
     const int d = pb.P.d, r = pb.P.r;
-    if (d % 32 != 0 || r % 4 != 0 || r < 16 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
+    if (!pb.has_ximg() || d % 32 != 0 || r % 4 != 0 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
     pl->NMT = (r + 127) / 128;
     pl->NNB = (d + 255) / 256;
     const int tiles = pl->NMT * pl->NNB;
@@ -558,9 +593,8 @@ bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
     pl->NSPLIT = kSMs / tiles;
     if (pl->NSPLIT > 8) pl->NSPLIT = 8;                     // partial records are sized for 8 row ranges
     pl->grid = tiles * pl->NSPLIT;
-    pl->smem = (size_t)(tcg::NS1 + tcg::NLO1) * 12 * tcg::CH1 + 1024;
-    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tcg::TR1, 32, true)) return false;
-    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tcg::TR1, 32, true)) return false;
+    pl->smem = (size_t)tcg::NIM1 * tcg::IMG1 + (size_t)tcg::NRAW1 * tcg::URAW1 + 1024;
+    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tcg::TR1, 128, false, 1)) return false;     // plain FP32 rows
     if (cudaFuncSetAttribute(tcg::k_pass1_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess)
         return false;
     return true;
@@ -568,10 +602,11 @@ bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
 
 void tcg_launch_first(const Problem& pb, const Tcg1Plan& pl)
 {
-    tcg::k_pass1_tcg<<<pl.grid, tcg::NTH1, pl.smem, pb.stream>>>(pl.tmX, pl.tmU, pb.ctl(), pb.P.n, pb.P.d, pb.P.r,
-                                                                 pl.NMT, pl.NNB, pl.NSPLIT, pb.part1());
+    tcg::k_pass1_tcg<<<pl.grid, tcg::NTH1, pl.smem, pb.stream>>>(pl.tmU, reinterpret_cast<const __half*>(pb.ximgT(0)),
+                                                                 reinterpret_cast<const __half*>(pb.ximgT(1)), pb.ctl(), pb.P.n, pb.P.d, pb.P.r,
+                                                                 pb.P.K, pl.NMT, pl.NNB, pl.NSPLIT, pb.part1());
     pb.count(1);
-    launch_red1(pb, pl.NSPLIT, 0, 1);
+    launch_red1(pb, pl.NSPLIT, 0, 0);
 }
 
 void tcg_launch_second(const Problem& pb, const TcgPlan& pl)

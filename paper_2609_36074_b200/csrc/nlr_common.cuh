@@ -62,7 +62,9 @@ struct Problem {
     float* theta() const { return reinterpret_cast<float*>(ws + L.theta); }
     // fp16 split images of X-hat (wide tensor-core shapes): h1 then h2, row-major n x d; transposed d x n_pad
     uint16_t* ximg(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximg) + (size_t)which * P.n * P.d; }
-    uint16_t* ximgT(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximgT) + (size_t)which * P.d * L.n_pad; }
+    // transposed images: [n_pad / 32 stages][ceil(d / 256) blocks][256 features][32 rows] halves each
+    size_t ximgT_halves() const { return (size_t)(L.n_pad / 32) * ((P.d + 255) / 256) * 256 * 32; }
+    uint16_t* ximgT(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximgT) + (size_t)which * ximgT_halves(); }
     bool has_ximg() const { return L.ximgT > L.ximg; }
     float* ytilde() const { return reinterpret_cast<float*>(ws + L.ytilde); }
     float* ybar() const { return reinterpret_cast<float*>(ws + L.ybar); }

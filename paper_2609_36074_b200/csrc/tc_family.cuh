@@ -63,8 +63,7 @@ void tcg_prepare(const Problem& pb);
 // Matching first product (Theta^T tiles of 128 columns x 256 features, split over row ranges): d a
 // multiple of 32, (r / 128) * (d / 256) tiles at most one per SM.  The vector pass runs separately.
 struct Tcg1Plan {
-    alignas(64) CUtensorMap tmX;   // X-hat boxes: 16 rows x 32 features, 128-byte swizzle with 32-byte atoms
-    alignas(64) CUtensorMap tmU;   // U boxes: 16 rows x 32 columns, same layout
+    alignas(64) CUtensorMap tmU;   // U slices: 32 rows x 128 columns FP32, plain rows
     int NMT, NNB, NSPLIT, grid;
     size_t smem;
 };
