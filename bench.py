@@ -46,7 +46,8 @@ def _peaks():
 # Keyed by (n, d, r, kernel path); anything else reports null.
 NCU_TRAFFIC_BYTES = {
     (1_000_000, 128, 16, "mma.tf32x3"): 640.0e6,
-    (10_000_000, 64, 100, "tf32x3"): 10.385e9,
+    (10_000_000, 64, 100, "f16x3+tf32x3"): 10.36e9,
+    (2_000_000, 768, 1000, "f16x3.tiled"): 22.96e9,
     (100_000_000, 32, 8, "ffma"): 19.49e9,
 }
 

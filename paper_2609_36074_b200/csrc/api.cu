@@ -277,7 +277,7 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
             h->path = h->use_ffma ? "ffma+tf32x3" : "generic+tf32x3";
             if (tc1_plan(h->pb, &h->tc1)) {
                 h->use_tc1 = true;
-                h->path = "tf32x3";
+                h->path = "f16x3+tf32x3";      // first product on the fp16 split, second on the TF32 split
             }
         }
         else if (tcg_plan(h->pb, &h->tcg, img)) {
