@@ -71,10 +71,13 @@ typedef struct {
     int32_t  pi_max_iters;  /* power-iteration cap for ||X_c||_2 (<=0: 100)                      */
     double   pi_tol;        /* stop when |sigma_k - sigma_{k-1}| <= pi_tol * sigma_k (<=0: 1e-7) */
     uint64_t pi_seed;       /* seed of the starting vector                                       */
-    int32_t  precision;     /* contraction arithmetic: 0 FP32 FFMA, 1 3xTF32 tcgen05 tensor      */
-                            /* cores, 2 the generic FFMA kernels whatever the shape              */
-                            /* (cross-checks), 3 3xTF32 warp-level MMA (skinny shapes),          */
-                            /* -1 let the library choose by shape                                */
+    int32_t  precision;     /* contraction arithmetic, always FP32-accurate with FP32           */
+                            /* accumulation: 0 FP32 FFMA; 1 tcgen05 tensor cores (3-product      */
+                            /* TF32 split, or 3-product FP16 split x 2^k = h1 + h2 with          */
+                            /* overflow-free power-of-two scales, which needs U in Omega:        */
+                            /* ||U||_F^2 = K); 2 the generic FFMA kernels whatever the shape     */
+                            /* (cross-checks); 3 3xTF32 warp-level MMA; -1 let the library       */
+                            /* choose by shape                                                   */
     int32_t  history;       /* 1: keep one gem_nlr_iter_info per iteration in the workspace      */
 } gem_nlr_params;
 
@@ -93,7 +96,9 @@ typedef struct {
 
 /* Bytes of caller-provided device workspace needed for these parameters (0 if invalid).
  * Includes the y/sqrt(n) and ybar vectors, Theta, p, s, the reduction partials, the
- * optional history and, when x_inplace == 0, a copy of X.                                      */
+ * optional history, when x_inplace == 0 a copy of X and, for the wide tensor-core shapes
+ * (precision -1 or 1, r > 256, d a multiple of 32, n >= 4096), the static fp16 split images
+ * of X-hat, row-major and transposed (8 n d bytes).                                            */
 size_t gem_nlr_workspace_bytes(const gem_nlr_params *params);
 
 /* Device bytes the paper's own buffer table would use for the same problem:
