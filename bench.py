@@ -46,7 +46,7 @@ def _peaks():
 # Keyed by (n, d, r, kernel path); anything else reports null.
 NCU_TRAFFIC_BYTES = {
     (1_000_000, 128, 16, "mma.tf32x3"): 640.0e6,
-    (10_000_000, 64, 100, "f16x3+tf32x3"): 10.36e9,
+    (10_000_000, 64, 100, "f16x3"): 10.36e9,
     (2_000_000, 768, 1000, "f16x3.tiled"): 22.96e9,
     (100_000_000, 32, 8, "ffma"): 19.49e9,
 }
@@ -273,7 +273,7 @@ def main():
         it_s = ms * 1e-3 / (args.steps * T)
         # MMA flops actually issued on the tensor-core paths: three products per useful product; the fp16 split
         # runs on the f16 pipe (peak = the measured bf16 figure), the TF32 split on the TF32 pipe
-        if "f16x3" in path:
+        if "f16x3" in path and "tf32" not in path:
             tpeak, tpeak_kind = _tensor_peak_tf32()
             tpeak, tpeak_kind = tpeak / TF32_OVER_BF16, "measured bf16 sustained (f16 pipe)"
         else:

@@ -64,12 +64,13 @@ Layout make_layout(const gem_nlr_params& P)
     L.setup = take(sizeof(double) * (3 * (size_t)d + 4 + (size_t)L.gs * d));
     L.hist = take(P.history ? sizeof(gem_nlr_iter_info) * (size_t)(P.T > 0 ? P.T : 1) : 0);
     L.xhat = take(P.x_inplace ? 0 : sizeof(float) * (size_t)n * d);
-    // Wide tensor-core shapes (the tiled tcgen05 pair): X-hat is static, so its two-term fp16 split is built
-    // once, row-major (second product) and transposed (first product): 2 x 2 x n x d halves.
+    // tcgen05 shapes: X-hat is static, so its two-term fp16 split is built once, row-major (second product)
+    // and transposed in blocks of fb features x 32 rows (first product): about 2 x 2 x n x d halves.
     L.n_pad = (n + 63) / 64 * 64;
-    const bool wide_tc = (P.precision == -1 || P.precision == 1) && r > 256 && d % 32 == 0 && n >= 4096;
-    L.ximg = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)n * d : 0);
-    L.ximgT = take(wide_tc ? sizeof(uint16_t) * 2 * (size_t)(L.n_pad / 32) * ((d + 255) / 256) * 256 * 32 : 0);
+    L.fb = d >= 256 ? 256 : d;
+    const bool tc_images = (P.precision == -1 || P.precision == 1) && r >= 32 && d % 32 == 0 && n >= 4096;
+    L.ximg = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)n * d : 0);
+    L.ximgT = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)(L.n_pad / 32) * ((d + L.fb - 1) / L.fb) * L.fb * 32 : 0);
     L.total = off;
     return L;
 }
@@ -274,10 +275,12 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
         float* img = reinterpret_cast<float*>((char*)workspace_dev + L.thimg);
         if (tc_plan(h->pb, &h->tc, img)) {
             h->use_tc = true;
-            h->path = h->use_ffma ? "ffma+tf32x3" : "generic+tf32x3";
+            h->path = h->use_ffma ? (h->tc.f16 ? "ffma+f16x3" : "ffma+tf32x3") : (h->tc.f16 ? "generic+f16x3" : "generic+tf32x3");
             if (tc1_plan(h->pb, &h->tc1)) {
                 h->use_tc1 = true;
-                h->path = "f16x3+tf32x3";      // first product on the fp16 split, second on the TF32 split
+                // first product on the fp16 split; second on the fp16 split when the static images of X-hat
+                // are in the workspace, else on the TF32 split
+                h->path = h->tc.f16 ? "f16x3" : "f16x3+tf32x3";
             }
         }
         else if (tcg_plan(h->pb, &h->tcg, img)) {
@@ -323,7 +326,7 @@ int gem_nlr_spectral_norm(gem_nlr_t* h, double* a_out)
     CK(h, cudaStreamSynchronize(h->pb.stream));
     h->a = a;
     h->normalized = true;
-    if (h->use_tcg) {                                    // static fp16 images of X-hat for the tiled tensor-core kernels
+    if (h->pb.has_ximg() && (h->use_tcg || h->use_tc)) {  // static fp16 images of X-hat for the tensor-core kernels
         tcg_prepare(h->pb);
         CK(h, cudaStreamSynchronize(h->pb.stream));
     }
@@ -337,7 +340,7 @@ int gem_nlr_set_normalized(gem_nlr_t* h, double a)
     if (!h->pb.P.x_inplace) return GEM_NLR_E_INVALID;  // X-hat must be in the caller's buffer
     h->a = a;
     h->normalized = true;
-    if (h->use_tcg) {
+    if (h->pb.has_ximg() && (h->use_tcg || h->use_tc)) {
         tcg_prepare(h->pb);
         CK(h, cudaStreamSynchronize(h->pb.stream));
     }

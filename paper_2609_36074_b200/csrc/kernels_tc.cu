@@ -58,8 +58,35 @@ __global__ void k_theta_images(const float* __restrict__ theta, int d, int r, in
     }
 }
 
+// FP16 variant of the images for the two-term fp16 split: Theta^T 2^eT = h1 + h2, boxes of NP rows x 64 bytes
+// (32 features) with the 64-byte swizzle.
+__global__ void k_theta_images_h(const float* __restrict__ theta, int d, int r, int NP, int eT, const Ctl* __restrict__ ctl,
+                                 __half* __restrict__ img_h1, __half* __restrict__ img_h2)
+{
+    if (ctl->stopped) return;
+    const float sT = ldexpf(1.0f, eT);
+    const int NB = d / 32;
+    const int total = NB * 32 * NP;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const int j = e / NP, k = e % NP;             // feature, column
+        const float v = (k < r) ? theta[(size_t)j * r + k] * sT : 0.f;
+        const __half h1 = __float2half_rn(v);
+        const __half h2 = __float2half_rn(v - __half2float(h1));
+        const int b = j >> 5, jj = j & 31, c = jj >> 3, w = jj & 7;
+        const size_t off = (size_t)b * NP * 32 + (size_t)k * 32 + (((c ^ ((k >> 1) & 3)) << 3) + w);
+        img_h1[off] = h1;
+        img_h2[off] = h2;
+    }
+}
+
+// F16 = false: 3-product TF32 split, X-hat boxes split inside the kernel (warps 18-21).
+// F16 = true:  3-product FP16 split on the static fp16 images of X-hat (tmX = image h1, tmX2 = image h2: boxes
+//              of 128 rows x 32 features = 64-byte rows, 64-byte swizzle) and fp16 Theta^T images; K = 16 MMAs,
+//              nothing is split inside the kernel and the accumulator carries the scale 2^(15 + eT).
+template <bool F16>
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU,
+k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmX2,
+           const __grid_constant__ CUtensorMap tmU, int eT,
            const float* __restrict__ U, const float* __restrict__ img_hi, const float* __restrict__ img_lo,
            const float* __restrict__ ybar, const float* __restrict__ p, const float* __restrict__ alpha_s,
            Ctl* __restrict__ ctl, int64_t n, int d, int r, int NP, int PW, int NSB, int NLO, int NUP, float alpha, int K,
@@ -83,7 +110,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     const int PAN_BYTES = TILE_M * PW * 4;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * ACC_COLS) tmem_cols <<= 1;
-    const uint32_t th_bytes = (uint32_t)NB * NP * 128;
+    const uint32_t th_bytes = (uint32_t)NB * NP * (F16 ? 64 : 128);
 
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t stage0 = smem_base;                                   // NSB boxes: raw, then hi in place
@@ -128,7 +155,8 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
 
     const int64_t n_tiles = (n + TILE_M - 1) / TILE_M;
     const float cf = ctl->c_f;
-    const float two_alpha = 2.0f * alpha;
+    // F16: the accumulator holds (x-hat 2^15)(Theta 2^eT) sums; the scales go into the 2 alpha factor
+    const float two_alpha = F16 ? 2.0f * alpha * ldexpf(1.0f, -15 - eT) : 2.0f * alpha;
     double sa = 0.0, sb = 0.0, sh = 0.0;
     double csum[2][2];                   // epilogue thread: running sums of its column (after the transpose-reduce) per
     csum[0][0] = csum[0][1] = csum[1][0] = csum[1][1] = 0.0;   // (panel of the group, 16-column half); over this quarter's rows
@@ -146,7 +174,12 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     const int g = i * NB + b, s = g % NSB;
                     if (g >= NSB) mbar_wait(xfree(s), ((g / NSB) - 1) & 1, &abort_flag, ctl);
                     mbar_expect_tx(xfull(s), BOX_BYTES);
-                    tma_load_2d(stage0 + (uint32_t)s * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
+                    if (F16) {      // image boxes h1 | h2, 8 KB each
+                        tma_load_2d(stage0 + (uint32_t)s * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
+                        tma_load_2d(stage0 + (uint32_t)s * BOX_BYTES + BOX_BYTES / 2, &tmX2, b * 32, row0, xfull(s));
+                    } else {
+                        tma_load_2d(stage0 + (uint32_t)s * BOX_BYTES, &tmX, b * 32, row0, xfull(s));
+                    }
                 }
             }
         }
@@ -181,35 +214,47 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_tf32(TILE_M, NP, 0, 0);
+            const uint32_t idesc = F16 ? umma_idesc_f16(TILE_M, NP, 0, 0) : umma_idesc_tf32(TILE_M, NP, 0, 0);
             mbar_wait(thfull, 0, &abort_flag, ctl);
             // Inside a tile the wait for the next box sits in the middle of the current box's k-steps, so the
-            // tensor pipe has MMAs queued while this thread polls.
+            // tensor pipe has MMAs queued while this thread polls.  F16: the boxes come ready from TMA (xfull);
+            // TF32: from the split warps (xsplit).
             int i = 0;
             for (int64_t t = blockIdx.x; t < n_tiles && !abort_flag; t += gridDim.x, ++i) {
                 const int a = i & 1;
                 // tile boundary: the accumulator hand-over of the previous tile is already committed, so the
                 // epilogue runs while this thread waits for a free accumulator and the first box
                 if (i >= 2) mbar_wait(accfree(a), ((i >> 1) - 1) & 1, &abort_flag, ctl);
-                mbar_wait(xsplit((i * NB) % NSB), ((i * NB) / NSB) & 1, &abort_flag, ctl);
+                mbar_wait(F16 ? xfull((i * NB) % NSB) : xsplit((i * NB) % NSB), ((i * NB) / NSB) & 1, &abort_flag, ctl);
                 const uint32_t tacc = tmem_base + (uint32_t)(a * ACC_COLS);
                 for (int b = 0; b < NB; ++b) {
-                    const int g = i * NB + b, s = g % NSB, l = g % NLO;
+                    const int g = i * NB + b, s = g % NSB, l = F16 ? 0 : g % NLO;
                     tc_fence_after();
-                    const uint32_t a_hi = stage0 + (uint32_t)s * BOX_BYTES, a_lo = lo0 + (uint32_t)l * BOX_BYTES;
-                    const uint32_t b_hi = th_hi_s + (uint32_t)b * NP * 128, b_lo = th_lo_s + (uint32_t)b * NP * 128;
-                    // descriptors once per box; a k-step (8 features = 32 bytes inside the 128-byte
-                    // swizzled row) advances the start-address field by 2
-                    const uint64_t da_hi = umma_desc_sw128(a_hi, 16, 1024), da_lo = umma_desc_sw128(a_lo, 16, 1024);
-                    const uint64_t db_hi = umma_desc_sw128(b_hi, 16, 1024), db_lo = umma_desc_sw128(b_lo, 16, 1024);
+                    if (F16) {
+                        const uint32_t a_h1 = stage0 + (uint32_t)s * BOX_BYTES, a_h2 = a_h1 + BOX_BYTES / 2;
+                        const uint32_t b_h1 = th_hi_s + (uint32_t)b * NP * 64, b_h2 = th_lo_s + (uint32_t)b * NP * 64;
+                        const uint64_t da1 = umma_desc_k_sw64(a_h1), da2 = umma_desc_k_sw64(a_h2);
+                        const uint64_t db1 = umma_desc_k_sw64(b_h1), db2 = umma_desc_k_sw64(b_h2);
+                        umma_f16_x3(tacc, da1, da2, db1, db2, idesc, b ? 1u : 0u);
+                        if (b + 1 < NB) mbar_wait(xfull((g + 1) % NSB), ((g + 1) / NSB) & 1, &abort_flag, ctl);
+                        umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
+                        umma_commit(xfree(s));
+                    } else {
+                        const uint32_t a_hi = stage0 + (uint32_t)s * BOX_BYTES, a_lo = lo0 + (uint32_t)l * BOX_BYTES;
+                        const uint32_t b_hi = th_hi_s + (uint32_t)b * NP * 128, b_lo = th_lo_s + (uint32_t)b * NP * 128;
+                        // descriptors once per box; a k-step (8 features = 32 bytes inside the 128-byte
+                        // swizzled row) advances the start-address field by 2
+                        const uint64_t da_hi = umma_desc_sw128(a_hi, 16, 1024), da_lo = umma_desc_sw128(a_lo, 16, 1024);
+                        const uint64_t db_hi = umma_desc_sw128(b_hi, 16, 1024), db_lo = umma_desc_sw128(b_lo, 16, 1024);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        if (ks == 2 && b + 1 < NB) mbar_wait(xsplit((g + 1) % NSB), ((g + 1) / NSB) & 1, &abort_flag, ctl);
-                        umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
-                                     (b | ks) ? 1u : 0u);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            if (ks == 2 && b + 1 < NB) mbar_wait(xsplit((g + 1) % NSB), ((g + 1) / NSB) & 1, &abort_flag, ctl);
+                            umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
+                                         (b | ks) ? 1u : 0u);
+                        }
+                        umma_commit(xfree(s));
+                        umma_commit(lofree(l));
                     }
-                    umma_commit(xfree(s));
-                    umma_commit(lofree(l));
                 }
                 umma_commit(accfull(a));
             }
@@ -218,7 +263,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         // ------------------------------ split: box -> hi (in place), lo ------------------------------
         const int st = threadIdx.x - (2 + 4 * NGROUPS) * 32;   // 0..127
         int i = 0;
-        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
+        for (int64_t t = blockIdx.x; !F16 && t < n_tiles; t += gridDim.x, ++i) {
             for (int b = 0; b < NB; ++b) {
                 const int g = i * NB + b, s = g % NSB, l = g % NLO;
                 mbar_wait(xfull(s), (g / NSB) & 1, &abort_flag, ctl);
@@ -395,30 +440,51 @@ bool tc_plan(const Problem& pb, TcPlan* pl, float* img_storage)
     if (NPAN > 8) return false;
     const int ACC_COLS = (NPAN * PW + 31) / 32 * 32;
     const size_t pan_bytes = (size_t)tc::TILE_M * PW * 4;
-    const size_t th = (size_t)NB * NP * 128;
+    // fp16 split on the static images of X-hat when the workspace holds them, else the TF32 split
+    const bool f16 = pb.has_ximg();
+    const size_t th = (size_t)NB * NP * (f16 ? 64 : 128);
     const size_t fixed = 2 * th + (size_t)2 * ACC_COLS * 4 + 1024;
     const size_t limit = 227 * 1024 - 2048;
-    // Ring sizes under the 227 KB limit.  The U panel ring comes first (a slot is released one
-    // panel after its store was issued, so fewer than 4 slots serialises the panel loads); then
-    // the lo boxes (split -> MMA -> free round trip); the raw X-hat box ring takes what is left
-    // and sets how far the TMA loads run ahead.
+    // Ring sizes under the 227 KB limit.  The U panel ring comes first (a group's slot is refilled only
+    // after its store, so more slots let the next tile's panels load during this tile's epilogue); then the
+    // lo boxes of the TF32 split (split -> MMA -> free round trip); the X-hat box ring takes what is left.
     int NSB = 0, NUP = 0, NLO = 0;
-    for (int nup = 4; nup >= 2 && !NSB; --nup)
-        for (int nlo = 3; nlo >= 2 && !NSB; --nlo)
-            for (int nsb = tc::MAX_RING; nsb >= (nlo == 3 ? 4 : 2); --nsb)
-                if (fixed + (size_t)(nsb + nlo) * tc::BOX_BYTES + (size_t)nup * pan_bytes <= limit) {
-                    NSB = nsb; NUP = nup; NLO = nlo; break;
-                }
+    if (f16) {
+        for (int nup = 8; nup >= 2 && !NSB; --nup)
+            for (int nsb = 6; nsb >= 4; --nsb)
+                if (fixed + (size_t)nsb * tc::BOX_BYTES + (size_t)nup * pan_bytes <= limit) { NSB = nsb; NUP = nup; break; }
+    } else {
+        for (int nup = 4; nup >= 2 && !NSB; --nup)
+            for (int nlo = 3; nlo >= 2 && !NSB; --nlo)
+                for (int nsb = tc::MAX_RING; nsb >= (nlo == 3 ? 4 : 2); --nsb)
+                    if (fixed + (size_t)(nsb + nlo) * tc::BOX_BYTES + (size_t)nup * pan_bytes <= limit) {
+                        NSB = nsb; NUP = nup; NLO = nlo; break;
+                    }
+    }
     if (!NSB) return false;
+    pl->f16 = f16;
+    {
+        int e;
+        frexpf(sqrtf((float)pb.P.K), &e);                  // |Theta_jk| <= ||X-hat||_2 ||U||_F = sqrt(K) <= 2^e
+        pl->eT = 14 - e;
+    }
     pl->NP = NP; pl->PW = PW; pl->NSB = NSB; pl->NLO = NLO; pl->NUP = NUP;
     pl->smem2 = fixed + (size_t)(NSB + NLO) * tc::BOX_BYTES + (size_t)NUP * pan_bytes;
     pl->img_hi = img_storage;
-    pl->img_lo = img_storage + (size_t)NB * 32 * NP;
-    if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc::TILE_M, 32)) return false;
+    pl->img_lo = f16 ? reinterpret_cast<float*>(reinterpret_cast<uint16_t*>(img_storage) + (size_t)NB * 32 * NP)
+                     : img_storage + (size_t)NB * 32 * NP;
+    if (f16) {
+        if (!make_tensor_map_2d_f16(&pl->tmX, pb.ximg(0), pb.P.n, d, d, tc::TILE_M, 32)) return false;
+        if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, d, tc::TILE_M, 32)) return false;
+    } else {
+        if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc::TILE_M, 32)) return false;
+        pl->tmX2 = pl->tmX;
+    }
     if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tc::TILE_M, PW)) return false;
     const int64_t tiles = (pb.P.n + tc::TILE_M - 1) / tc::TILE_M;
     pl->g2 = (int)(tiles < kSMs ? tiles : kSMs);
-    if (cudaFuncSetAttribute(tc::k_pass2_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
+    if (cudaFuncSetAttribute(tc::k_pass2_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess ||
+        cudaFuncSetAttribute(tc::k_pass2_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
         return false;
     return true;
 }
@@ -427,10 +493,19 @@ void tc_launch_second(const Problem& pb, const TcPlan& pl)
 {
     const int d = pb.P.d, r = pb.P.r;
     const int total = d * pl.NP;
-    tc::k_theta_images<<<(total + 255) / 256, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NP, pb.ctl(), pl.img_hi, pl.img_lo);
-    tc::k_pass2_tc<<<pl.g2, tc::NTHREADS, pl.smem2, pb.stream>>>(
-        pl.tmX, pl.tmU, pb.U, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NP,
-        pl.PW, pl.NSB, pl.NLO, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
+    if (pl.f16) {
+        tc::k_theta_images_h<<<(total + 255) / 256, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NP, pl.eT, pb.ctl(),
+                                                                         reinterpret_cast<__half*>(pl.img_hi),
+                                                                         reinterpret_cast<__half*>(pl.img_lo));
+        tc::k_pass2_tc<true><<<pl.g2, tc::NTHREADS, pl.smem2, pb.stream>>>(
+            pl.tmX, pl.tmX2, pl.tmU, pl.eT, pb.U, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d,
+            r, pl.NP, pl.PW, pl.NSB, pl.NLO, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
+    } else {
+        tc::k_theta_images<<<(total + 255) / 256, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NP, pb.ctl(), pl.img_hi, pl.img_lo);
+        tc::k_pass2_tc<false><<<pl.g2, tc::NTHREADS, pl.smem2, pb.stream>>>(
+            pl.tmX, pl.tmX2, pl.tmU, 0, pb.U, pl.img_hi, pl.img_lo, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r,
+            pl.NP, pl.PW, pl.NSB, pl.NLO, pl.NUP, pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
+    }
     pb.count(2);
 }
 

@@ -66,13 +66,13 @@ __global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, 
 }
 
 // X-hat (n x d FP32) -> its fp16 split images x 2^15 = h1 + h2: row-major (n x d), and transposed in the
-// exact shared-memory form the first product consumes: for every stage of 32 data rows and block of 256
-// features one contiguous 16 KB box [feature][32 rows] with the 64-byte swizzle already applied (zero
+// exact shared-memory form the first product consumes: for every stage of 32 data rows and block of fb
+// features one contiguous box [feature][32 rows] with the 64-byte swizzle already applied (zero
 // beyond n and d), so that a box arrives with one bulk copy.  One block per 32 x 32 tile; the
 // transposition goes through shared memory.
 __global__ void __launch_bounds__(256)
-k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, __half* __restrict__ h1, __half* __restrict__ h2,
-             __half* __restrict__ h1T, __half* __restrict__ h2T)
+k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, int fb, __half* __restrict__ h1,
+             __half* __restrict__ h2, __half* __restrict__ h1T, __half* __restrict__ h2T)
 {
     __shared__ __half t1[32][33], t2[32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;            // 32 x 8
@@ -94,9 +94,9 @@ k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, __hal
     for (int i = 0; i < 4; ++i) {
         const int f = f0 + ty + 8 * i;
         const int64_t row = row0 + tx;
-        if (row < n_pad) {                                 // features d .. 256 NNB - 1 of the last block stay zero (memset)
-            const int nnb = (d + 255) / 256, nbk = f >> 8, m = f & 255, kk = tx;       // kk = row inside the stage
-            const size_t off = (((size_t)blockIdx.x * nnb + nbk) * 256 + m) * 32 + (size_t)((((kk >> 3) ^ ((m >> 1) & 3)) << 3) + (kk & 7));
+        if (row < n_pad) {                                 // features beyond d of the last block stay zero (memset)
+            const int nnb = (d + fb - 1) / fb, nbk = f / fb, m = f - nbk * fb, kk = tx;     // kk = row inside the stage
+            const size_t off = (((size_t)blockIdx.x * nnb + nbk) * fb + m) * 32 + (size_t)((((kk >> 3) ^ ((m >> 1) & 3)) << 3) + (kk & 7));
             if (f < d) { h1T[off] = t1[tx][ty + 8 * i]; h2T[off] = t2[tx][ty + 8 * i]; }
         }
     }
@@ -576,7 +576,7 @@ void tcg_prepare(const Problem& pb)
 {
     cudaMemsetAsync(pb.ximgT(0), 0, sizeof(uint16_t) * 2 * pb.ximgT_halves(), pb.stream);
     const dim3 grid((unsigned)((pb.L.n_pad + 31) / 32), (unsigned)((pb.P.d + 31) / 32));
-    tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.P.d, pb.L.n_pad,
+    tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.P.d, pb.L.n_pad, pb.L.fb,
                                                    reinterpret_cast<__half*>(pb.ximg(0)), reinterpret_cast<__half*>(pb.ximg(1)),
                                                    reinterpret_cast<__half*>(pb.ximgT(0)), reinterpret_cast<__half*>(pb.ximgT(1)));
     pb.count(1);
@@ -585,7 +585,7 @@ void tcg_prepare(const Problem& pb)
 bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
 {
     const int d = pb.P.d, r = pb.P.r;
-    if (!pb.has_ximg() || d % 32 != 0 || r % 4 != 0 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
+    if (!pb.has_ximg() || pb.L.fb != 256 || d % 32 != 0 || r % 4 != 0 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
     pl->NMT = (r + 127) / 128;
     pl->NNB = (d + 255) / 256;
     const int tiles = pl->NMT * pl->NNB;

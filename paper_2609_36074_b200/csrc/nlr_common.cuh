@@ -30,7 +30,8 @@ struct Ctl {
 struct Layout {
     size_t ctl, p, s, alpha_s, theta, thimg, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
     size_t ximg, ximgT;      // fp16 split images of X-hat (row-major and transposed), wide tensor-core shapes only (else 0 bytes)
-    int64_t n_pad;           // row count of the transposed images' rows, n rounded up to 64
+    int64_t n_pad;           // n rounded up to 64: the transposed images cover n_pad / 32 stages of 32 rows
+    int fb;                  // features per block of the transposed images: 256, or d when d < 256
     int g1x, g1y_d, g1y_r;   // generic pass-1 grid: row chunks, d tiles, r tiles
     int gv;                  // vector kernel CTAs
     int g2x, g2y;            // generic pass-2 grid: row-tile CTAs, column tiles
@@ -62,8 +63,8 @@ struct Problem {
     float* theta() const { return reinterpret_cast<float*>(ws + L.theta); }
     // fp16 split images of X-hat (wide tensor-core shapes): h1 then h2, row-major n x d; transposed d x n_pad
     uint16_t* ximg(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximg) + (size_t)which * P.n * P.d; }
-    // transposed images: [n_pad / 32 stages][ceil(d / 256) blocks][256 features][32 rows] halves each
-    size_t ximgT_halves() const { return (size_t)(L.n_pad / 32) * ((P.d + 255) / 256) * 256 * 32; }
+    // transposed images: [n_pad / 32 stages][ceil(d / fb) blocks][fb features][32 rows] halves each
+    size_t ximgT_halves() const { return (size_t)(L.n_pad / 32) * ((P.d + L.fb - 1) / L.fb) * L.fb * 32; }
     uint16_t* ximgT(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximgT) + (size_t)which * ximgT_halves(); }
     bool has_ximg() const { return L.ximgT > L.ximg; }
     float* ytilde() const { return reinterpret_cast<float*>(ws + L.ytilde); }

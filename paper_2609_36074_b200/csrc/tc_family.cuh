@@ -6,8 +6,11 @@
 namespace gemnlr {
 
 struct TcPlan {
-    alignas(64) CUtensorMap tmX;   // X-hat boxes: 128 rows x 32 features
+    alignas(64) CUtensorMap tmX;   // X-hat boxes: 128 rows x 32 features (FP32, or the fp16 image h1)
+    alignas(64) CUtensorMap tmX2;  // fp16 image h2 (fp16 split only)
     alignas(64) CUtensorMap tmU;   // U panels: 128 rows x 32 columns (load and store)
+    bool f16;                      // two-term fp16 split on the static images of X-hat, else the TF32 split
+    int eT;                        // Theta is scaled by 2^eT before its fp16 split
     int NP;                        // r padded to a multiple of 16 (MMA N)
     int PW;                        // columns per U panel: 16 (plain rows) or 32 (128-byte swizzle)
     int NSB, NLO, NUP;             // raw/hi box ring, lo box ring, U panel ring sizes
