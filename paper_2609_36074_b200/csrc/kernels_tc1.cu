@@ -51,9 +51,13 @@ constexpr int MAX_RING = 8;
 constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
 constexpr int UIMG = 128 * 64;                 // one fp16 image of the U operand: 128 columns x 32 data rows
 
+// XIMG = true: the X-hat operand comes from the static transposed fp16 images (one contiguous, pre-swizzled
+// box of d x 32 halves per stage and image, bulk-copied straight into the image stage); the raw stage then
+// holds the U rows only and the teams convert only U.  XIMG = false: the teams convert the FP32 rows of X-hat too.
+template <bool XIMG>
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
-           float* __restrict__ ytilde, float* __restrict__ ybar, Ctl* __restrict__ ctl,
+k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __half* __restrict__ xT1,
+           const __half* __restrict__ xT2, float* __restrict__ ytilde, float* __restrict__ ybar, Ctl* __restrict__ ctl,
            const float* __restrict__ p, int64_t n, int d, int r, int K, int NSR, int NLO, double gamma,
            double* __restrict__ part)
 {
@@ -72,9 +76,9 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
     // raw stage: the TR rows of U then those of X-hat exactly as they lie in global memory (row pitch r and
     // d floats): the rows of a stage are contiguous there, so each operand arrives with one bulk copy
     const int URAW = (TR * r * 4 + 127) / 128 * 128;
-    const int STAGE = (URAW + TR * d * 4 + 1023) / 1024 * 1024;
-    const int XIMG = d * 64;                       // one fp16 image of the X-hat operand: d features x 32 data rows
-    const int IMG = 2 * UIMG + 2 * XIMG;           // image stage: U h1, U h2, X h1, X h2
+    const int STAGE = (URAW + (XIMG ? 0 : TR * d * 4) + 1023) / 1024 * 1024;
+    const int XIMG_BYTES = d * 64;                 // one fp16 image of the X-hat operand: d features x 32 data rows
+    const int IMG = 2 * UIMG + 2 * XIMG_BYTES;           // image stage: U h1, U h2, X h1, X h2
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * d) tmem_cols <<= 1;
 
@@ -92,7 +96,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_RING; ++s) {
-            mbar_init(full(s), 1); mbar_init(split(s), 4); mbar_init(rawfree(s), 4); mbar_init(lofree(s), 1);
+            mbar_init(full(s), 1); mbar_init(split(s), XIMG ? 5 : 4); mbar_init(rawfree(s), 4); mbar_init(lofree(s), 1);
         }
         for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), 4); }
         abort_flag = 0;
@@ -136,9 +140,23 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
                 const int64_t row0 = (g_lo + g) * TR;
                 const int rows = (n - row0 < TR) ? (int)(n - row0) : TR;
                 const uint32_t dst = raw0 + (uint32_t)s * STAGE;
-                mbar_expect_tx(full(s), (uint32_t)(rows * (r + d) * 4));
-                bulk_load_1d(dst, U + row0 * r, (uint32_t)(rows * r * 4), full(s));
-                bulk_load_1d(dst + URAW, X + row0 * d, (uint32_t)(rows * d * 4), full(s));
+                if (XIMG) {
+                    mbar_expect_tx(full(s), (uint32_t)(rows * r * 4));
+                    bulk_load_1d(dst, U + row0 * r, (uint32_t)(rows * r * 4), full(s));
+                    // the X-hat boxes of this stage go straight into its image stage, once the MMAs of the
+                    // stage that used it last are done
+                    const int l = g % NLO;
+                    if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+                    const uint32_t im = img0 + (uint32_t)l * IMG;
+                    const size_t xoff = (size_t)(g_lo + g) * d * 32;          // one block of d features per stage
+                    mbar_expect_tx(split(l), (uint32_t)(2 * XIMG_BYTES));
+                    bulk_load_1d(im + 2 * UIMG, xT1 + xoff, (uint32_t)XIMG_BYTES, split(l));
+                    bulk_load_1d(im + 2 * UIMG + XIMG_BYTES, xT2 + xoff, (uint32_t)XIMG_BYTES, split(l));
+                } else {
+                    mbar_expect_tx(full(s), (uint32_t)(rows * (r + d) * 4));
+                    bulk_load_1d(dst, U + row0 * r, (uint32_t)(rows * r * 4), full(s));
+                    bulk_load_1d(dst + URAW, X + row0 * d, (uint32_t)(rows * d * 4), full(s));
+                }
             }
         }
     } else if (warp == 1) {
@@ -159,7 +177,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
                 // A = U images (M = 128 columns), B = X-hat images (N = d features), K-major; a k-step of 16 data
                 // rows (32 bytes inside the 64-byte swizzled row) advances the start address by 2
                 const uint64_t da1 = umma_desc_k_sw64(im), da2 = umma_desc_k_sw64(im + UIMG);
-                const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG), db2 = umma_desc_k_sw64(im + 2 * UIMG + XIMG);
+                const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG), db2 = umma_desc_k_sw64(im + 2 * UIMG + XIMG_BYTES);
                 umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
                 int ln = l + 1, lphn = lph;
                 if (ln == NLO) { ln = 0; lphn ^= 1; }
@@ -256,7 +274,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
                 ybar[myrow] = yb_l;
             }
             // ---- X-hat boxes -> fp16 images: thread = (feature tt & 31, data rows 8 (tt >> 5) .. + 7) of a box ----
-            for (int b = 0; b < NBX; ++b) {
+            for (int b = 0; !XIMG && b < NBX; ++b) {
                 float v[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
@@ -265,7 +283,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U,
                 split_h8(v, h1, h2);
                 const uint32_t io = kimg_off(b * 32 + lane, tw);
                 sts128u(im + 2 * UIMG + io, h1);
-                sts128u(im + 2 * UIMG + XIMG + io, h2);
+                sts128u(im + 2 * UIMG + XIMG_BYTES + io, h2);
             }
             fence_proxy_async();
             __syncwarp();
@@ -337,7 +355,8 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     if (d % 32 != 0 || d > 256 || r % 4 != 0 || r < 8 || r > 128 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
     if ((size_t)d * r > 16384) return false;          // partial records of the shared reduction kernel
     const int NBX = d / 32;
-    const size_t stage = (((size_t)tc1::TR * r * 4 + 127) / 128 * 128 + (size_t)tc1::TR * d * 4 + 1023) / 1024 * 1024;
+    const bool ximg = pb.has_ximg() && pb.L.fb == d;          // one block of d features per stage in the transposed images
+    const size_t stage = (((size_t)tc1::TR * r * 4 + 127) / 128 * 128 + (ximg ? 0 : (size_t)tc1::TR * d * 4) + 1023) / 1024 * 1024;
     const size_t img = (size_t)2 * tc1::UIMG + (size_t)2 * d * 64;
     const size_t limit = 227 * 1024 - 2048;
     int NLO = 0, NSR = 0;
@@ -345,21 +364,29 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
         for (int nsr = 6; nsr >= 3; --nsr)
             if ((size_t)nsr * stage + (size_t)nlo * img + 1024 <= limit) { NSR = nsr; NLO = nlo; break; }
     if (!NSR) return false;
-    pl->NSR = NSR; pl->NLO = NLO;
+    pl->NSR = NSR; pl->NLO = NLO; pl->ximg = ximg;
     pl->smem = (size_t)NSR * stage + (size_t)NLO * img + 1024;
     if (pl->smem < (size_t)8 * 128 * 4 + 1024) pl->smem = (size_t)8 * 128 * 4 + 1024;     // s scratch of the tail
     const int64_t stages = (pb.P.n + tc1::TR - 1) / tc1::TR;
     pl->grid = (int)(stages < kSMs ? stages : kSMs);
-    if (cudaFuncSetAttribute(tc1::k_pass1_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(tc1::k_pass1_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess ||
+        cudaFuncSetAttribute(tc1::k_pass1_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem) != cudaSuccess)
         return false;
     return true;
 }
 
 void tc1_launch_first(const Problem& pb, const Tc1Plan& pl)
 {
-    tc1::k_pass1_tc<<<pl.grid, tc1::NTHREADS, pl.smem, pb.stream>>>(
-        pb.X, pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.P.d, pb.P.r, pb.P.K, pl.NSR, pl.NLO, pb.gamma,
-        pb.part1());
+    const __half* x1 = pl.ximg ? reinterpret_cast<const __half*>(pb.ximgT(0)) : nullptr;
+    const __half* x2 = pl.ximg ? reinterpret_cast<const __half*>(pb.ximgT(1)) : nullptr;
+    if (pl.ximg)
+        tc1::k_pass1_tc<true><<<pl.grid, tc1::NTHREADS, pl.smem, pb.stream>>>(
+            pb.X, pb.U, x1, x2, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.P.d, pb.P.r, pb.P.K, pl.NSR, pl.NLO,
+            pb.gamma, pb.part1());
+    else
+        tc1::k_pass1_tc<false><<<pl.grid, tc1::NTHREADS, pl.smem, pb.stream>>>(
+            pb.X, pb.U, x1, x2, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.P.d, pb.P.r, pb.P.K, pl.NSR, pl.NLO,
+            pb.gamma, pb.part1());
     pb.count(1);
 }
 

@@ -35,7 +35,8 @@ namespace gemnlr {
 struct Tc1Plan {
     alignas(64) CUtensorMap tmX;   // X-hat boxes: 32 rows x 32 features
     alignas(64) CUtensorMap tmU;   // U boxes: 32 rows x 32 columns
-    int NSR, NLO;                  // raw stage ring, lo stage ring
+    int NSR, NLO;                  // raw stage ring, image stage ring
+    bool ximg;                     // X-hat operand from the static transposed fp16 images
     int grid;
     size_t smem;
 };
