@@ -202,19 +202,23 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
         float p1[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) p1[j] = sp[lane + 32 * j];
-        // ytilde of this warp's eight rows (lane k < 8 holds row 8 tw + k) is requested one of the team's
-        // stages ahead, so its DRAM latency is not paid inside the stage
+        // ytilde of this warp's eight rows (lane 4 k holds row 8 tw + k: the lane group that ends up with the
+        // row's dot product) is requested one of the team's stages ahead, so its DRAM latency is not paid
+        // inside the stage
+        const bool owner = (lane & 3) == 0;
+        const float cs = cf * sU, inv_sU = 1.0f / sU;      // everything below works on v = u 2^eU: scaling by a
+                                                           // power of two commutes with every FP32 rounding
         float yt_next = 0.f;
         if (team < my_stages) {
-            const int64_t row_f = (g_lo + team) * TR + 8 * tw + (lane & 7);
-            if (lane < 8 && row_f < n) yt_next = ytilde[row_f];
+            const int64_t row_f = (g_lo + team) * TR + 8 * tw + (lane >> 2);
+            if (owner && row_f < n) yt_next = ytilde[row_f];
         }
         for (int g = team; g < my_stages; g += NTEAMS) {
             const int s = g % NSR, l = g % NLO;
             const int64_t srow0 = (g_lo + g) * TR;
-            const int64_t myrow = srow0 + 8 * tw + (lane & 7);
+            const int64_t myrow = srow0 + 8 * tw + (lane >> 2);
             float yt_l = yt_next;
-            yt_next = (g + NTEAMS < my_stages && lane < 8 && myrow + NTEAMS * TR < n) ? ytilde[myrow + NTEAMS * TR] : 0.f;
+            yt_next = (g + NTEAMS < my_stages && owner && myrow + NTEAMS * TR < n) ? ytilde[myrow + NTEAMS * TR] : 0.f;
             float yb_l = 0.f;
             mbar_wait_spin(full(s), (g / NSR) & 1, &abort_flag, ctl);
             if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
@@ -228,21 +232,36 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 for (int j = 0; j < 4; ++j) {        // columns beyond r and rows beyond n are zero
                     const float w = (lane + 32 * j < r && 8 * tw + k < rows_here)
                                         ? lds32f(hi_s + (uint32_t)(((8 * tw + k) * r + lane + 32 * j) * 4)) : 0.f;
-                    u[k][j] = cf * w;
+                    u[k][j] = cs * w;                // v = u 2^eU with u = fl(c_f w)
                     dot[k] = fmaf(u[k][j], p1[j], dot[k]);
                 }
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-                for (int k = 0; k < 8; ++k) dot[k] += __shfl_xor_sync(0xffffffffu, dot[k], o);
-            // row scalars: lane k < 8 owns row 8 tw + k (dot[] is the same in every lane)
+            // the eight row sums by recursive halving: lane l ends up with the total of row (l >> 2) & 7
+            float q;
             {
-                float q = dot[0];
+                float e4[4], e2[2];
+                const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4;
 #pragma unroll
-                for (int k = 1; k < 8; ++k) q = ((lane & 7) == k) ? dot[k] : q;
-                const float qm1 = q - 1.0f;
-                if (lane < 8) {
+                for (int i = 0; i < 4; ++i) {
+                    const float send = b4 ? dot[i] : dot[i + 4], keep = b4 ? dot[i + 4] : dot[i];
+                    e4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float send = b3 ? e4[i] : e4[i + 2], keep = b3 ? e4[i + 2] : e4[i];
+                    e2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+                }
+                {
+                    const float send = b2 ? e2[0] : e2[1], keep = b2 ? e2[1] : e2[0];
+                    q = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+                }
+                q += __shfl_xor_sync(0xffffffffu, q, 2);
+                q += __shfl_xor_sync(0xffffffffu, q, 1);
+            }
+            // row scalars: lane 4 k owns row 8 tw + k
+            {
+                const float qm1 = q * inv_sU - 1.0f;
+                if (owner) {
                     if (dual) yt_l = (float)((double)yt_l + gamma * (double)qm1);
                     yb_l = (float)((double)yt_l + gamma * (double)qm1);
                     if (myrow < n) {
@@ -253,23 +272,23 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
             }
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-                const float yb = __shfl_sync(0xffffffffu, yb_l, k);
+                const float yb = __shfl_sync(0xffffffffu, yb_l, 4 * k);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) s_acc[j] = fmaf(u[k][j], yb, s_acc[j]);     // rows beyond n: u = 0
+                for (int j = 0; j < 4; ++j) s_acc[j] = fmaf(u[k][j], yb, s_acc[j]);     // rows beyond n: u = 0; scaled by 2^eU
             }
             // images of u 2^eU (u = c_f w rounded to FP32, as the plain definition has it): one chunk per column
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 float v[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) v[k] = u[k][j] * sU;
+                for (int k = 0; k < 8; ++k) v[k] = u[k][j];
                 uint4 h1, h2;
                 split_h8(v, h1, h2);
                 const uint32_t io = kimg_off(lane + 32 * j, tw);
                 sts128u(im + io, h1);
                 sts128u(im + UIMG + io, h2);
             }
-            if (lane < 8 && myrow < n) {
+            if (owner && myrow < n) {
                 if (dual) ytilde[myrow] = yt_l;
                 ybar[myrow] = yb_l;
             }
@@ -331,7 +350,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
     float* sscr = reinterpret_cast<float*>(smem);             // [vector warps][128 columns]
     if (warp >= 6) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + lane + 32 * k] = s_acc[k];
+        for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + lane + 32 * k] = s_acc[k] * ldexpf(1.0f, -eU);
     }
     __syncthreads();
     if (threadIdx.x < r) {
