@@ -46,7 +46,7 @@ namespace tc1 {
 constexpr int TR = 32;                         // data rows per stage (4 k-steps)
 constexpr int CHUNK_BYTES = TR * 128;          // one box: TR rows x 32 floats
 constexpr int NTEAMS = 3;                      // vector / split teams of four warps, taking stages round-robin
-constexpr int NTHREADS = (6 + 4 * NTEAMS) * 32;
+constexpr int NTHREADS = (6 + 4 * NTEAMS + 1) * 32;   // + the X-hat image producer (last warp)
 constexpr int MAX_RING = 8;
 constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
 constexpr int UIMG = 128 * 64;                 // one fp16 image of the U operand: 128 columns x 32 data rows
@@ -143,20 +143,27 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 if (XIMG) {
                     mbar_expect_tx(full(s), (uint32_t)(rows * r * 4));
                     bulk_load_1d(dst, U + row0 * r, (uint32_t)(rows * r * 4), full(s));
-                    // the X-hat boxes of this stage go straight into its image stage, once the MMAs of the
-                    // stage that used it last are done
-                    const int l = g % NLO;
-                    if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
-                    const uint32_t im = img0 + (uint32_t)l * IMG;
-                    const size_t xoff = (size_t)(g_lo + g) * d * 32;          // one block of d features per stage
-                    mbar_expect_tx(split(l), (uint32_t)(2 * XIMG_BYTES));
-                    bulk_load_1d(im + 2 * UIMG, xT1 + xoff, (uint32_t)XIMG_BYTES, split(l));
-                    bulk_load_1d(im + 2 * UIMG + XIMG_BYTES, xT2 + xoff, (uint32_t)XIMG_BYTES, split(l));
                 } else {
                     mbar_expect_tx(full(s), (uint32_t)(rows * (r + d) * 4));
                     bulk_load_1d(dst, U + row0 * r, (uint32_t)(rows * r * 4), full(s));
                     bulk_load_1d(dst + URAW, X + row0 * d, (uint32_t)(rows * d * 4), full(s));
                 }
+            }
+        }
+    } else if (warp == 6 + 4 * NTEAMS) {
+        // ------------------------------ X-hat image producer ------------------------------
+        // Its own thread: the image ring is released by the MMAs, the raw ring by the teams; one thread
+        // serving both would let the U loads run only one stage ahead.  The boxes of a stage go straight
+        // into its image stage, once the MMAs of the stage that used it last are done.
+        if (XIMG && lane == 0) {
+            for (int g = 0; g < my_stages && !abort_flag; ++g) {
+                const int l = g % NLO;
+                if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+                const uint32_t im = img0 + (uint32_t)l * IMG;
+                const size_t xoff = (size_t)(g_lo + g) * d * 32;          // one block of d features per stage
+                mbar_expect_tx(split(l), (uint32_t)(2 * XIMG_BYTES));
+                bulk_load_1d(im + 2 * UIMG, xT1 + xoff, (uint32_t)XIMG_BYTES, split(l));
+                bulk_load_1d(im + 2 * UIMG + XIMG_BYTES, xT2 + xoff, (uint32_t)XIMG_BYTES, split(l));
             }
         }
     } else if (warp == 1) {
@@ -190,7 +197,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 if (abort_flag) break;
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= 6 && warp < 6 + 4 * NTEAMS) {
         // ------------------------------ vector pass + split ------------------------------
         // A warp takes 8 consecutive data rows of a stage, a lane the columns lane + 32 j of U (scalar loads
         // from the plain FP32 rows: consecutive lanes, consecutive words).  NTEAMS teams of four warps take
@@ -348,7 +355,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
     float* sscr = reinterpret_cast<float*>(smem);             // [vector warps][128 columns]
-    if (warp >= 6) {
+    if (warp >= 6 && warp < 6 + 4 * NTEAMS) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + lane + 32 * k] = s_acc[k] * ldexpf(1.0f, -eU);
     }

@@ -376,7 +376,7 @@ constexpr int UIMG1 = 128 * 64;                // fp16 image of the U operand: 1
 constexpr int XIMG1 = 256 * 64;                // fp16 image of the X-hat operand: 256 features x 32 data rows
 constexpr int IMG1 = 2 * UIMG1 + 2 * XIMG1;    // U h1, U h2, X h1, X h2: 48 KB
 constexpr int FLUSH1 = 128;                    // stages per accumulation period (4096 rows)
-constexpr int NTH1 = (2 + 4 + 4 * NT1) * 32;   // producer, MMA issuer, 4 epilogue, 4 NT1 team warps
+constexpr int NTH1 = (2 + 4 + 4 * NT1 + 1) * 32;   // U producer, MMA issuer, 4 epilogue, 4 NT1 team warps, X-hat image producer
 
 __global__ void __launch_bounds__(NTH1, 1)
 k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ xT1,
@@ -439,11 +439,20 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
-                const int s = g % NRAW1, l = g % NIM1;
+                const int s = g % NRAW1;
                 const int row0 = (int)((g_lo + g) * TR1);
                 if (g >= NRAW1) mbar_wait_spin(ufree(s), ((g / NRAW1) - 1) & 1, &abort_flag, ctl);
                 mbar_expect_tx(ufull(s), URAW1);
                 tma_load_2d(raw0 + (uint32_t)s * URAW1, &tmU, c0, row0, ufull(s));
+            }
+        }
+    } else if (warp == 6 + 4 * NT1) {
+        // ------------------------------ X-hat image producer ------------------------------
+        // Its own thread: the image ring is released by the MMAs, the raw U ring by the teams; one thread
+        // serving both would let the U loads run only one stage ahead.
+        if (lane == 0) {
+            for (int g = 0; g < my_stages && !abort_flag; ++g) {
+                const int l = g % NIM1;
                 if (g >= NIM1) mbar_wait_spin(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
                 const uint32_t im = img0 + (uint32_t)l * IMG1;
                 const size_t xoff = ((size_t)(g_lo + g) * NNB + nb) * (256 * 32);      // this stage's box of the feature block
@@ -479,7 +488,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
                 if (abort_flag) break;
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= 6 && warp < 6 + 4 * NT1) {
         // ------------------------------ U teams: FP32 slice -> K-major fp16 images ------------------------------
         const int vw = warp - 6, team = vw >> 2, tw = vw & 3;
         const int tt = tw * 32 + lane;                     // column of the slice
