@@ -136,7 +136,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int s = g % NSR;
-                if (g >= NSR) mbar_wait_spin(rawfree(s), ((g / NSR) - 1) & 1, &abort_flag, ctl);
+                if (g >= NSR) mbar_wait_backoff(rawfree(s), ((g / NSR) - 1) & 1, &abort_flag, ctl);
                 const int64_t row0 = (g_lo + g) * TR;
                 const int rows = (n - row0 < TR) ? (int)(n - row0) : TR;
                 const uint32_t dst = raw0 + (uint32_t)s * STAGE;
@@ -158,7 +158,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
         if (XIMG && lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int l = g % NLO;
-                if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+                if (g >= NLO) mbar_wait_backoff(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
                 const uint32_t im = img0 + (uint32_t)l * IMG;
                 const size_t xoff = (size_t)(g_lo + g) * d * 32;          // one block of d features per stage
                 mbar_expect_tx(split(l), (uint32_t)(2 * XIMG_BYTES));
@@ -227,8 +227,8 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
             float yt_l = yt_next;
             yt_next = (g + NTEAMS < my_stages && owner && myrow + NTEAMS * TR < n) ? ytilde[myrow + NTEAMS * TR] : 0.f;
             float yb_l = 0.f;
-            mbar_wait_spin(full(s), (g / NSR) & 1, &abort_flag, ctl);
-            if (g >= NLO) mbar_wait_spin(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
+            mbar_wait_backoff(full(s), (g / NSR) & 1, &abort_flag, ctl);
+            if (g >= NLO) mbar_wait_backoff(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
             const uint32_t hi_s = raw0 + (uint32_t)s * STAGE, im = img0 + (uint32_t)l * IMG;
             const int rows_here = (n - srow0 < TR) ? (int)(n - srow0) : TR;
             float u[8][4], dot[8];

@@ -171,7 +171,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                 const int row0 = (int)(t * TILE_M);
                 for (int kb = 0; kb < KB; ++kb, ++g) {
                     const int s = (int)(g % NS);
-                    if (g >= NS) mbar_wait_spin(xfree(s), (uint32_t)((g / NS) - 1) & 1, &abort_flag, ctl);
+                    if (g >= NS) mbar_wait_backoff(xfree(s), (uint32_t)((g / NS) - 1) & 1, &abort_flag, ctl);
                     const uint32_t dst = stage0 + (uint32_t)s * STAGE;
                     const size_t boff = ((size_t)(kb * NCB + cb) * NBLK) * KC;
                     mbar_expect_tx(xfull(s), STAGE);
@@ -441,7 +441,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int s = g % NRAW1;
                 const int row0 = (int)((g_lo + g) * TR1);
-                if (g >= NRAW1) mbar_wait_spin(ufree(s), ((g / NRAW1) - 1) & 1, &abort_flag, ctl);
+                if (g >= NRAW1) mbar_wait_backoff(ufree(s), ((g / NRAW1) - 1) & 1, &abort_flag, ctl);
                 mbar_expect_tx(ufull(s), URAW1);
                 tma_load_2d(raw0 + (uint32_t)s * URAW1, &tmU, c0, row0, ufull(s));
             }
@@ -453,7 +453,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
                 const int l = g % NIM1;
-                if (g >= NIM1) mbar_wait_spin(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
+                if (g >= NIM1) mbar_wait_backoff(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
                 const uint32_t im = img0 + (uint32_t)l * IMG1;
                 const size_t xoff = ((size_t)(g_lo + g) * NNB + nb) * (256 * 32);      // this stage's box of the feature block
                 mbar_expect_tx(imgfull(l), 2 * XIMG1);
@@ -494,14 +494,14 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
         const int tt = tw * 32 + lane;                     // column of the slice
         for (int g = team; g < my_stages; g += NT1) {
             const int s = g % NRAW1, l = g % NIM1;
-            mbar_wait_spin(ufull(s), (g / NRAW1) & 1, &abort_flag, ctl);
+            mbar_wait_backoff(ufull(s), (g / NRAW1) & 1, &abort_flag, ctl);
             const uint32_t rs = raw0 + (uint32_t)s * URAW1;
             float uv[4][8];
 #pragma unroll
             for (int kg = 0; kg < 4; ++kg)
 #pragma unroll
                 for (int k = 0; k < 8; ++k) uv[kg][k] = lds32f(rs + (uint32_t)(((8 * kg + k) * 128 + tt) * 4));
-            if (g >= NIM1) mbar_wait_spin(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
+            if (g >= NIM1) mbar_wait_backoff(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
             const uint32_t im = img0 + (uint32_t)l * IMG1;
 #pragma unroll
             for (int kg = 0; kg < 4; ++kg) {

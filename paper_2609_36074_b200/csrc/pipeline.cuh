@@ -87,6 +87,29 @@ __device__ __forceinline__ void mbar_wait_spin(uint32_t bar, uint32_t parity, vo
     ctl->stopped = 1;
 }
 
+// Bounded wait by polling with a short sleep between polls: for roles that may wait long (a team waiting
+// for the MMAs to free an image stage, a producer waiting for a free slot).  A pure polling loop would
+// take issue slots from the single MMA-issuing thread on the same scheduler; the sleep (~100 ns) bounds
+// the extra hand-over latency.
+__device__ __forceinline__ void mbar_wait_backoff(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                  Ctl* ctl)
+{
+    if (*abort_flag) return;
+    for (uint32_t i = 0; i < (kSpinLimit << 2); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return;
+        __nanosleep(100);
+    }
+    *abort_flag = 1u;
+    ctl->status = GEM_NLR_E_TIMEOUT;
+    ctl->stopped = 1;
+}
+
 // Same bounded wait for roles that are not on the critical path of the tensor pipe: the hardware may
 // suspend the thread for up to ~1 us per attempt instead of letting it poll, so that waiting warps do not
 // take issue slots from the single thread that issues the MMAs on the same scheduler.
