@@ -79,8 +79,12 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
     const int STAGE = (URAW + (XIMG ? 0 : TR * d * 4) + 1023) / 1024 * 1024;
     const int XIMG_BYTES = d * 64;                 // one fp16 image of the X-hat operand: d features x 32 data rows
     const int IMG = 2 * UIMG + 2 * XIMG_BYTES;           // image stage: U h1, U h2, X h1, X h2
+    // d <= 128: the X-hat images h1 | h2 are used as one N = 2 d operand (2 MMAs per k-step, accumulator of 2 d
+    // columns whose halves the epilogue adds); else 3 MMAs per k-step into d columns
+    const bool wideB = d <= 128;
+    const int ACC = wideB ? 2 * d : d;             // TMEM columns per accumulator buffer
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < 2 * d) tmem_cols <<= 1;
+    while ((int)tmem_cols < 2 * ACC) tmem_cols <<= 1;
 
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t raw0 = smem_base;                                   // NSR raw stages
@@ -169,7 +173,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f16(128, d, 0, 0);
+            const uint32_t idesc = umma_idesc_f16(128, d, 0, 0), idesc2 = umma_idesc_f16(128, 2 * d, 0, 0);
             // The wait for the next stage sits between the two k-steps of the current one, so the tensor pipe
             // has MMAs queued while this thread polls.
             if (my_stages > 0) mbar_wait_spin(split(0), 0, &abort_flag, ctl);
@@ -179,17 +183,19 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
             for (int g = 0; g < my_stages; ++g) {
                 if (in_period == 0 && period >= 2) mbar_wait_spin(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
                 tc_fence_after();
-                const uint32_t tacc = tmem_base + (uint32_t)(a * d);
+                const uint32_t tacc = tmem_base + (uint32_t)(a * ACC);
                 const uint32_t im = img0 + (uint32_t)l * IMG;
                 // A = U images (M = 128 columns), B = X-hat images (N = d features), K-major; a k-step of 16 data
                 // rows (32 bytes inside the 64-byte swizzled row) advances the start address by 2
                 const uint64_t da1 = umma_desc_k_sw64(im), da2 = umma_desc_k_sw64(im + UIMG);
                 const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG), db2 = umma_desc_k_sw64(im + 2 * UIMG + XIMG_BYTES);
-                umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
+                if (wideB) umma_f16_x2(tacc, da1, da2, db1, idesc2, idesc, in_period ? 1u : 0u);
+                else umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
                 int ln = l + 1, lphn = lph;
                 if (ln == NLO) { ln = 0; lphn ^= 1; }
                 if (g + 1 < my_stages) mbar_wait_spin(split(ln), (uint32_t)lphn, &abort_flag, ctl);
-                umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
+                if (wideB) umma_f16_x2(tacc, da1 + 2, da2 + 2, db1 + 2, idesc2, idesc, 1u);
+                else umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
                 umma_commit(lofree(l));
                 if (in_period == FLUSH - 1 || g == my_stages - 1) umma_commit(accfull(a));
                 l = ln; lph = lphn;
@@ -335,7 +341,13 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
             tc_fence_after();
             for (int c = 0; c * 16 < d; ++c) {
                 float v[16];
-                tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * d + c * 16), v);
+                tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * ACC + c * 16), v);
+                if (wideB) {            // second half of the accumulator: the h1 h2' products
+                    float v2[16];
+                    tmem_ld16(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * ACC + d + c * 16), v2);
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) v[k] += v2[k];
+                }
                 if (j < r) {
                     double* o = out + (size_t)(c * 16) * r + j;
 #pragma unroll

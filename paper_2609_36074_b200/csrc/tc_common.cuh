@@ -211,6 +211,23 @@ __device__ __forceinline__ void umma_f16_x3(uint32_t tmem_d, uint64_t a1, uint64
         : "memory");
 }
 
+// Two MMAs of one k-step when the B images h1 | h2 are contiguous (N = 2 n): D[:, 0..2n) (+)= A1 [B1 | B2],
+// then D[:, 0..n) += A2 B1.  Columns 0..n-1 collect h1 h1' + h2 h1', columns n..2n-1 collect h1 h2'; the
+// reader of the accumulator adds the two halves.  One MMA instruction fewer per k-step: an instruction costs
+// the issuing thread ~130 cycles whatever its N, which is what bounds narrow tiles.
+__device__ __forceinline__ void umma_f16_x2(uint32_t tmem_d, uint64_t a1, uint64_t a2, uint64_t b12, uint32_t idesc_2n,
+                                            uint32_t idesc_n, uint32_t accumulate_first)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, t;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "setp.eq.b32 t, %7, %7;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %3, %4, {%7, %7, %7, %7}, p;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %3, %5, {%7, %7, %7, %7}, t;\n\t}"
+        ::"r"(tmem_d), "l"(a1), "l"(a2), "l"(b12), "r"(idesc_2n), "r"(idesc_n), "r"(accumulate_first), "r"(0u)
+        : "memory");
+}
+
 // Eight scaled values (consecutive data rows of one column) -> the two fp16 chunks h1, h2 (16 bytes each).
 __device__ __forceinline__ void split_h8(const float* v, uint4& h1, uint4& h2)
 {
