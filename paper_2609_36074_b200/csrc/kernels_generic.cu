@@ -75,16 +75,17 @@ k_rowvec(float* __restrict__ U, float* __restrict__ ytilde, float* __restrict__ 
     }
 }
 
-// Vector pass for wide factors (128 < r <= 1024, r a multiple of 4): one warp per row, all of the
-// row's 16-byte pieces requested at once (up to 8 per lane), s accumulated in FP32 over 16 rows and
-// then folded into per-warp FP64 sums.  Same outputs as k_rowvec.
+// Vector pass for factors with 32 < r <= 1024, r a multiple of 4: a warp takes 8 / NK rows at a time, a lane
+// NK 16-byte pieces of each (NK = 1, 2, 4, 8 for r <= 128, 256, 512, 1024), all requested at once; s is
+// accumulated in FP32 over 16 rows and then folded into per-warp FP64 sums.  Same outputs as k_rowvec.
 constexpr int RVW_WARPS = 8;
-template <bool MATERIALIZE>
+template <bool MATERIALIZE, int NK>
 __global__ void __launch_bounds__(RVW_WARPS * 32)
 k_rowvec_wide(float* __restrict__ U, float* __restrict__ ytilde, float* __restrict__ ybar,
               const Ctl* __restrict__ ctl, const float* __restrict__ p, int64_t n, int r, double gamma,
               double* __restrict__ part, int ignore_stop)
 {
+    constexpr int ROWS = 8 / NK;
     if (!ignore_stop && ctl->stopped) return;
     extern __shared__ double sm_s[];              // [RVW_WARPS][r]
     __shared__ double sm_red[2][RVW_WARPS];
@@ -94,16 +95,16 @@ k_rowvec_wide(float* __restrict__ U, float* __restrict__ ytilde, float* __restri
     const int r4 = r >> 2;
     double* my_s = sm_s + (size_t)warp * r;
     for (int j = lane; j < r; j += 32) my_s[j] = 0.0;
-    float4 p4[8], sacc[8];
+    float4 p4[NK], sacc[NK];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+    for (int k = 0; k < NK; ++k) {
         const int c4 = lane + 32 * k;
         p4[k] = (c4 < r4) ? reinterpret_cast<const float4*>(p)[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
         sacc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     auto flush = [&]() {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < NK; ++k) {
             const int c4 = lane + 32 * k;
             if (c4 < r4) {
                 double* o = my_s + 4 * c4;
@@ -114,40 +115,50 @@ k_rowvec_wide(float* __restrict__ U, float* __restrict__ ytilde, float* __restri
     };
     double qq = 0.0, yq = 0.0;
     int since = 0;
-    const int64_t stride = (int64_t)gridDim.x * RVW_WARPS;
-    for (int64_t row = (int64_t)blockIdx.x * RVW_WARPS + warp; row < n; row += stride) {
-        float4* urow = reinterpret_cast<float4*>(U + row * r);
-        float4 u[8];
+    const int64_t stride = (int64_t)gridDim.x * RVW_WARPS * ROWS;
+    for (int64_t row0 = ((int64_t)blockIdx.x * RVW_WARPS + warp) * ROWS; row0 < n; row0 += stride) {
+        float4 u[ROWS][NK];
+        float yt[ROWS];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int c4 = lane + 32 * k;
-            u[k] = (c4 < r4) ? __ldcs(urow + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        float yt = ytilde[row];
-        float acc = 0.f;
+        for (int i = 0; i < ROWS; ++i) {           // rows beyond n and pieces beyond r read as zero
+            const float4* urow = reinterpret_cast<const float4*>(U + (row0 + i) * r);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            u[k].x *= cf; u[k].y *= cf; u[k].z *= cf; u[k].w *= cf;
-            acc = fmaf(u[k].x, p4[k].x, acc); acc = fmaf(u[k].y, p4[k].y, acc);
-            acc = fmaf(u[k].z, p4[k].z, acc); acc = fmaf(u[k].w, p4[k].w, acc);
-        }
-        acc = warp_sum(acc);
-        const float q = acc - 1.0f;
-        if (dual) yt = (float)((double)yt + gamma * (double)q);
-        const float yb = (float)((double)yt + gamma * (double)q);
-        if (lane == 0) {
-            if (dual) ytilde[row] = yt;
-            ybar[row] = yb;
-            qq += (double)q * (double)q;
-            yq += (double)yt * (double)q;
+            for (int k = 0; k < NK; ++k) {
+                const int c4 = lane + 32 * k;
+                u[i][k] = (c4 < r4 && row0 + i < n) ? __ldcs(urow + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            yt[i] = (row0 + i < n) ? ytilde[row0 + i] : 0.f;
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            sacc[k].x = fmaf(u[k].x, yb, sacc[k].x); sacc[k].y = fmaf(u[k].y, yb, sacc[k].y);
-            sacc[k].z = fmaf(u[k].z, yb, sacc[k].z); sacc[k].w = fmaf(u[k].w, yb, sacc[k].w);
-            if (MATERIALIZE && lane + 32 * k < r4) urow[lane + 32 * k] = u[k];
+        for (int i = 0; i < ROWS; ++i) {
+            float acc = 0.f;
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                u[i][k].x *= cf; u[i][k].y *= cf; u[i][k].z *= cf; u[i][k].w *= cf;
+                acc = fmaf(u[i][k].x, p4[k].x, acc); acc = fmaf(u[i][k].y, p4[k].y, acc);
+                acc = fmaf(u[i][k].z, p4[k].z, acc); acc = fmaf(u[i][k].w, p4[k].w, acc);
+            }
+            acc = warp_sum(acc);
+            const float q = acc - 1.0f;
+            float y = yt[i];
+            if (dual) y = (float)((double)y + gamma * (double)q);
+            const float yb = (float)((double)y + gamma * (double)q);
+            if (lane == 0 && row0 + i < n) {
+                if (dual) ytilde[row0 + i] = y;
+                ybar[row0 + i] = yb;
+                qq += (double)q * (double)q;
+                yq += (double)y * (double)q;
+            }
+            float4* urow = reinterpret_cast<float4*>(U + (row0 + i) * r);
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                sacc[k].x = fmaf(u[i][k].x, yb, sacc[k].x); sacc[k].y = fmaf(u[i][k].y, yb, sacc[k].y);
+                sacc[k].z = fmaf(u[i][k].z, yb, sacc[k].z); sacc[k].w = fmaf(u[i][k].w, yb, sacc[k].w);
+                if (MATERIALIZE && lane + 32 * k < r4 && row0 + i < n) urow[lane + 32 * k] = u[i][k];
+            }
         }
-        if (++since == 16) { flush(); since = 0; }
+        since += ROWS;
+        if (since >= 16) { flush(); since = 0; }
     }
     flush();
     if (lane == 0) { sm_red[0][warp] = qq; sm_red[1][warp] = yq; }
@@ -163,6 +174,48 @@ k_rowvec_wide(float* __restrict__ U, float* __restrict__ ytilde, float* __restri
         for (int w = 0; w < RVW_WARPS; ++w) { a += sm_red[0][w]; b += sm_red[1][w]; }
         out[r] = a;
         out[r + 1] = b;
+    }
+}
+
+// Column sums of c_f * U for 32 < r <= 1024, r a multiple of 4: the block sweeps groups of 256 / (r / 4) rows,
+// thread t owning the 16-byte piece t % (r / 4) of row t / (r / 4) of each group (so a group is one contiguous
+// span and a thread always meets the same four columns), eight groups requested at once, FP64 sums in
+// registers.  part[blockIdx][0..r-1].
+__global__ void __launch_bounds__(256)
+k_colsum_vec(const float* __restrict__ U, const Ctl* __restrict__ ctl, int64_t n, int r, double* __restrict__ part)
+{
+    __shared__ double sm[1024];                   // [rows of a group][r]
+    const int r4 = r >> 2;
+    const int per = 256 / r4;                     // rows of a group
+    const int t = threadIdx.x;
+    const bool active = t < per * r4;
+    const int my_row = t / r4;
+    const float cf = ctl->c_f;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    const float4* U4 = reinterpret_cast<const float4*>(U);
+    for (int64_t g0 = (int64_t)blockIdx.x * 8; g0 * per < n; g0 += (int64_t)gridDim.x * 8) {
+        float4 w[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int64_t row = (g0 + k) * per + my_row;
+            w[k] = (active && row < n) ? __ldcs(U4 + (g0 + k) * per * r4 + t) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            acc[0] += (double)(cf * w[k].x); acc[1] += (double)(cf * w[k].y);
+            acc[2] += (double)(cf * w[k].z); acc[3] += (double)(cf * w[k].w);
+        }
+    }
+    if (active) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) sm[4 * t + c] = acc[c];      // = sm[my_row][4 (t % r4) + c]
+    }
+    __syncthreads();
+    double* out = part + (size_t)blockIdx.x * (r + 2);
+    for (int j = t; j < r; j += 256) {
+        double v = 0.0;
+        for (int i = 0; i < per; ++i) v += sm[i * r + j];
+        out[j] = v;
     }
 }
 
@@ -651,13 +704,29 @@ static int small_grid(const Problem& pb)
     return (int)(g < 1 ? 1 : g);
 }
 
-static bool wide_r(int r) { return r > 128 && r <= 1024 && r % 4 == 0; }
+static bool wide_r(int r) { return r > 32 && r <= 1024 && r % 4 == 0; }
+static int wide_nk(int r) { return r <= 128 ? 1 : r <= 256 ? 2 : r <= 512 ? 4 : 8; }
 static int wide_grid(const Problem& pb)
 {
-    int64_t g = (pb.P.n + RVW_WARPS - 1) / RVW_WARPS;
+    const int rows_per = RVW_WARPS * (8 / wide_nk(pb.P.r));
+    int64_t g = (pb.P.n + rows_per - 1) / rows_per;
     const int cap = pb.L.gv < kSMs * 2 ? pb.L.gv : kSMs * 2;
     if (g > cap) g = cap;
     return (int)(g < 1 ? 1 : g);
+}
+
+template <bool MAT, int NK>
+static void launch_rowvec_wide(const Problem& pb, int grid, int ignore_stop)
+{
+    const auto& P = pb.P;
+    const size_t sm = sizeof(double) * RVW_WARPS * (size_t)P.r;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_rowvec_wide<MAT, NK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * 8);
+        attr_set = true;
+    }
+    k_rowvec_wide<MAT, NK><<<grid, RVW_WARPS * 32, sm, pb.stream>>>(
+        pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
 }
 
 template <bool MAT>
@@ -683,19 +752,10 @@ static int launch_rowvec(const Problem& pb, bool materialize, int ignore_stop)
     }
     if (wide_r(P.r)) {
         const int grid = wide_grid(pb);
-        const size_t sm = sizeof(double) * RVW_WARPS * (size_t)P.r;
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaFuncSetAttribute(k_rowvec_wide<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * 8);
-            cudaFuncSetAttribute(k_rowvec_wide<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * 8);
-            attr_set = true;
-        }
-        if (materialize)
-            k_rowvec_wide<true><<<grid, RVW_WARPS * 32, sm, pb.stream>>>(
-                pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
-        else
-            k_rowvec_wide<false><<<grid, RVW_WARPS * 32, sm, pb.stream>>>(
-                pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), P.n, P.r, pb.gamma, pb.part1v(), ignore_stop);
+        const int nk = wide_nk(P.r);
+#define RVW_CASE(NK) case NK: if (materialize) launch_rowvec_wide<true, NK>(pb, grid, ignore_stop); else launch_rowvec_wide<false, NK>(pb, grid, ignore_stop); break;
+        switch (nk) { RVW_CASE(1) RVW_CASE(2) RVW_CASE(4) RVW_CASE(8) default: break; }
+#undef RVW_CASE
         pb.count();
         return grid;
     }
@@ -721,6 +781,9 @@ void launch_init_colsum(const Problem& pb)
 #define CS_CASE(R4) case R4: k_colsum_small<R4><<<grid, 256, 0, pb.stream>>>(pb.U, pb.ctl(), P.n, pb.part1v()); break;
         switch (P.r / 4) { CS_CASE(1) CS_CASE(2) CS_CASE(3) CS_CASE(4) CS_CASE(5) CS_CASE(6) CS_CASE(7) CS_CASE(8) default: break; }
 #undef CS_CASE
+    } else if (wide_r(P.r)) {
+        grid = pb.L.gv < kSMs * 4 ? pb.L.gv : kSMs * 4;
+        k_colsum_vec<<<grid, 256, 0, pb.stream>>>(pb.U, pb.ctl(), P.n, P.r, pb.part1v());
     } else {
         set_rv_attr(P.r);
         k_colsum<<<grid, RV_WARPS * 32, rv_smem(P.r), pb.stream>>>(pb.U, pb.ctl(), P.n, P.r, pb.part1v());
