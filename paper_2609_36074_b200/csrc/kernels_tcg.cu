@@ -20,7 +20,8 @@
 //   warp 1       MMA issuer: per chunk 2 k-steps x 3 products; commits free the stage
 //   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); accumulators read in the 16x256b
 //                fragment layout, old U entries straight from global memory (every 4-lane group reads and
-//                writes one 32-byte sector of a row), FP64 statistics; column sums by warp shuffles,
+//                writes one 32-byte sector of a row), requested two 16-column groups ahead; statistics in
+//                FP32 over a thread's 16 entries of a group, then FP64; column sums by warp shuffles,
 //                combined across the four quarters in fixed order
 // Every mbarrier wait is bounded (error status GEM_NLR_E_TIMEOUT, kernel runs to its end, TMEM freed).
 #include "nlr_common.cuh"
@@ -222,6 +223,29 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         const int half = (warp - 2) >> 2;
         const int g4 = lane >> 2, tq = lane & 3;
         const int et = (warp - 2) * 32 + lane;            // 0..255 among the epilogue threads
+        // The old entries of U do not depend on the accumulator: they are requested two 16-column groups
+        // ahead (across item boundaries too), so their DRAM latency is off the epilogue's critical path.
+        // Group index c = 8 (item ordinal) + jj.
+        const int64_t my_items = (n_items > blockIdx.x) ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+        auto request = [&](int64_t c, float2 (&dst)[4][2]) {
+            const int64_t w = blockIdx.x + (c >> 3) * gridDim.x;
+            const bool in = (c >> 3) < my_items;
+            const int64_t t = w / NCB;
+            const int col0 = (int)(w % NCB) * NBLK + half * 128 + (int)(c & 7) * 16;
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                    const int cc = col0 + 8 * b + 2 * tq;
+                    dst[x][b] = (in && row < n && cc < r) ? __ldcs(reinterpret_cast<const float2*>(U + row * (int64_t)r + cc))
+                                                          : make_float2(0.f, 0.f);
+                }
+            }
+        };
+        float2 wq0[4][2], wq1[4][2];
+        request(0, wq0);
+        request(1, wq1);
         int i = 0;
         for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
             const int a = i & 1;
@@ -252,13 +276,11 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
 #pragma unroll
                 for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int b = 0; b < 2; ++b) {
-                        const int c = col0 + 8 * b + 2 * tq;
-                        wold[x][b] = (valid[x] && c < r) ? __ldcs(reinterpret_cast<const float2*>(urow[x] + c))
-                                                         : make_float2(0.f, 0.f);
-                    }
+                    for (int b = 0; b < 2; ++b) { wold[x][b] = wq0[x][b]; wq0[x][b] = wq1[x][b]; }
+                request((int64_t)i * 8 + jj + 2, wq1);
                 tmem_ld_wait();
                 float cs[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+                float fa = 0.f, fb = 0.f, fh = 0.f;     // FP32 over the thread's 16 entries of the group, then FP64
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
                     const int c = col0 + 8 * b + 2 * tq;
@@ -274,13 +296,13 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                         v0 = fmaf(nay[x], p2.x, v0); v1 = fmaf(nay[x], p2.y, v1);
                         v0 -= s2.x; v1 -= s2.y;
                         const float w0 = live ? fmaxf(v0, 0.f) : 0.f, w1 = live ? fmaxf(v1, 0.f) : 0.f;
-                        const double wd0 = (double)w0, ud0 = (double)u0, wd1 = (double)w1, ud1 = (double)u1;
-                        sa = fma(wd0, wd0, sa); sb = fma(ud0, ud0, sb); sh = fma(wd0, ud0, sh);
-                        sa = fma(wd1, wd1, sa); sb = fma(ud1, ud1, sb); sh = fma(wd1, ud1, sh);
+                        fa = fmaf(w0, w0, fa); fb = fmaf(u0, u0, fb); fh = fmaf(w0, u0, fh);
+                        fa = fmaf(w1, w1, fa); fb = fmaf(u1, u1, fb); fh = fmaf(w1, u1, fh);
                         cs[b][0] += w0; cs[b][1] += w1;
                         if (live) *reinterpret_cast<float2*>(urow[x] + c) = make_float2(w0, w1);
                     }
                 }
+                sa += (double)fa; sb += (double)fb; sh += (double)fh;
                 // column sums over the 32 rows of the quarter: the 8 row groups g4 of the warp
 #pragma unroll
                 for (int b = 0; b < 2; ++b)
