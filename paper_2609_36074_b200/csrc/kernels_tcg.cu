@@ -19,8 +19,9 @@
 //   warp 0       producer (TMA / bulk copies, 4-stage ring)
 //   warp 1       MMA issuer: per chunk 2 k-steps x 3 products; commits free the stage
 //   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); accumulators read in the 16x256b
-//                fragment layout, old U entries straight from global memory (every 4-lane group reads and
-//                writes one 32-byte sector of a row), requested two 16-column groups ahead; statistics in
+//                fragment layout and swapped between neighbouring lanes so that a thread owns 4 consecutive
+//                columns; old U entries straight from global memory (every 4-lane group reads and writes 64
+//                contiguous bytes of a row), requested two 16-column groups ahead; statistics in
 //                FP32 over a thread's 16 entries of a group, then FP64; column sums by warp shuffles,
 //                combined across the four quarters in fixed order
 // Every mbarrier wait is bounded (error status GEM_NLR_E_TIMEOUT, kernel runs to its end, TMEM freed).
@@ -226,24 +227,27 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         // The old entries of U do not depend on the accumulator: they are requested two 16-column groups
         // ahead (across item boundaries too), so their DRAM latency is off the epilogue's critical path.
         // Group index c = 8 (item ordinal) + jj.
+        // Neighbouring lanes (tq ^ 1) swap half of their accumulator fragment, so that a thread owns four
+        // consecutive columns of each of its rows: columns cbase .. cbase + 3 of the 16-column group with
+        // cbase = 0, 8, 4, 12 for tq = 0, 1, 2, 3.  A 4-lane group then reads and writes 64 contiguous bytes of
+        // a row with one 16-byte access per lane: half as many memory instructions (and passes through the L1
+        // pipeline, which the tensor core's operand fetches share) as with the raw fragment's 8-byte pairs.
+        const bool odd = tq & 1;
+        const int cbase = 4 * (tq >> 1) + 8 * (tq & 1);
         const int64_t my_items = (n_items > blockIdx.x) ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-        auto request = [&](int64_t c, float2 (&dst)[4][2]) {
+        auto request = [&](int64_t c, float4 (&dst)[4]) {
             const int64_t w = blockIdx.x + (c >> 3) * gridDim.x;
             const bool in = (c >> 3) < my_items;
             const int64_t t = w / NCB;
-            const int col0 = (int)(w % NCB) * NBLK + half * 128 + (int)(c & 7) * 16;
+            const int cc = (int)(w % NCB) * NBLK + half * 128 + (int)(c & 7) * 16 + cbase;
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
-#pragma unroll
-                for (int b = 0; b < 2; ++b) {
-                    const int cc = col0 + 8 * b + 2 * tq;
-                    dst[x][b] = (in && row < n && cc < r) ? __ldcs(reinterpret_cast<const float2*>(U + row * (int64_t)r + cc))
-                                                          : make_float2(0.f, 0.f);
-                }
+                dst[x] = (in && row < n && cc < r) ? __ldcs(reinterpret_cast<const float4*>(U + row * (int64_t)r + cc))
+                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         };
-        float2 wq0[4][2], wq1[4][2];
+        float4 wq0[4], wq1[4];
         request(0, wq0);
         request(1, wq1);
         int i = 0;
@@ -266,54 +270,56 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
             tc_fence_after();
 #pragma unroll 1
             for (int jj = 0; jj < 8; ++jj) {
-                const int col0 = cb * NBLK + half * 128 + jj * 16;
+                const int c = cb * NBLK + half * 128 + jj * 16 + cbase;      // this thread's four columns
                 // acc[x2][...]: x2 = 0: rows g4, g4 + 8; x2 = 1: rows g4 + 16, g4 + 24
                 float acc[2][8];
                 const uint32_t tcol = (uint32_t)(a * NBLK + half * 128 + jj * 16);
                 tmem_ld_16x256b_x2(tmem_base + ((uint32_t)(q * 32) << 16) + tcol, acc[0]);
                 tmem_ld_16x256b_x2(tmem_base + ((uint32_t)(q * 32 + 16) << 16) + tcol, acc[1]);
-                float2 wold[4][2];
+                float4 wold[4];
 #pragma unroll
-                for (int x = 0; x < 4; ++x)
-#pragma unroll
-                    for (int b = 0; b < 2; ++b) { wold[x][b] = wq0[x][b]; wq0[x][b] = wq1[x][b]; }
+                for (int x = 0; x < 4; ++x) { wold[x] = wq0[x]; wq0[x] = wq1[x]; }
                 request((int64_t)i * 8 + jj + 2, wq1);
+                const float4 p4 = *reinterpret_cast<const float4*>(sp + c);
+                const float4 s4 = *reinterpret_cast<const float4*>(sas + c);
+                const bool cok = c < r;
                 tmem_ld_wait();
-                float cs[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+                float cs[4] = {0.f, 0.f, 0.f, 0.f};
                 float fa = 0.f, fb = 0.f, fh = 0.f;     // FP32 over the thread's 16 entries of the group, then FP64
 #pragma unroll
-                for (int b = 0; b < 2; ++b) {
-                    const int c = col0 + 8 * b + 2 * tq;
-                    const float2 p2 = *reinterpret_cast<const float2*>(sp + c);
-                    const float2 s2 = *reinterpret_cast<const float2*>(sas + c);
+                for (int x = 0; x < 4; ++x) {
+                    // row g4 + 8 x: registers 4 b + 2 (x & 1) + {0, 1} of load x >> 1 hold columns 8 b + 2 tq + {0, 1}
+                    const float b0x = acc[x >> 1][2 * (x & 1)], b0y = acc[x >> 1][2 * (x & 1) + 1];
+                    const float b1x = acc[x >> 1][4 + 2 * (x & 1)], b1y = acc[x >> 1][4 + 2 * (x & 1) + 1];
+                    const float rx = __shfl_xor_sync(0xffffffffu, odd ? b0x : b1x, 1);
+                    const float ry = __shfl_xor_sync(0xffffffffu, odd ? b0y : b1y, 1);
+                    const float av[4] = {odd ? rx : b0x, odd ? ry : b0y, odd ? b1x : rx, odd ? b1y : ry};
+                    const float uw[4] = {wold[x].x, wold[x].y, wold[x].z, wold[x].w};
+                    const float pv[4] = {p4.x, p4.y, p4.z, p4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w};
+                    const bool live = valid[x] && cok;
+                    float wv[4];
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const bool live = valid[x] && c < r;
-                        // rows g4 + 8 x: x = 0, 1 from the first load (registers 4b + 0..1 / 4b + 2..3), x = 2, 3 from the second
-                        const float a0 = acc[x >> 1][4 * b + 2 * (x & 1)], a1 = acc[x >> 1][4 * b + 2 * (x & 1) + 1];
-                        const float u0 = live ? cf * wold[x][b].x : 0.f, u1 = live ? cf * wold[x][b].y : 0.f;
-                        float v0 = fmaf(two_alpha, a0, u0), v1 = fmaf(two_alpha, a1, u1);
-                        v0 = fmaf(nay[x], p2.x, v0); v1 = fmaf(nay[x], p2.y, v1);
-                        v0 -= s2.x; v1 -= s2.y;
-                        const float w0 = live ? fmaxf(v0, 0.f) : 0.f, w1 = live ? fmaxf(v1, 0.f) : 0.f;
-                        fa = fmaf(w0, w0, fa); fb = fmaf(u0, u0, fb); fh = fmaf(w0, u0, fh);
-                        fa = fmaf(w1, w1, fa); fb = fmaf(u1, u1, fb); fh = fmaf(w1, u1, fh);
-                        cs[b][0] += w0; cs[b][1] += w1;
-                        if (live) *reinterpret_cast<float2*>(urow[x] + c) = make_float2(w0, w1);
+                    for (int e = 0; e < 4; ++e) {
+                        const float u = live ? cf * uw[e] : 0.f;
+                        float v = fmaf(two_alpha, av[e], u);
+                        v = fmaf(nay[x], pv[e], v);
+                        v -= sv[e];
+                        wv[e] = live ? fmaxf(v, 0.f) : 0.f;
+                        fa = fmaf(wv[e], wv[e], fa); fb = fmaf(u, u, fb); fh = fmaf(wv[e], u, fh);
+                        cs[e] += wv[e];
                     }
+                    if (live) *reinterpret_cast<float4*>(urow[x] + c) = make_float4(wv[0], wv[1], wv[2], wv[3]);
                 }
                 sa += (double)fa; sb += (double)fb; sh += (double)fh;
                 // column sums over the 32 rows of the quarter: the 8 row groups g4 of the warp
 #pragma unroll
-                for (int b = 0; b < 2; ++b)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        float v = cs[b][e];
-                        v += __shfl_xor_sync(0xffffffffu, v, 4);
-                        v += __shfl_xor_sync(0xffffffffu, v, 8);
-                        v += __shfl_xor_sync(0xffffffffu, v, 16);
-                        if (lane < 4) my_tmp[jj * 16 + 8 * b + 2 * tq + e] = v;
-                    }
+                for (int e = 0; e < 4; ++e) {
+                    float v = cs[e];
+                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                    if (lane < 4) my_tmp[jj * 16 + cbase + e] = v;
+                }
             }
             tc_fence_before();
             __syncwarp();
