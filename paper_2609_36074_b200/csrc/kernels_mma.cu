@@ -351,8 +351,8 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
             float2 w0[NT], w1[NT];
 #pragma unroll
             for (int nn = 0; nn < NT; ++nn) {
-                w0[nn] = v0 ? __ldcs(reinterpret_cast<const float2*>(U + row0 * R + 8 * nn + 2 * tq)) : make_float2(0.f, 0.f);
-                w1[nn] = v1 ? __ldcs(reinterpret_cast<const float2*>(U + row1 * R + 8 * nn + 2 * tq)) : make_float2(0.f, 0.f);
+                w0[nn] = v0 ? __ldcg(reinterpret_cast<const float2*>(U + row0 * R + 8 * nn + 2 * tq)) : make_float2(0.f, 0.f);
+                w1[nn] = v1 ? __ldcg(reinterpret_cast<const float2*>(U + row1 * R + 8 * nn + 2 * tq)) : make_float2(0.f, 0.f);
             }
             const float yb0 = v0 ? ybar[row0] : 0.f;
             const float yb1 = v1 ? ybar[row1] : 0.f;
@@ -406,8 +406,8 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
                     csum[nn][k & 1] += wd;
                     wn[k] = w;
                 }
-                if (v0) *reinterpret_cast<float2*>(U + row0 * R + 8 * nn + 2 * tq) = make_float2(wn[0], wn[1]);
-                if (v1) *reinterpret_cast<float2*>(U + row1 * R + 8 * nn + 2 * tq) = make_float2(wn[2], wn[3]);
+                if (v0) __stcg(reinterpret_cast<float2*>(U + row0 * R + 8 * nn + 2 * tq), make_float2(wn[0], wn[1]));
+                if (v1) __stcg(reinterpret_cast<float2*>(U + row1 * R + 8 * nn + 2 * tq), make_float2(wn[2], wn[3]));
             }
         }
     }

@@ -243,7 +243,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
-                dst[x] = (in && row < n && cc < r) ? __ldcs(reinterpret_cast<const float4*>(U + row * (int64_t)r + cc))
+                dst[x] = (in && row < n && cc < r) ? __ldcg(reinterpret_cast<const float4*>(U + row * (int64_t)r + cc))
                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         };
@@ -308,7 +308,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                         fa = fmaf(wv[e], wv[e], fa); fb = fmaf(u, u, fb); fh = fmaf(wv[e], u, fh);
                         cs[e] += wv[e];
                     }
-                    if (live) *reinterpret_cast<float4*>(urow[x] + c) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+                    if (live) __stcg(reinterpret_cast<float4*>(urow[x] + c), make_float4(wv[0], wv[1], wv[2], wv[3]));
                 }
                 sa += (double)fa; sb += (double)fb; sh += (double)fh;
                 // column sums over the 32 rows of the quarter: the 8 row groups g4 of the warp
