@@ -47,7 +47,7 @@ def _peaks():
 NCU_TRAFFIC_BYTES = {
     (1_000_000, 128, 16, "mma.tf32x3"): 640.0e6,
     (10_000_000, 64, 100, "f16x3"): 10.36e9,
-    (2_000_000, 768, 1000, "f16x3.tiled"): 22.96e9,
+    (2_000_000, 768, 1000, "f16x3.tiled"): 21.52e9,
     (100_000_000, 32, 8, "ffma"): 19.49e9,
 }
 
