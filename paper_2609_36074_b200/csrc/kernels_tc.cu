@@ -313,6 +313,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 mbar_wait(ufull(sl), (h / NUP) & 1, &abort_flag, ctl);
 #pragma unroll 1
                 for (int hf = 0; hf < PW / 16; ++hf) {
+                    if (pn * PW + hf * 16 >= r) break;       // columns beyond r: nothing to compute, TMA clips the store
                     float acc[16], wn[16];
                     tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * ACC_COLS + pn * PW + hf * 16), acc);
                     // Statistics of these 16 entries in FP32 (w >= 0, u >= 0: no cancellation), folded into the
@@ -322,6 +323,10 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     for (int cc = 0; cc < 4; ++cc) {
                         const int c = hf * 4 + cc;
                         const int col0 = pn * PW + 4 * c;
+                        if (col0 >= r) {                     // r is a multiple of 4: the whole quad is beyond r
+                            wn[4 * cc] = wn[4 * cc + 1] = wn[4 * cc + 2] = wn[4 * cc + 3] = 0.f;
+                            continue;
+                        }
                         const uint32_t addr = (PW == 32) ? pan + (uint32_t)rl * 128 + (uint32_t)((c ^ (rl & 7)) << 4)
                                                          : pan + (uint32_t)rl * 64 + (uint32_t)(c << 4);
                         const float4 w4 = lds128(addr);
