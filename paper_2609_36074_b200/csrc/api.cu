@@ -39,7 +39,13 @@ Layout make_layout(const gem_nlr_params& P)
     L.g2y = (int)ceil_div(r, G2_RT);
     L.g2x = clampi(ceil_div(kSMs * 4, L.g2y), 1, ceil_div(n, G2_TM));
     L.gs = clampi(ceil_div(n, 8), 1, kSMs * 4);
-    L.nred1 = (int)ceil_div((int64_t)d * r, 64);
+    // tcgen05 shapes: X-hat is static, so its two-term fp16 split is built once (below).  Those kernels see the
+    // feature count rounded up to a multiple of 32 (zero features in the images), so Theta, its partial records
+    // and the reduction are sized for dp x r.
+    const bool tc_images = (P.precision == -1 || P.precision == 1) && r >= 32 && n >= 4096;
+    const int dp = tc_images ? (d + 31) / 32 * 32 : d;
+    L.dp = dp;
+    L.nred1 = (int)ceil_div((int64_t)dp * r, 64);
 
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -47,30 +53,29 @@ Layout make_layout(const gem_nlr_params& P)
     L.p = take(sizeof(float) * r);
     L.s = take(sizeof(float) * r);
     L.alpha_s = take(sizeof(float) * r);
-    L.theta = take(sizeof(float) * (size_t)d * r);
+    L.theta = take(sizeof(float) * (size_t)dp * r);
     L.thimg = take(sizeof(float) * 2 * (size_t)((d + 31) / 32 * 32) * (r > 256 ? (r + 255) / 256 * 256 : (r + 15) / 16 * 16));
     L.ytilde = take(sizeof(float) * (size_t)n);
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families
-    size_t p1 = sizeof(double) * (size_t)(L.g1x > 8 || r <= 256 ? L.g1x : 8) * d * r;   // r > 256: up to 8 row ranges of the tiled tcgen05 first product
-    size_t p1_fast = ((size_t)d * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)d * r + r + 4) : 0;
+    size_t p1 = sizeof(double) * (size_t)(L.g1x > 8 || !tc_images ? L.g1x : 8) * dp * r;   // r > 256: up to 8 row ranges of the tiled tcgen05 first product
+    size_t p1_fast = ((size_t)dp * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)dp * r + r + 4) : 0;
     L.part1 = take(p1 > p1_fast ? p1 : p1_fast);
     L.part1v = take(sizeof(double) * (size_t)L.gv * (r + 2));
     size_t p2 = sizeof(double) * (size_t)L.g2x * L.g2y * (3 + G2_RT);
     size_t p2_fast = sizeof(double) * (size_t)kSMs * 4 * (4 + (size_t)r);
     L.part2 = take(p2 > p2_fast ? p2 : p2_fast);
     // generic family: nred1 block shares; fused reduction: one share per 16 entries of a record + r + 2 sums
-    L.red1 = take(sizeof(double) * ((size_t)L.nred1 + ((size_t)d * r + r + 2 + 15) / 16 + r + 2 + 8));
+    L.red1 = take(sizeof(double) * ((size_t)L.nred1 + ((size_t)dp * r + r + 2 + 15) / 16 + r + 2 + 8));
     L.setup = take(sizeof(double) * (3 * (size_t)d + 4 + (size_t)L.gs * d));
     L.hist = take(P.history ? sizeof(gem_nlr_iter_info) * (size_t)(P.T > 0 ? P.T : 1) : 0);
     L.xhat = take(P.x_inplace ? 0 : sizeof(float) * (size_t)n * d);
     // tcgen05 shapes: X-hat is static, so its two-term fp16 split is built once, row-major (second product)
     // and transposed in blocks of fb features x 32 rows (first product): about 2 x 2 x n x d halves.
     L.n_pad = (n + 63) / 64 * 64;
-    L.fb = d >= 256 ? 256 : d;
-    const bool tc_images = (P.precision == -1 || P.precision == 1) && r >= 32 && d % 32 == 0 && n >= 4096;
-    L.ximg = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)n * d : 0);
-    L.ximgT = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)(L.n_pad / 32) * ((d + L.fb - 1) / L.fb) * L.fb * 32 : 0);
+    L.fb = dp >= 256 ? 256 : dp;
+    L.ximg = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)n * dp : 0);
+    L.ximgT = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)(L.n_pad / 32) * ((dp + L.fb - 1) / L.fb) * L.fb * 32 : 0);
     L.total = off;
     return L;
 }
@@ -81,6 +86,7 @@ using namespace gemnlr;
 
 struct gem_nlr {
     Problem pb;
+    Problem pbp;           // the view of pb for the fp16-image tensor-core kernels: P.d = L.dp
     float* X_in;
     bool normalized;
     bool loaded;           // p = U^T 1 is on the device for the current U
@@ -166,21 +172,21 @@ static void launch_iteration(gem_nlr_t* h)
     cudaEvent_t* e = prof ? h->ev + h->ev_used : nullptr;
     if (prof) cudaEventRecord(e[0], h->pb.stream);
     if (h->use_tc1) {
-        tc1_launch_first(h->pb, h->tc1);
-        red1_fused_launch(h->pb, h->tc1.grid, 0);
+        tc1_launch_first(h->pbp, h->tc1);
+        red1_fused_launch(h->pbp, h->tc1.grid, 0);
     } else if (h->use_ffma) {
         if (h->use_mma) mma_launch_first(h->pb, h->ffma, 0);
         else ffma_launch_first(h->pb, h->ffma, 0);
     } else {
         launch_vector_pass(h->pb);
-        if (h->use_tcg1) tcg_launch_first(h->pb, h->tcg1);
+        if (h->use_tcg1) tcg_launch_first(h->pbp, h->tcg1);
         else launch_generic_pass1(h->pb, 0);
         launch_fin1(h->pb, 0);
     }
     if (prof) cudaEventRecord(e[1], h->pb.stream);
     if (h->use_tc || h->use_ffma || h->use_tcg) {
-        if (h->use_tcg) tcg_launch_second(h->pb, h->tcg);
-        else if (h->use_tc) tc_launch_second(h->pb, h->tc);
+        if (h->use_tcg) tcg_launch_second(h->pbp, h->tcg);
+        else if (h->use_tc) tc_launch_second(h->pbp, h->tc);
         else if (h->use_mma) mma_launch_second(h->pb, h->ffma);
         else ffma_launch_second(h->pb, h->ffma);
         if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
@@ -254,6 +260,9 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     h->path = "generic";
     h->err[0] = 0;
     h->pb.launches = &h->launches;
+    h->pb.dx = params->d;
+    h->pbp = h->pb;
+    h->pbp.P.d = L.dp;
     // Kernel families by shape.  precision 3: the warp-level TF32 (mma.sync, 3-product split) kernels
     // where instantiated, else generic; precision -1 prefers them to the FFMA kernels for d >= 64.
     // precision 2: generic only.  precision 0: FFMA family where a shape is
@@ -273,20 +282,20 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     }
     if (want_tc && !(params->precision == -1 && h->use_ffma)) {
         float* img = reinterpret_cast<float*>((char*)workspace_dev + L.thimg);
-        if (tc_plan(h->pb, &h->tc, img)) {
+        if (tc_plan(h->pbp, &h->tc, img)) {
             h->use_tc = true;
             h->path = h->use_ffma ? (h->tc.f16 ? "ffma+f16x3" : "ffma+tf32x3") : (h->tc.f16 ? "generic+f16x3" : "generic+tf32x3");
-            if (tc1_plan(h->pb, &h->tc1)) {
+            if (tc1_plan(h->pbp, &h->tc1)) {
                 h->use_tc1 = true;
                 // first product on the fp16 split; second on the fp16 split when the static images of X-hat
                 // are in the workspace, else on the TF32 split
                 h->path = h->tc.f16 ? "f16x3" : "f16x3+tf32x3";
             }
         }
-        else if (tcg_plan(h->pb, &h->tcg, img)) {
+        else if (tcg_plan(h->pbp, &h->tcg, img)) {
             h->use_tcg = true;
             h->path = "generic+f16x3.tiled";
-            if (tcg1_plan(h->pb, &h->tcg1)) {
+            if (tcg1_plan(h->pbp, &h->tcg1)) {
                 h->use_tcg1 = true;
                 h->path = "f16x3.tiled";
             }
@@ -301,6 +310,10 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
     int rc = reset_ctl(h, 0);
     if (rc == GEM_NLR_OK &&
         cudaMemsetAsync(h->pb.ytilde(), 0, sizeof(float) * (size_t)params->n, h->pb.stream) != cudaSuccess)
+        rc = GEM_NLR_E_CUDA;
+    // the padding rows of Theta (features d .. dp - 1) are written only by the image kernels' own reduction
+    if (rc == GEM_NLR_OK &&
+        cudaMemsetAsync(h->pb.theta(), 0, sizeof(float) * (size_t)L.dp * params->r, h->pb.stream) != cudaSuccess)
         rc = GEM_NLR_E_CUDA;
     if (rc != GEM_NLR_OK) {
         cudaFreeHost(h->host_ctl);
@@ -327,7 +340,7 @@ int gem_nlr_spectral_norm(gem_nlr_t* h, double* a_out)
     h->a = a;
     h->normalized = true;
     if (h->pb.has_ximg() && (h->use_tcg || h->use_tc)) {  // static fp16 images of X-hat for the tensor-core kernels
-        tcg_prepare(h->pb);
+        tcg_prepare(h->pbp);
         CK(h, cudaStreamSynchronize(h->pb.stream));
     }
     if (a_out) *a_out = a;
@@ -341,7 +354,7 @@ int gem_nlr_set_normalized(gem_nlr_t* h, double a)
     h->a = a;
     h->normalized = true;
     if (h->pb.has_ximg() && (h->use_tcg || h->use_tc)) {
-        tcg_prepare(h->pb);
+        tcg_prepare(h->pbp);
         CK(h, cudaStreamSynchronize(h->pb.stream));
     }
     return GEM_NLR_OK;

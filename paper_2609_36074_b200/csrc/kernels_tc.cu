@@ -447,6 +447,7 @@ bool tc_plan(const Problem& pb, TcPlan* pl, float* img_storage)
     const size_t pan_bytes = (size_t)tc::TILE_M * PW * 4;
     // fp16 split on the static images of X-hat when the workspace holds them, else the TF32 split
     const bool f16 = pb.has_ximg();
+    if (!f16 && d != pb.dx) return false;                     // the TF32 variant reads X-hat itself: no feature padding
     const size_t th = (size_t)NB * NP * (f16 ? 64 : 128);
     const size_t fixed = 2 * th + (size_t)2 * ACC_COLS * 4 + 1024;
     const size_t limit = 227 * 1024 - 2048;

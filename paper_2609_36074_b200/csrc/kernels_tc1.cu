@@ -394,6 +394,7 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     if ((size_t)d * r > 16384) return false;          // partial records of the shared reduction kernel
     const int NBX = d / 32;
     const bool ximg = pb.has_ximg() && pb.L.fb == d;          // one block of d features per stage in the transposed images
+    if (!ximg && d != pb.dx) return false;                    // without images X-hat itself is read: no feature padding
     const size_t stage = (((size_t)tc1::TR * r * 4 + 127) / 128 * 128 + (ximg ? 0 : (size_t)tc1::TR * d * 4) + 1023) / 1024 * 1024;
     const size_t img = (size_t)2 * tc1::UIMG + (size_t)2 * d * 64;
     const size_t limit = 227 * 1024 - 2048;

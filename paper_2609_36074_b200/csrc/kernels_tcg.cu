@@ -67,13 +67,14 @@ __global__ void k_theta_images64(const float* __restrict__ theta, int d, int r, 
     }
 }
 
-// X-hat (n x d FP32) -> its fp16 split images x 2^15 = h1 + h2: row-major (n x d), and transposed in the
+// X-hat (n rows of dx features, FP32) -> its fp16 split images x 2^15 = h1 + h2 over d >= dx features (zero beyond
+// dx): row-major (n x d), and transposed in the
 // exact shared-memory form the first product consumes: for every stage of 32 data rows and block of fb
 // features one contiguous box [feature][32 rows] with the 64-byte swizzle already applied (zero
 // beyond n and d), so that a box arrives with one bulk copy.  One block per 32 x 32 tile; the
 // transposition goes through shared memory.
 __global__ void __launch_bounds__(256)
-k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, int fb, __half* __restrict__ h1,
+k_ximg_build(const float* __restrict__ X, int64_t n, int dx, int d, int64_t n_pad, int fb, __half* __restrict__ h1,
              __half* __restrict__ h2, __half* __restrict__ h1T, __half* __restrict__ h2T)
 {
     __shared__ __half t1[32][33], t2[32][33];
@@ -84,7 +85,7 @@ k_ximg_build(const float* __restrict__ X, int64_t n, int d, int64_t n_pad, int f
     for (int i = 0; i < 4; ++i) {
         const int64_t row = row0 + ty + 8 * i;
         const int f = f0 + tx;
-        const float v = (row < n && f < d) ? X[row * d + f] * 32768.0f : 0.f;
+        const float v = (row < n && f < dx) ? X[row * dx + f] * 32768.0f : 0.f;      // features dx .. d - 1: zero padding
         const __half a = __float2half_rn(v);
         const __half b = __float2half_rn(v - __half2float(a));
         if (row < n && f < d) { h1[row * d + f] = a; h2[row * d + f] = b; }
@@ -409,7 +410,7 @@ constexpr int NTH1 = (2 + 4 + 4 * NT1 + 1) * 32;   // U producer, MMA issuer, 4 
 __global__ void __launch_bounds__(NTH1, 1)
 k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ xT1,
             const __half* __restrict__ xT2, Ctl* __restrict__ ctl, int64_t n, int d, int r, int K,
-            int NMT, int NNB, int NSPLIT, double* __restrict__ part)
+            int NMT, int NNB, int NSPLIT, int fb, double* __restrict__ part)
 {
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
@@ -421,8 +422,8 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int mt = blockIdx.x % NMT, nb = (blockIdx.x / NMT) % NNB, sp = blockIdx.x / (NMT * NNB);
     const int c0 = mt * 128;                               // first column of U of this item
-    const int f0 = nb * 256;
-    const int Nb = (d - f0 < 256) ? d - f0 : 256;          // features of this item (multiple of 32)
+    const int f0 = nb * fb;                                // fb = features per block of the transposed images: 256, or d < 256
+    const int Nb = (d - f0 < fb) ? d - f0 : fb;            // features of this item (multiple of 32)
 
     const uint32_t img0 = smem_u32(smem);
     const uint32_t raw0 = img0 + (uint32_t)NIM1 * IMG1;
@@ -483,10 +484,11 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
                 const int l = g % NIM1;
                 if (g >= NIM1) mbar_wait_backoff(imgfree(l), ((g / NIM1) - 1) & 1, &abort_flag, ctl);
                 const uint32_t im = img0 + (uint32_t)l * IMG1;
-                const size_t xoff = ((size_t)(g_lo + g) * NNB + nb) * (256 * 32);      // this stage's box of the feature block
-                mbar_expect_tx(imgfull(l), 2 * XIMG1);
-                bulk_load_1d(im + 2 * UIMG1, xT1 + xoff, XIMG1, imgfull(l));
-                bulk_load_1d(im + 2 * UIMG1 + XIMG1, xT2 + xoff, XIMG1, imgfull(l));
+                const size_t xoff = ((size_t)(g_lo + g) * NNB + nb) * ((size_t)fb * 32);   // this stage's box of the feature block
+                const uint32_t xbytes = (uint32_t)fb * 64;
+                mbar_expect_tx(imgfull(l), 2 * xbytes);
+                bulk_load_1d(im + 2 * UIMG1, xT1 + xoff, xbytes, imgfull(l));
+                bulk_load_1d(im + 2 * UIMG1 + XIMG1, xT2 + xoff, xbytes, imgfull(l));
             }
         }
     } else if (warp == 1) {
@@ -613,7 +615,7 @@ void tcg_prepare(const Problem& pb)
 {
     cudaMemsetAsync(pb.ximgT(0), 0, sizeof(uint16_t) * 2 * pb.ximgT_halves(), pb.stream);
     const dim3 grid((unsigned)((pb.L.n_pad + 31) / 32), (unsigned)((pb.P.d + 31) / 32));
-    tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.P.d, pb.L.n_pad, pb.L.fb,
+    tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.dx, pb.P.d, pb.L.n_pad, pb.L.fb,
                                                    reinterpret_cast<__half*>(pb.ximg(0)), reinterpret_cast<__half*>(pb.ximg(1)),
                                                    reinterpret_cast<__half*>(pb.ximgT(0)), reinterpret_cast<__half*>(pb.ximgT(1)));
     pb.count(1);
@@ -622,9 +624,10 @@ void tcg_prepare(const Problem& pb)
 bool tcg1_plan(const Problem& pb, Tcg1Plan* pl)
 {
     const int d = pb.P.d, r = pb.P.r;
+    // 256-feature blocks only (d >= 256): narrower blocks with more row ranges are not enabled
     if (!pb.has_ximg() || pb.L.fb != 256 || d % 32 != 0 || r % 4 != 0 || pb.P.n < 4096 || pb.P.n > 2000000000ll) return false;
     pl->NMT = (r + 127) / 128;
-    pl->NNB = (d + 255) / 256;
+    pl->NNB = (d + pb.L.fb - 1) / pb.L.fb;
     const int tiles = pl->NMT * pl->NNB;
     if (tiles > kSMs) return false;
     pl->NSPLIT = kSMs / tiles;
@@ -641,7 +644,7 @@ void tcg_launch_first(const Problem& pb, const Tcg1Plan& pl)
 {
     tcg::k_pass1_tcg<<<pl.grid, tcg::NTH1, pl.smem, pb.stream>>>(pl.tmU, reinterpret_cast<const __half*>(pb.ximgT(0)),
                                                                  reinterpret_cast<const __half*>(pb.ximgT(1)), pb.ctl(), pb.P.n, pb.P.d, pb.P.r,
-                                                                 pb.P.K, pl.NMT, pl.NNB, pl.NSPLIT, pb.part1());
+                                                                 pb.P.K, pl.NMT, pl.NNB, pl.NSPLIT, pb.L.fb, pb.part1());
     pb.count(1);
     launch_red1(pb, pl.NSPLIT, 0, 0);
 }

@@ -30,6 +30,7 @@ struct Ctl {
 struct Layout {
     size_t ctl, p, s, alpha_s, theta, thimg, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
     size_t ximg, ximgT;      // fp16 split images of X-hat (row-major and transposed), wide tensor-core shapes only (else 0 bytes)
+    int dp;                  // d rounded up to a multiple of 32 when the fp16 images exist, else d: feature count of the image kernels
     int64_t n_pad;           // n rounded up to 64: the transposed images cover n_pad / 32 stages of 32 rows
     int fb;                  // features per block of the transposed images: 256, or d when d < 256
     int g1x, g1y_d, g1y_r;   // generic pass-1 grid: row chunks, d tiles, r tiles
@@ -47,6 +48,10 @@ Layout make_layout(const gem_nlr_params& P);
 
 struct Problem {
     gem_nlr_params P;
+    int dx;          // features per row of X as stored (row pitch).  P.d equals dx except in the view the
+                     // fp16-image tensor-core kernels get, where P.d is dx rounded up to a multiple of 32:
+                     // those kernels read X-hat only through its images, whose padding features are zero,
+                     // so Theta gains zero rows and nothing else changes
     float* X;        // X-hat once normalized
     float* U;
     char*  ws;

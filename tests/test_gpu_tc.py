@@ -92,3 +92,50 @@ def test_tiled_tc_trajectory_is_reproducible_and_matches_oracle():
     Uo, _, infoo, _, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, hp["T_min"])
     assert u_err(outs[0][0], Uo) <= TOL_U
     assert rel(outs[0][1]["rho"], infoo["rho"]) <= 1e-4
+
+
+# ---- feature counts that are not a multiple of 32: the fp16-image kernels see d rounded up (zero features in the
+# images, zero rows in Theta); includes the shapes of the paper's own scaling study (d = 50, r = 3 K) ----
+# (n, d, K, r, kernel path)
+PADDED_D_SHAPES = [(5000, 50, 60, 60, "f16x3"), (6001, 50, 20, 60, "f16x3"), (4500, 200, 100, 100, "generic+f16x3"),
+                   (4300, 300, 400, 400, "f16x3.tiled"), (4200, 110, 300, 300, "generic+f16x3.tiled")]
+
+
+@pytest.mark.parametrize("n,d,K,r,path", PADDED_D_SHAPES)
+def test_padded_feature_count_teacher_forced(n, d, K, r, path):
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 0)
+    X, _, _ = synth.make_mixture(spec)
+    Xhat, _, _ = oracle.normalize(X)
+    U0 = synth.make_u0(n, r, K, seed=0)
+    hp = synth.default_hparams(K)
+    s = make_solver(Xhat, U0, K, hp, precision=-1)
+    assert s.path() == path, s.path()
+    s.destroy()
+    recs = teacher_forced_steps(Xhat, U0, K, hp, steps=3, tol_u=TOL_U, solver_kw=dict(precision=-1))
+    for rec in recs:
+        assert rec["a"] <= 1e-6 and rec["b"] <= 1e-6 and rec["h"] <= 1e-6, rec
+        assert rec["c"] <= 2e-7 and rec["delta"] <= 1e-6, rec
+        assert rec["rho"] <= 1e-5 and rec["fhat"] <= TOL_F, rec
+        assert rec["dual"][0] == rec["dual"][1] and rec["stop"][0] == rec["stop"][1], rec
+
+
+def test_padded_feature_count_full_run_with_setup():
+    """Whole job on raw X (mean, power iteration, normalisation, images, iterations) at d = 50, r = 60."""
+    import torch
+    n, d, K, r, T = 20000, 50, 20, 60, 25
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 3)
+    X, _, _ = synth.make_mixture(spec)
+    U0 = synth.make_u0(n, r, K, seed=3)
+    hp = dict(synth.default_hparams(K), eps_d=0.2)
+    Xd, Ud = torch.from_numpy(X.copy()).cuda(), torch.from_numpy(U0.copy()).cuda()
+    s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"], T=T, T_min=T)
+    a = s.spectral_norm()
+    assert s.path() == "f16x3", s.path()
+    rc, info, iters = s.run()
+    assert rc == gem.ITER_CAP and iters == T, (rc, s.last_error())
+    Xhat, a_o, _ = oracle.normalize(X)
+    assert rel(a, a_o) <= 1e-5
+    Uo, _, infoo, _, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, T)
+    assert u_err(s.U.cpu().numpy(), Uo) <= 5e-4          # the two sides normalise with their own a (1e-5 apart)
+    assert rel(info["fhat"], infoo["fhat"]) <= 1e-4 and rel(info["rho"], infoo["rho"]) <= 1e-3
+    s.destroy()
