@@ -96,9 +96,10 @@ typedef struct {
 
 /* Bytes of caller-provided device workspace needed for these parameters (0 if invalid).
  * Includes the y/sqrt(n) and ybar vectors, Theta, p, s, the reduction partials, the
- * optional history, when x_inplace == 0 a copy of X and, for the wide tensor-core shapes
- * (precision -1 or 1, r > 256, d a multiple of 32, n >= 4096), the static fp16 split images
- * of X-hat, row-major and transposed (8 n d bytes).                                            */
+ * optional history, when x_inplace == 0 a copy of X and, for the tensor-core shapes
+ * (precision -1 or 1, r >= 32, n >= 4096), the static fp16 split images of X-hat, row-major
+ * and transposed (8 n d' bytes, d' = d rounded up to a multiple of 32: the image kernels see
+ * zero features beyond d, so any d is accepted).                                               */
 size_t gem_nlr_workspace_bytes(const gem_nlr_params *params);
 
 /* Device bytes the paper's own buffer table would use for the same problem:
