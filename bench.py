@@ -230,11 +230,14 @@ def main():
 
     # labels (S7) timed on their own
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    lab = torch.empty(n, dtype=torch.int32, device=dev)
+    solver.labels(lab)                      # untimed first call (allocation, module load)
     e0.record()
-    solver.labels()
+    solver.labels(lab)
     e1.record()
     torch.cuda.synchronize()
     labels_ms = e0.elapsed_time(e1)
+    del lab
     path = solver.path()
     P = make_params(n, d, K, r=r, **kw)
     ws_bytes = gem.workspace_bytes(P)

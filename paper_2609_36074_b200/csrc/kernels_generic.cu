@@ -567,6 +567,84 @@ __global__ void k_labels(const float* __restrict__ U, int64_t n, int r, int32_t*
     }
 }
 
+// Row-argmax read-out with 16-byte loads (r a multiple of 4).  Narrow factors (r <= 32): a thread takes two rows
+// at a time, all their pieces requested before the first comparison.  Wider ones (r <= 1024): a warp takes
+// 8 / NK rows at a time, a lane NK pieces of each (as in k_rowvec_wide); elements are visited in increasing
+// column order inside a lane and the lanes are combined on (value, index), so ties go to the smallest index.
+__global__ void __launch_bounds__(256)
+k_labels_small4(const float* __restrict__ U, int64_t n, int r4, int32_t* __restrict__ labels)
+{
+    const float4* U4 = reinterpret_cast<const float4*>(U);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; row < n; row += 2 * stride) {
+        const int64_t row1 = row + stride;
+        float4 a[8], b[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            a[c] = (c < r4) ? __ldcs(U4 + row * r4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            b[c] = (c < r4 && row1 < n) ? __ldcs(U4 + row1 * r4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float bva = a[0].x, bvb = b[0].x;
+        int ba = 0, bb = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            if (c < r4) {
+                const float va[4] = {a[c].x, a[c].y, a[c].z, a[c].w}, vb[4] = {b[c].x, b[c].y, b[c].z, b[c].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (va[e] > bva) { bva = va[e]; ba = 4 * c + e; }
+                    if (vb[e] > bvb) { bvb = vb[e]; bb = 4 * c + e; }
+                }
+            }
+        }
+        labels[row] = ba;
+        if (row1 < n) labels[row1] = bb;
+    }
+}
+
+template <int NK>
+__global__ void __launch_bounds__(256)
+k_labels_wide(const float* __restrict__ U, int64_t n, int r, int32_t* __restrict__ labels)
+{
+    constexpr int ROWS = 8 / NK;
+    const int lane = threadIdx.x & 31, r4 = r >> 2;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t row0 = warp * ROWS; row0 < n; row0 += nwarps * ROWS) {
+        float4 u[ROWS][NK];
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i)
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                const int c4 = lane + 32 * k;
+                u[i][k] = (c4 < r4 && row0 + i < n) ? __ldcs(reinterpret_cast<const float4*>(U + (row0 + i) * r) + c4)
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i) {
+            float bv = -INFINITY;
+            int best = 0x7fffffff;
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                const int c4 = lane + 32 * k;
+                if (c4 < r4) {
+                    const float v[4] = {u[i][k].x, u[i][k].y, u[i][k].z, u[i][k].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (v[e] > bv) { bv = v[e]; best = 4 * c4 + e; }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int ob = __shfl_xor_sync(0xffffffffu, best, o);
+                if (ov > bv || (ov == bv && ob < best)) { bv = ov; best = ob; }
+            }
+            if (lane == 0 && row0 + i < n) labels[row0 + i] = best;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // Thread-per-row variants of the vector pass and of the column sums for narrow factors
 // (r = 4 R4 <= 32): a thread reads its whole row with 16-byte loads (consecutive threads read
@@ -867,6 +945,27 @@ void launch_objective(const Problem& pb)
 void launch_labels(const Problem& pb, int32_t* labels)
 {
     const auto& P = pb.P;
+    if (P.r % 4 == 0 && P.r <= 32) {
+        int64_t blocks = (P.n + 511) / 512;
+        if (blocks > kSMs * 8) blocks = kSMs * 8;
+        k_labels_small4<<<(int)(blocks < 1 ? 1 : blocks), 256, 0, pb.stream>>>(pb.U, P.n, P.r / 4, labels);
+        pb.count();
+        return;
+    }
+    if (wide_r(P.r)) {
+        const int nk = wide_nk(P.r);
+        int64_t blocks = (P.n + 8 * (8 / nk) - 1) / (8 * (8 / nk));
+        if (blocks > kSMs * 8) blocks = kSMs * 8;
+        const int g = (int)(blocks < 1 ? 1 : blocks);
+        switch (nk) {
+        case 1: k_labels_wide<1><<<g, 256, 0, pb.stream>>>(pb.U, P.n, P.r, labels); break;
+        case 2: k_labels_wide<2><<<g, 256, 0, pb.stream>>>(pb.U, P.n, P.r, labels); break;
+        case 4: k_labels_wide<4><<<g, 256, 0, pb.stream>>>(pb.U, P.n, P.r, labels); break;
+        default: k_labels_wide<8><<<g, 256, 0, pb.stream>>>(pb.U, P.n, P.r, labels); break;
+        }
+        pb.count();
+        return;
+    }
     int blocks = (int)((P.n + 255) / 256);
     if (P.r > 32) blocks = (int)((P.n + 7) / 8);
     if (blocks > kSMs * 16) blocks = kSMs * 16;

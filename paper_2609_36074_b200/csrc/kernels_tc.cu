@@ -269,7 +269,6 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 mbar_wait(xfull(s), (g / NSB) & 1, &abort_flag, ctl);
                 if (g >= NLO) mbar_wait(lofree(l), ((g / NLO) - 1) & 1, &abort_flag, ctl);
                 const uint32_t hi_a = stage0 + (uint32_t)s * BOX_BYTES, lo_a = lo0 + (uint32_t)l * BOX_BYTES;
-#pragma unroll
                 float4 xin[BOX_BYTES / 16 / 128];
 #pragma unroll
                 for (int k = 0; k < BOX_BYTES / 16 / 128; ++k) xin[k] = lds128(hi_a + (uint32_t)(k * 128 + st) * 16);
@@ -296,8 +295,6 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         const int grp = (warp - 2) >> 2;                  // epilogue group
         const int rl = q * 32 + lane;                     // row of the tile owned by this thread
         const int gt = (q * 32 + lane);                   // 0..127 inside the group
-        // column (within a 16-column half) whose sum this lane holds after colsum16
-        const int ccol = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
         int i = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
             const int a = i & 1;

@@ -44,7 +44,6 @@ namespace gemnlr {
 namespace tc1 {
 
 constexpr int TR = 32;                         // data rows per stage (4 k-steps)
-constexpr int CHUNK_BYTES = TR * 128;          // one box: TR rows x 32 floats
 constexpr int NTEAMS = 3;                      // vector / split teams of four warps, taking stages round-robin
 constexpr int NTHREADS = (6 + 4 * NTEAMS + 1) * 32;   // + the X-hat image producer (last warp)
 constexpr int MAX_RING = 8;
@@ -72,7 +71,6 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int NBX = d / 32;                        // X-hat boxes per stage
-    const int NBU = (r + 31) / 32;                 // U boxes per stage (M = 128 reads 4; missing ones are never written: see below)
     // raw stage: the TR rows of U then those of X-hat exactly as they lie in global memory (row pitch r and
     // d floats): the rows of a stage are contiguous there, so each operand arrives with one bulk copy
     const int URAW = (TR * r * 4 + 127) / 128 * 128;
@@ -211,7 +209,6 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
         // (reductions, FP64 row scalars, conversions) against a budget of ~900, so several are in flight.
         const int vw = warp - 6;                           // 0 .. 4 NTEAMS - 1
         const int team = vw >> 2, tw = vw & 3;             // team; data rows 8 tw .. 8 tw + 7 of the team's stages
-        const int tt = tw * 32 + lane;                     // 0..127 inside the team
         float p1[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) p1[j] = sp[lane + 32 * j];
@@ -305,7 +302,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 if (dual) ytilde[myrow] = yt_l;
                 ybar[myrow] = yb_l;
             }
-            // ---- X-hat boxes -> fp16 images: thread = (feature tt & 31, data rows 8 (tt >> 5) .. + 7) of a box ----
+            // ---- X-hat boxes -> fp16 images: thread = (feature lane, data rows 8 tw .. 8 tw + 7) of a box ----
             for (int b = 0; !XIMG && b < NBX; ++b) {
                 float v[8];
 #pragma unroll
@@ -392,7 +389,6 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     const int d = pb.P.d, r = pb.P.r;
     if (d % 32 != 0 || d > 256 || r % 4 != 0 || r < 8 || r > 128 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
     if ((size_t)d * r > 16384) return false;          // partial records of the shared reduction kernel
-    const int NBX = d / 32;
     const bool ximg = pb.has_ximg() && pb.L.fb == d;          // one block of d features per stage in the transposed images
     if (!ximg && d != pb.dx) return false;                    // without images X-hat itself is read: no feature padding
     const size_t stage = (((size_t)tc1::TR * r * 4 + 127) / 128 * 128 + (ximg ? 0 : (size_t)tc1::TR * d * 4) + 1023) / 1024 * 1024;
