@@ -91,7 +91,7 @@ k_pi_pass_vec(const float* __restrict__ X, int64_t n, const double* __restrict__
     constexpr int D = 4 * LPR * NCH;
     constexpr int RPW = 32 / LPR;                       // rows per warp and step
     __shared__ double sv[D], smean[D];
-    __shared__ double sacc[PI_WARPS][D];
+    __shared__ double sfold[D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane % LPR, rg = lane / LPR;
     for (int j = threadIdx.x; j < D; j += blockDim.x) { sv[j] = v[j]; smean[j] = mean[j]; }
@@ -123,21 +123,26 @@ k_pi_pass_vec(const float* __restrict__ X, int64_t n, const double* __restrict__
 #pragma unroll
         for (int k = 0; k < NCH * 4; ++k) acc[k] = fma(z, xc[k], acc[k]);
     }
-    // fold the row groups of the warp (lanes with equal sub), then the warps in warp order
+    // fold the row groups of the warp (lanes with equal sub), then the warps one after the other in warp order
+    // into one shared record
 #pragma unroll
     for (int k = 0; k < NCH * 4; ++k) {
         double t = acc[k];
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (rg == 0) sacc[warp][4 * (sub + (k >> 2) * LPR) + (k & 3)] = t;
+        acc[k] = t;
     }
-    __syncthreads();
-    for (int j = threadIdx.x; j < D; j += blockDim.x) {
-        double t = 0.0;
+    for (int w = 0; w < PI_WARPS; ++w) {
+        if (warp == w && rg == 0) {
 #pragma unroll
-        for (int w = 0; w < PI_WARPS; ++w) t += sacc[w][j];
-        part[(size_t)blockIdx.x * D + j] = t;
+            for (int k = 0; k < NCH * 4; ++k) {
+                const int j = 4 * (sub + (k >> 2) * LPR) + (k & 3);
+                sfold[j] = (w == 0) ? acc[k] : sfold[j] + acc[k];
+            }
+        }
+        __syncthreads();
     }
+    for (int j = threadIdx.x; j < D; j += blockDim.x) part[(size_t)blockIdx.x * D + j] = sfold[j];
 }
 
 // w = sum of the per-CTA partials in CTA order (the result of one application of X_c^T X_c to v).
@@ -267,7 +272,7 @@ int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, dou
         switch (d) {
 #define PI_CASE(DD, LPR, NCH) case DD: k_pi_pass_vec<LPR, NCH><<<g, PI_WARPS * 32, 0, st>>>(X_in, P.n, mean, v, part); break;
             PI_CASE(16, 4, 1) PI_CASE(32, 8, 1) PI_CASE(64, 16, 1) PI_CASE(128, 32, 1) PI_CASE(256, 32, 2)
-            PI_CASE(384, 32, 3) PI_CASE(512, 32, 4)
+            PI_CASE(384, 32, 3) PI_CASE(512, 32, 4) PI_CASE(640, 32, 5) PI_CASE(768, 32, 6)
 #undef PI_CASE
             default: k_pi_pass<<<g, PI_WARPS * 32, smem, st>>>(X_in, P.n, d, mean, v, part); break;
         }

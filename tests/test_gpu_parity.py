@@ -125,7 +125,7 @@ def test_tiny_mixtures_recover_exact_kmeans_partition(K, seed):
     s.destroy()
 
 
-@pytest.mark.parametrize("n,d,center", [(5000, 16, 1), (3000, 37, 1), (2048, 128, 0), (700, 300, 1)])
+@pytest.mark.parametrize("n,d,center", [(5000, 16, 1), (3000, 37, 1), (2048, 128, 0), (700, 300, 1), (1500, 768, 1), (900, 512, 0)])
 def test_setup_matches_oracle(n, d, center):
     rng = np.random.default_rng(n + d)
     X = (rng.standard_normal((n, d)) * rng.uniform(0.3, 3.0, size=d) + rng.uniform(-4, 4, size=d)
