@@ -31,3 +31,17 @@ def test_storage_accounting_closed_forms():
     assert gem.workspace_bytes(make_params(n, d, r, x_inplace=0)) >= ws + 4 * n * d
     assert gem.workspace_bytes(make_params(0, d, r)) == 0          # invalid
     assert gem.workspace_bytes(make_params(n, d, 4, r=2)) == 0     # r < K
+
+
+def test_image_workspace_rounds_the_feature_count_up():
+    # The tensor-core shapes (r >= 32, n >= 4096) keep fp16 split images of X-hat, row-major and transposed:
+    # 8 n d' bytes with d' = d rounded up to a multiple of 32, so d = 50 costs what d = 64 costs there;
+    # below n = 4096 and for narrow factors there are no images.
+    n, r = 100_000, 60
+    base = gem.workspace_bytes(make_params(n, 64, r, precision=2))           # generic only: no images
+    w64 = gem.workspace_bytes(make_params(n, 64, r))
+    w50 = gem.workspace_bytes(make_params(n, 50, r))
+    assert 8 * n * 64 <= w64 - base <= 8 * n * 64 + 64 * 64 * 128 + 2 ** 20
+    assert abs(w50 - w64) <= 2 ** 20                                         # Theta and partials sized for d' too
+    assert gem.workspace_bytes(make_params(4000, 50, r)) == gem.workspace_bytes(make_params(4000, 50, r, precision=2))
+    assert gem.workspace_bytes(make_params(n, 50, 16)) == gem.workspace_bytes(make_params(n, 50, 16, precision=2))
