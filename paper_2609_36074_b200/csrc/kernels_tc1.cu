@@ -45,7 +45,20 @@ namespace tc1 {
 
 constexpr int TR = 32;                         // data rows per stage (4 k-steps)
 constexpr int NTEAMS = 3;                      // vector / split teams of four warps, taking stages round-robin
-constexpr int NTHREADS = (6 + 4 * NTEAMS + 1) * 32;   // + the X-hat image producer (last warp)
+constexpr int NTHREADS = 20 * 32;
+// Warp roles.  A warp runs on scheduler (warp index mod 4).  The thread that issues the MMAs executes a serial
+// stream of ~100 instructions per stage; when it shared its scheduler with three busy team warps that
+// stream, not the tensor pipe or the teams, set the stage rate (device timelines: no wait on its path, 1400
+// cycles per stage).  So scheduler 1 hosts only light roles: the issuer (warp 1), one of the four epilogue
+// warps (5: the TMEM lane quarter of a warp is fixed by its index mod 4), the two producers (9, 13) and an
+// idle warp (17); the twelve team warps are the warps of schedulers 0, 2 and 3 outside the epilogue group 4-7.
+__device__ __forceinline__ bool is_team_warp(int w) { return (w & 3) != 1 && (w >> 2) != 1; }
+__device__ __forceinline__ int team_warp_index(int w)          // 0 .. 11 over the team warps in increasing order
+{
+    const int q = w >> 2, res = w & 3;
+    return (q == 0 ? 0 : q - 1) * 3 + (res == 0 ? 0 : res - 1);
+}
+constexpr int WARP_UPROD = 9, WARP_XPROD = 13, WARP_ISSUER = 1, WARP_EPI0 = 4;
 constexpr int MAX_RING = 8;
 constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
 constexpr int UIMG = 128 * 64;                 // one fp16 image of the U operand: 128 columns x 32 data rows
@@ -105,7 +118,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
         fence_barrier_init();
     }
     if (threadIdx.x < 128) sp[threadIdx.x] = (threadIdx.x < r) ? p[threadIdx.x] : 0.f;
-    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
+    if (warp == WARP_ISSUER) tmem_alloc(smem_u32(&tmem_base_s), tmem_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -133,7 +146,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
     float s_acc[4] = {0.f, 0.f, 0.f, 0.f};         // vector warps: s partial of this lane's 4 columns
     double* const out = part + (size_t)blockIdx.x * ((size_t)d * r + r + 2);
 
-    if (warp == 0) {
+    if (warp == WARP_UPROD) {
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
@@ -152,7 +165,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 }
             }
         }
-    } else if (warp == 6 + 4 * NTEAMS) {
+    } else if (warp == WARP_XPROD) {
         // ------------------------------ X-hat image producer ------------------------------
         // Its own thread: the image ring is released by the MMAs, the raw ring by the teams; one thread
         // serving both would let the U loads run only one stage ahead.  The boxes of a stage go straight
@@ -168,7 +181,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 bulk_load_1d(im + 2 * UIMG + XIMG_BYTES, xT2 + xoff, (uint32_t)XIMG_BYTES, split(l));
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == WARP_ISSUER) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(128, d, 0, 0), idesc2 = umma_idesc_f16(128, 2 * d, 0, 0);
@@ -178,15 +191,18 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
             // image slot l and its phase, accumulator a and position in the accumulation period: kept
             // incrementally (this thread's instruction stream is the critical path of the kernel)
             int l = 0, lph = 0, a = 0, in_period = 0, period = 0;
+            // descriptors of image stage 0; the address field counts 16-byte units, so stage l adds l * IMG / 16
+            const uint64_t da1_0 = umma_desc_k_sw64(img0), da2_0 = umma_desc_k_sw64(img0 + UIMG);
+            const uint64_t db1_0 = umma_desc_k_sw64(img0 + 2 * UIMG), db2_0 = umma_desc_k_sw64(img0 + 2 * UIMG + XIMG_BYTES);
+            const uint64_t dstep = (uint64_t)(IMG >> 4);
             for (int g = 0; g < my_stages; ++g) {
                 if (in_period == 0 && period >= 2) mbar_wait_spin(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * ACC);
-                const uint32_t im = img0 + (uint32_t)l * IMG;
                 // A = U images (M = 128 columns), B = X-hat images (N = d features), K-major; a k-step of 16 data
                 // rows (32 bytes inside the 64-byte swizzled row) advances the start address by 2
-                const uint64_t da1 = umma_desc_k_sw64(im), da2 = umma_desc_k_sw64(im + UIMG);
-                const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG), db2 = umma_desc_k_sw64(im + 2 * UIMG + XIMG_BYTES);
+                const uint64_t doff = dstep * (uint64_t)l;
+                const uint64_t da1 = da1_0 + doff, da2 = da2_0 + doff, db1 = db1_0 + doff, db2 = db2_0 + doff;
                 if (wideB) umma_f16_x2(tacc, da1, da2, db1, idesc2, idesc, in_period ? 1u : 0u);
                 else umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
                 int ln = l + 1, lphn = lph;
@@ -198,16 +214,15 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                 if (in_period == FLUSH - 1 || g == my_stages - 1) umma_commit(accfull(a));
                 l = ln; lph = lphn;
                 if (++in_period == FLUSH) { in_period = 0; ++period; a ^= 1; }
-                if (abort_flag) break;
             }
         }
-    } else if (warp >= 6 && warp < 6 + 4 * NTEAMS) {
+    } else if (is_team_warp(warp)) {
         // ------------------------------ vector pass + split ------------------------------
         // A warp takes 8 consecutive data rows of a stage, a lane the columns lane + 32 j of U (scalar loads
         // from the plain FP32 rows: consecutive lanes, consecutive words).  NTEAMS teams of four warps take
         // the stages round-robin: a stage costs a team a few thousand cycles of mostly dependent latency
         // (reductions, FP64 row scalars, conversions) against a budget of ~900, so several are in flight.
-        const int vw = warp - 6;                           // 0 .. 4 NTEAMS - 1
+        const int vw = team_warp_index(warp);              // 0 .. 4 NTEAMS - 1
         const int team = vw >> 2, tw = vw & 3;             // team; data rows 8 tw .. 8 tw + 7 of the team's stages
         float p1[4];
 #pragma unroll
@@ -325,7 +340,7 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
         yq = warp_sum(yq);
         if (lane == 0) { sq[0][vw] = qq; sq[1][vw] = yq; }
     }
-    if (warp >= 2 && warp < 6) {
+    if (warp >= WARP_EPI0 && warp < WARP_EPI0 + 4) {
         // ------------------------------ epilogue: FP64 fold of the accumulator ------------------------------
         // Thread = column j of U (TMEM lane).  Each hand-over adds the FP32
         // accumulator of the period into this CTA's FP64 partial record (Theta^T entry (j, f) lives at
@@ -362,11 +377,11 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
     // Every MMA has completed (the epilogue waited for the last hand-over): the rings are scratch now.
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
+    if (warp == WARP_ISSUER) tmem_dealloc(tmem_base, tmem_cols);
     float* sscr = reinterpret_cast<float*>(smem);             // [vector warps][128 columns]
-    if (warp >= 6 && warp < 6 + 4 * NTEAMS) {
+    if (is_team_warp(warp)) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) sscr[(warp - 6) * 128 + lane + 32 * k] = s_acc[k] * ldexpf(1.0f, -eU);
+        for (int k = 0; k < 4; ++k) sscr[team_warp_index(warp) * 128 + lane + 32 * k] = s_acc[k] * ldexpf(1.0f, -eU);
     }
     __syncthreads();
     if (threadIdx.x < r) {

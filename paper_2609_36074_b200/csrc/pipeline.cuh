@@ -72,7 +72,9 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ void mbar_wait_spin(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                                Ctl* ctl)
 {
-    if (*abort_flag) return;
+    // The barrier is tested first and the abort flag only every 64 polls: the caller is a single thread whose
+    // instruction stream sets the stage rate, and a shared-memory read of the flag in front of every wait
+    // costs it tens of cycles per stage.  Once the flag is up a wait therefore returns within 64 polls.
     for (uint32_t i = 0; i < (kSpinLimit << 4); ++i) {
         uint32_t ok;
         asm volatile(
@@ -81,6 +83,7 @@ __device__ __forceinline__ void mbar_wait_spin(uint32_t bar, uint32_t parity, vo
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return;
+        if ((i & 63u) == 63u && *abort_flag) return;
     }
     *abort_flag = 1u;
     ctl->status = GEM_NLR_E_TIMEOUT;
