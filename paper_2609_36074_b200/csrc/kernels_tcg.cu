@@ -191,9 +191,11 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         // so the tensor pipe has work queued while this thread polls.
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(TILE_M, NBLK, 0, 0);
+            const uint64_t da1_0 = umma_desc_k_sw64(stage0), da2_0 = umma_desc_k_sw64(stage0 + A_BOX);
+            const uint64_t db1_0 = umma_desc_k_sw64(stage0 + 2 * A_BOX), db2_0 = umma_desc_k_sw64(stage0 + 2 * A_BOX + B_BOX);
             int64_t g = 0;
             int i = 0;
-            for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x, ++i) {
+            for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
                 const int a = i & 1;
                 // item boundary: the previous accumulator is already handed over; wait for a free one and for
                 // the first chunk
@@ -203,9 +205,9 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                 for (int kb = 0; kb < KB; ++kb, ++g) {
                     const int s = (int)(g % NS);
                     tc_fence_after();
-                    const uint32_t st = stage0 + (uint32_t)s * STAGE;
-                    const uint64_t da1 = umma_desc_k_sw64(st), da2 = umma_desc_k_sw64(st + A_BOX);
-                    const uint64_t db1 = umma_desc_k_sw64(st + 2 * A_BOX), db2 = umma_desc_k_sw64(st + 2 * A_BOX + B_BOX);
+                    // descriptors of stage 0 plus s * STAGE / 16 in the address field (16-byte units)
+                    const uint64_t doff = (uint64_t)(STAGE >> 4) * (uint64_t)s;
+                    const uint64_t da1 = da1_0 + doff, da2 = da2_0 + doff, db1 = db1_0 + doff, db2 = db2_0 + doff;
                     // a k-step (16 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
                     umma_f16_x3(tacc, da1, da2, db1, db2, idesc, kb ? 1u : 0u);
                     if (kb + 1 < KB) mbar_wait_spin(xfull((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
@@ -405,7 +407,18 @@ constexpr int UIMG1 = 128 * 64;                // fp16 image of the U operand: 1
 constexpr int XIMG1 = 256 * 64;                // fp16 image of the X-hat operand: 256 features x 32 data rows
 constexpr int IMG1 = 2 * UIMG1 + 2 * XIMG1;    // U h1, U h2, X h1, X h2: 48 KB
 constexpr int FLUSH1 = 128;                    // stages per accumulation period (4096 rows)
-constexpr int NTH1 = (2 + 4 + 4 * NT1 + 1) * 32;   // U producer, MMA issuer, 4 epilogue, 4 NT1 team warps, X-hat image producer
+constexpr int NTH1 = 16 * 32;
+// Warp roles of the first product.  A warp runs on scheduler (warp index mod 4) and the thread that issues the
+// MMAs executes a serial instruction stream whose speed sets the stage rate, so scheduler 1 hosts only light
+// roles: the issuer (warp 1), one epilogue warp (5; the TMEM lane quarter of a warp is its index mod 4), the
+// two producers (9, 13).  The eight team warps are 0, 2, 3, 8, 10, 11, 12, 14 (15 idles).
+constexpr int W1_ISSUER = 1, W1_EPI0 = 4, W1_UPROD = 9, W1_XPROD = 13;
+__device__ __forceinline__ bool is_team_warp1(int w) { return (w & 3) != 1 && (w >> 2) != 1 && w != 15; }
+__device__ __forceinline__ int team_warp_index1(int w)         // 0 .. 7 over the team warps in increasing order
+{
+    const int q = w >> 2, res = w & 3;
+    return (q == 0 ? 0 : q - 1) * 3 + (res == 0 ? 0 : res - 1);
+}
 
 __global__ void __launch_bounds__(NTH1, 1)
 k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ xT1,
@@ -441,7 +454,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
         abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), 512);
+    if (warp == W1_ISSUER) tmem_alloc(smem_u32(&tmem_base_s), 512);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -464,7 +477,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
     const float sU = ldexpf(1.0f, eU);
     const double unscale = ldexp(1.0, -15 - eU);
 
-    if (warp == 0) {
+    if (warp == W1_UPROD) {
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             for (int g = 0; g < my_stages && !abort_flag; ++g) {
@@ -475,7 +488,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
                 tma_load_2d(raw0 + (uint32_t)s * URAW1, &tmU, c0, row0, ufull(s));
             }
         }
-    } else if (warp == 6 + 4 * NT1) {
+    } else if (warp == W1_XPROD) {
         // ------------------------------ X-hat image producer ------------------------------
         // Its own thread: the image ring is released by the MMAs, the raw U ring by the teams; one thread
         // serving both would let the U loads run only one stage ahead.
@@ -491,21 +504,23 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
                 bulk_load_1d(im + 2 * UIMG1 + XIMG1, xT2 + xoff, xbytes, imgfull(l));
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == W1_ISSUER) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(128, Nb, 0, 0);
             if (my_stages > 0) mbar_wait_spin(imgfull(0), 0, &abort_flag, ctl);
             int l = 0, lph = 0, a = 0, in_period = 0, period = 0;
+            // descriptors of image stage 0; the address field counts 16-byte units, so stage l adds l * IMG1 / 16
+            const uint64_t da1_0 = umma_desc_k_sw64(img0), da2_0 = umma_desc_k_sw64(img0 + UIMG1);
+            const uint64_t db1_0 = umma_desc_k_sw64(img0 + 2 * UIMG1), db2_0 = umma_desc_k_sw64(img0 + 2 * UIMG1 + XIMG1);
             for (int g = 0; g < my_stages; ++g) {
                 if (in_period == 0 && period >= 2) mbar_wait_spin(accfree(a), ((period >> 1) - 1) & 1, &abort_flag, ctl);
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + (uint32_t)(a * 256);
-                const uint32_t im = img0 + (uint32_t)l * IMG1;
                 // K-major images; a k-step of 16 data rows (32 bytes inside the 64-byte swizzled row) advances
                 // the start address by 2
-                const uint64_t da1 = umma_desc_k_sw64(im), da2 = umma_desc_k_sw64(im + UIMG1);
-                const uint64_t db1 = umma_desc_k_sw64(im + 2 * UIMG1), db2 = umma_desc_k_sw64(im + 2 * UIMG1 + XIMG1);
+                const uint64_t doff = (uint64_t)(IMG1 >> 4) * (uint64_t)l;
+                const uint64_t da1 = da1_0 + doff, da2 = da2_0 + doff, db1 = db1_0 + doff, db2 = db2_0 + doff;
                 umma_f16_x3(tacc, da1, da2, db1, db2, idesc, in_period ? 1u : 0u);
                 int ln = l + 1, lphn = lph;
                 if (ln == NIM1) { ln = 0; lphn ^= 1; }
@@ -515,12 +530,11 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
                 if (in_period == FLUSH1 - 1 || g == my_stages - 1) umma_commit(accfull(a));
                 l = ln; lph = lphn;
                 if (++in_period == FLUSH1) { in_period = 0; ++period; a ^= 1; }
-                if (abort_flag) break;
             }
         }
-    } else if (warp >= 6 && warp < 6 + 4 * NT1) {
+    } else if (is_team_warp1(warp)) {
         // ------------------------------ U teams: FP32 slice -> K-major fp16 images ------------------------------
-        const int vw = warp - 6, team = vw >> 2, tw = vw & 3;
+        const int vw = team_warp_index1(warp), team = vw >> 2, tw = vw & 3;
         const int tt = tw * 32 + lane;                     // column of the slice
         for (int g = team; g < my_stages; g += NT1) {
             const int s = g % NRAW1, l = g % NIM1;
@@ -551,8 +565,8 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
                 mbar_arrive(ufree(s));
             }
         }
-    } else {
-        // ------------------------------ epilogue: FP64 fold of the accumulator (warps 2-5) ------------------------------
+    } else if (warp >= W1_EPI0 && warp < W1_EPI0 + 4) {
+        // ------------------------------ epilogue: FP64 fold of the accumulator (warps 4-7) ------------------------------
         // thread = column j of U (TMEM lane); entry (feature f, column j) of this row range's partial
         const int q4 = warp & 3;
         const int j = c0 + q4 * 32 + lane;
@@ -580,7 +594,7 @@ k_pass1_tcg(const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) tmem_dealloc(tmem_base, 512);
+    if (warp == W1_ISSUER) tmem_dealloc(tmem_base, 512);
 }
 
 }  // namespace tcg
