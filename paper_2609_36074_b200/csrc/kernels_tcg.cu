@@ -193,26 +193,32 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
             const uint32_t idesc = umma_idesc_f16(TILE_M, NBLK, 0, 0);
             const uint64_t da1_0 = umma_desc_k_sw64(stage0), da2_0 = umma_desc_k_sw64(stage0 + A_BOX);
             const uint64_t db1_0 = umma_desc_k_sw64(stage0 + 2 * A_BOX), db2_0 = umma_desc_k_sw64(stage0 + 2 * A_BOX + B_BOX);
-            int64_t g = 0;
+            // stage slot and the parity of its current phase, accumulator index and its phase: kept incrementally
+            // in 32-bit registers (this thread's instruction stream is on the critical path)
+            int s = 0;
+            uint32_t ph = 0;
             int i = 0;
             for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
                 const int a = i & 1;
                 // item boundary: the previous accumulator is already handed over; wait for a free one and for
                 // the first chunk
                 if (i >= 2) mbar_wait_spin(accfree(a), (uint32_t)((i >> 1) - 1) & 1, &abort_flag, ctl);
-                mbar_wait_spin(xfull((int)(g % NS)), (uint32_t)(g / NS) & 1, &abort_flag, ctl);
+                mbar_wait_spin(xfull(s), ph, &abort_flag, ctl);
                 const uint32_t tacc = tmem_base + (uint32_t)(a * NBLK);
-                for (int kb = 0; kb < KB; ++kb, ++g) {
-                    const int s = (int)(g % NS);
+                for (int kb = 0; kb < KB; ++kb) {
                     tc_fence_after();
                     // descriptors of stage 0 plus s * STAGE / 16 in the address field (16-byte units)
-                    const uint64_t doff = (uint64_t)(STAGE >> 4) * (uint64_t)s;
+                    const uint64_t doff = (uint64_t)(uint32_t)((STAGE >> 4) * s);
                     const uint64_t da1 = da1_0 + doff, da2 = da2_0 + doff, db1 = db1_0 + doff, db2 = db2_0 + doff;
                     // a k-step (16 features = 32 bytes inside the 64-byte swizzled row) advances the start address by 2
                     umma_f16_x3(tacc, da1, da2, db1, db2, idesc, kb ? 1u : 0u);
-                    if (kb + 1 < KB) mbar_wait_spin(xfull((int)((g + 1) % NS)), (uint32_t)((g + 1) / NS) & 1, &abort_flag, ctl);
+                    int sn = s + 1;
+                    uint32_t phn = ph;
+                    if (sn == NS) { sn = 0; phn ^= 1u; }
+                    if (kb + 1 < KB) mbar_wait_spin(xfull(sn), phn, &abort_flag, ctl);
                     umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
                     umma_commit(xfree(s));
+                    s = sn; ph = phn;
                 }
                 umma_commit(accfull(a));
             }
