@@ -361,11 +361,17 @@ k_pass1_tc(const float* __restrict__ X, const float* __restrict__ U, const __hal
                     for (int k = 0; k < 16; ++k) v[k] += v2[k];
                 }
                 if (j < r) {
+                    // eight old values are requested before the first store: two memory round trips per group
+                    // instead of sixteen dependent ones (the compiler cannot reorder the loads past the
+                    // stores itself), so a fold stays far shorter than an accumulation period
                     double* o = out + (size_t)(c * 16) * r + j;
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const double prev = (period == 0) ? 0.0 : o[(size_t)k * r];
-                        o[(size_t)k * r] = prev + unscale * (double)v[k];
+                    for (int h = 0; h < 16; h += 8) {
+                        double prev[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) prev[k] = (period == 0) ? 0.0 : __ldcg(o + (size_t)(h + k) * r);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) o[(size_t)(h + k) * r] = prev[k] + unscale * (double)v[h + k];
                     }
                 }
             }
