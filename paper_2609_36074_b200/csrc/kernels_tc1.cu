@@ -22,15 +22,16 @@
 // The accumulator is Theta^T: TMEM lane = column j of U (M = 128, columns beyond r are zero), TMEM
 // column = feature f (N = d).
 //
-// One persistent CTA per SM, 14 warps:
-//   warp 0       producer: per stage one bulk copy of the TR rows of U and one of X-hat (contiguous in
-//                global memory).
-//   warps 6-17   vector + split, three teams taking stages round-robin: one warp per row does the row-local
-//                vector work on the U boxes, then both operands are converted into the image ring;
+// One persistent CTA per SM, 20 warps (roles by warp index: see the role constants below):
+//   U producer   per stage one bulk copy of the TR rows of U (contiguous in global memory); without the static
+//                images also of the rows of X-hat.
+//   X producer   per stage the pre-swizzled transposed fp16 image boxes of X-hat, straight into the image stage.
+//   teams        vector + split, three teams of four warps taking stages round-robin: a warp does the row-local
+//                vector work on 8 rows of U, then the operands are converted into the image ring;
 //                the raw stage goes back to the producer as soon as the team has read it.
-//   warp 1       MMA issuer (2 k-steps x 3 products per stage).  Every FLUSH stages the accumulator is
-//                handed to the epilogue and the other TMEM buffer is started from zero.
-//   warps 2-5    epilogue: add each handed-over accumulator, rescaled, into this CTA's FP64 partial of
+//   MMA issuer   2 k-steps x 3 products per stage (2 x 2 with the stacked N = 2 d operand).  Every FLUSH stages
+//                the accumulator is handed to the epilogue and the other TMEM buffer is started from zero.
+//   epilogue     four warps add each handed-over accumulator, rescaled, into this CTA's FP64 partial of
 //                Theta^T (thread = column j of U).
 // Partials have the layout of the FFMA family's first product, so k_red1_fused reduces them.
 // Every mbarrier wait is bounded (GEM_NLR_E_TIMEOUT; the kernel runs to its end and frees its TMEM).
