@@ -215,20 +215,26 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             const uint32_t idesc = F16 ? umma_idesc_f16(TILE_M, NP, 0, 0) : umma_idesc_tf32(TILE_M, NP, 0, 0);
-            mbar_wait(thfull, 0, &abort_flag, ctl);
+            mbar_wait_spin(thfull, 0, &abort_flag, ctl);
             // Inside a tile the wait for the next box sits in the middle of the current box's k-steps, so the
             // tensor pipe has MMAs queued while this thread polls.  F16: the boxes come ready from TMA (xfull);
-            // TF32: from the split warps (xsplit).
+            // TF32: from the split warps (xsplit).  Ring positions and phase parities are kept incrementally in
+            // 32-bit registers and the barrier is polled without suspension: this thread's instruction stream
+            // shares a scheduler with four epilogue warps and sets the rate at which MMAs reach the tensor pipe.
+            int s = 0, l = 0;
+            uint32_t sph = 0;                    // parity of the current fill of box slot s
             int i = 0;
-            for (int64_t t = blockIdx.x; t < n_tiles && !abort_flag; t += gridDim.x, ++i) {
+            for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++i) {
                 const int a = i & 1;
                 // tile boundary: the accumulator hand-over of the previous tile is already committed, so the
                 // epilogue runs while this thread waits for a free accumulator and the first box
-                if (i >= 2) mbar_wait(accfree(a), ((i >> 1) - 1) & 1, &abort_flag, ctl);
-                mbar_wait(F16 ? xfull((i * NB) % NSB) : xsplit((i * NB) % NSB), ((i * NB) / NSB) & 1, &abort_flag, ctl);
+                if (i >= 2) mbar_wait_spin(accfree(a), ((i >> 1) - 1) & 1, &abort_flag, ctl);
+                mbar_wait_spin(F16 ? xfull(s) : xsplit(s), sph, &abort_flag, ctl);
                 const uint32_t tacc = tmem_base + (uint32_t)(a * ACC_COLS);
                 for (int b = 0; b < NB; ++b) {
-                    const int g = i * NB + b, s = g % NSB, l = F16 ? 0 : g % NLO;
+                    int sn = s + 1;
+                    uint32_t sphn = sph;
+                    if (sn == NSB) { sn = 0; sphn ^= 1u; }
                     tc_fence_after();
                     if (F16) {
                         const uint32_t a_h1 = stage0 + (uint32_t)s * BOX_BYTES, a_h2 = a_h1 + BOX_BYTES / 2;
@@ -236,7 +242,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                         const uint64_t da1 = umma_desc_k_sw64(a_h1), da2 = umma_desc_k_sw64(a_h2);
                         const uint64_t db1 = umma_desc_k_sw64(b_h1), db2 = umma_desc_k_sw64(b_h2);
                         umma_f16_x3(tacc, da1, da2, db1, db2, idesc, b ? 1u : 0u);
-                        if (b + 1 < NB) mbar_wait(xfull((g + 1) % NSB), ((g + 1) / NSB) & 1, &abort_flag, ctl);
+                        if (b + 1 < NB) mbar_wait_spin(xfull(sn), sphn, &abort_flag, ctl);
                         umma_f16_x3(tacc, da1 + 2, da2 + 2, db1 + 2, db2 + 2, idesc, 1u);
                         umma_commit(xfree(s));
                     } else {
@@ -248,13 +254,15 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                         const uint64_t db_hi = umma_desc_sw128(b_hi, 16, 1024), db_lo = umma_desc_sw128(b_lo, 16, 1024);
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {
-                            if (ks == 2 && b + 1 < NB) mbar_wait(xsplit((g + 1) % NSB), ((g + 1) / NSB) & 1, &abort_flag, ctl);
+                            if (ks == 2 && b + 1 < NB) mbar_wait_spin(xsplit(sn), sphn, &abort_flag, ctl);
                             umma_tf32_x3(tacc, da_hi + 2 * ks, da_lo + 2 * ks, db_hi + 2 * ks, db_lo + 2 * ks, idesc,
                                          (b | ks) ? 1u : 0u);
                         }
                         umma_commit(xfree(s));
                         umma_commit(lofree(l));
+                        if (++l == NLO) l = 0;
                     }
+                    s = sn; sph = sphn;
                 }
                 umma_commit(accfull(a));
             }
