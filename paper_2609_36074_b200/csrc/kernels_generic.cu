@@ -620,10 +620,12 @@ k_labels_wide(const float* __restrict__ U, int64_t n, int r, int32_t* __restrict
                 u[i][k] = (c4 < r4 && row0 + i < n) ? __ldcs(reinterpret_cast<const float4*>(U + (row0 + i) * r) + c4)
                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+        float bv[ROWS];
+        int best[ROWS];
 #pragma unroll
         for (int i = 0; i < ROWS; ++i) {
-            float bv = -INFINITY;
-            int best = 0x7fffffff;
+            bv[i] = -INFINITY;
+            best[i] = 0x7fffffff;
 #pragma unroll
             for (int k = 0; k < NK; ++k) {
                 const int c4 = lane + 32 * k;
@@ -631,16 +633,45 @@ k_labels_wide(const float* __restrict__ U, int64_t n, int r, int32_t* __restrict
                     const float v[4] = {u[i][k].x, u[i][k].y, u[i][k].z, u[i][k].w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        if (v[e] > bv) { bv = v[e]; best = 4 * c4 + e; }
+                        if (v[e] > bv[i]) { bv[i] = v[e]; best[i] = 4 * c4 + e; }
+                }
+            }
+        }
+        auto merge = [](float& v, int& b, float ov, int ob) {
+            if (ov > v || (ov == v && ob < b)) { v = ov; b = ob; }
+        };
+        if constexpr (ROWS == 8) {
+            // the eight rows' candidates by recursive halving: after the exchanges over lane bits 4, 3, 2 a lane
+            // holds the candidate of row 4 (bit 4) + 2 (bit 3) + (bit 2) over its 4-lane group's share
+#pragma unroll
+            for (int lvl = 0; lvl < 3; ++lvl) {
+                const int o = 16 >> lvl, m = 4 >> lvl;                 // lane bit, candidates kept
+                const bool up = lane & o;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (i < m) {
+                        const float sv = up ? bv[i] : bv[i + m];
+                        const int sb = up ? best[i] : best[i + m];
+                        float kv = up ? bv[i + m] : bv[i];
+                        int kb = up ? best[i + m] : best[i];
+                        merge(kv, kb, __shfl_xor_sync(0xffffffffu, sv, o), __shfl_xor_sync(0xffffffffu, sb, o));
+                        bv[i] = kv; best[i] = kb;
+                    }
                 }
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                const int ob = __shfl_xor_sync(0xffffffffu, best, o);
-                if (ov > bv || (ov == bv && ob < best)) { bv = ov; best = ob; }
+            for (int o = 2; o > 0; o >>= 1)
+                merge(bv[0], best[0], __shfl_xor_sync(0xffffffffu, bv[0], o), __shfl_xor_sync(0xffffffffu, best[0], o));
+            const int row_l = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+            if ((lane & 3) == 0 && row0 + row_l < n) labels[row0 + row_l] = best[0];
+        } else {
+#pragma unroll
+            for (int i = 0; i < ROWS; ++i) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1)
+                    merge(bv[i], best[i], __shfl_xor_sync(0xffffffffu, bv[i], o), __shfl_xor_sync(0xffffffffu, best[i], o));
+                if (lane == 0 && row0 + i < n) labels[row0 + i] = best[i];
             }
-            if (lane == 0 && row0 + i < n) labels[row0 + i] = best;
         }
     }
 }

@@ -232,6 +232,15 @@ def test_labels_tie_break_and_wide_rows():
         s = gem.GemNlr(Xd, torch.from_numpy(Ur).cuda(), 2)
         assert np.array_equal(s.labels().cpu().numpy(), oracle.labels(Ur))
         s.destroy()
+    # every read-out kernel (thread per row with 16-byte loads; warp per 8 / 4 / 2 / 1 rows; the scalar fallback),
+    # ragged row counts, many ties
+    for n, r in ((1003, 16), (1003, 32), (517, 100), (1001, 128), (301, 200), (203, 300), (77, 1000), (50, 1030)):
+        Ur = rng.integers(0, 3, size=(n, r)).astype(np.float32)
+        Ur[n // 2] = 1.0
+        Xd = torch.zeros(n, 4, device="cuda")
+        s = gem.GemNlr(Xd, torch.from_numpy(Ur).cuda(), 2)
+        assert np.array_equal(s.labels().cpu().numpy(), oracle.labels(Ur)), (n, r)
+        s.destroy()
 
 
 def test_host_buffer_job_matches_device_job():
