@@ -54,13 +54,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait.  abort_flag lives in shared memory and is shared by the whole CTA.
+// Bounded wait.  abort_flag lives in shared memory and is shared by the whole CTA; it is looked at only after
+// a failed attempt (every 64th), so the common case -- the phase is already complete -- costs one instruction.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                           Ctl* ctl)
 {
-    if (*abort_flag) return;
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return;
+        if ((i & 63u) == 63u && *abort_flag) return;
+    }
     *abort_flag = 1u;
     ctl->status = GEM_NLR_E_TIMEOUT;
     ctl->stopped = 1;
