@@ -559,13 +559,33 @@ int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U
     int32_t* Ld = (int32_t*)((char*)Ud + align_up(4 * n * P.r, 256));
     char* ws = (char*)Ld + align_up(4 * n, 256);
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemcpyAsync(Xd, X_host, 4 * n * P.d, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(Ud, U_host, 4 * n * P.r, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // X goes first on the caller's stream; the starting factor follows on a side stream once X has arrived, so that
+    // its transfer overlaps the setup (mean, power iteration, normalization, images), which needs X only.
+    cudaStream_t side = nullptr;
+    cudaEvent_t x_there = nullptr, u_there = nullptr;
+    if (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&x_there, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&u_there, cudaEventDisableTiming) != cudaSuccess) {
+        if (side) cudaStreamDestroy(side);
+        if (x_there) cudaEventDestroy(x_there);
         return GEM_NLR_E_CUDA;
+    }
+    auto release = [&]() { cudaStreamDestroy(side); cudaEventDestroy(x_there); cudaEventDestroy(u_there); };
+    if (cudaMemcpyAsync(Xd, X_host, 4 * n * P.d, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaEventRecord(x_there, st) != cudaSuccess ||
+        cudaStreamWaitEvent(side, x_there, 0) != cudaSuccess ||
+        cudaMemcpyAsync(Ud, U_host, 4 * n * P.r, cudaMemcpyHostToDevice, side) != cudaSuccess ||
+        cudaEventRecord(u_there, side) != cudaSuccess) {
+        cudaStreamSynchronize(side);
+        release();
+        return GEM_NLR_E_CUDA;
+    }
     gem_nlr_t* h = nullptr;
     int rc = gem_nlr_create(&h, &P, Xd, Ud, ws, make_layout(P).total, cuda_stream);
-    if (rc < 0) return rc;
+    if (rc < 0) { cudaStreamSynchronize(side); release(); return rc; }
     rc = gem_nlr_spectral_norm(h, a_out);
+    // nothing before this point touches U; the iterations wait for it on the caller's stream
+    if (cudaStreamWaitEvent(st, u_there, 0) != cudaSuccess) rc = GEM_NLR_E_CUDA;
     int run_rc = rc;
     if (rc >= 0) run_rc = gem_nlr_run(h, last, iters_done);
     if (run_rc >= 0 || run_rc == GEM_NLR_E_BREAKDOWN) {
@@ -579,6 +599,8 @@ int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U
         if (cudaStreamSynchronize(st) != cudaSuccess) run_rc = GEM_NLR_E_CUDA;
     }
     gem_nlr_destroy(h);
+    cudaStreamSynchronize(side);
+    release();
     return run_rc;
 }
 
