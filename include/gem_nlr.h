@@ -155,7 +155,10 @@ int gem_nlr_history(gem_nlr_t *h, gem_nlr_iter_info *records_host, int32_t max_r
  * which: 0 Theta (d*r floats), 1 p (r), 2 s (r), 3 ytilde (n), 4 ybar (n), 5 X-hat (n*d).      */
 int gem_nlr_buffer(gem_nlr_t *h, int32_t which, void **ptr_dev);
 
-/* Name of the kernel family chosen for the two contractions ("generic", "ffma", "tf32x3").     */
+/* Name of the kernel family chosen for the two contractions: "generic", "ffma", "mma.tf32x3",
+ * "f16x3" (tcgen05, fp16 split, both products), "f16x3.tiled" (the same for r > 256), or
+ * "first+second" when the two products come from different families, e.g. "generic+f16x3",
+ * "generic+f16x3.tiled", "f16x3+tf32x3".  The string is static.                                  */
 const char *gem_nlr_path(gem_nlr_t *h);
 
 /* Text of the last CUDA error seen by this handle ("" if none).                                */
