@@ -140,6 +140,68 @@ def test_movement_identity_matches_direct_norm():
         assert abs(info["a"] - np.sum(W ** 2)) <= 1e-6 * info["a"]
         assert abs(info["h"] - np.sum(W * Uprev)) <= 1e-6 * abs(info["h"])
         assert abs(info["c"] - float(np.float32(np.sqrt(4 / info["a"])))) <= 2e-7 * info["c"]
+        # Section 4.3: rho = ||q||_2 / sqrt(n), with q = U p - 1 taken from the NEW factor
+        Unew = st.U.astype(np.float64)
+        q_direct = Unew @ Unew.sum(0) - 1.0
+        rho_direct = np.linalg.norm(q_direct) / np.sqrt(200)
+        assert abs(info["rho"] - rho_direct) <= 1e-6 * rho_direct
+        assert abs(info["rho"] - np.linalg.norm(st.q.astype(np.float64)) / np.sqrt(200)) <= 1e-12 * info["rho"]
+
+
+def _trajectory_with_gate_crossing(eps_d, eps_c, T_min, iters=400):
+    spec = dataclasses.replace(synth.config(1).with_n(400), seed=1)
+    X, _, _ = synth.make_mixture(spec)
+    hp = synth.default_hparams(spec.K)
+    Xhat, _, _ = oracle.normalize(X)
+    st = oracle.State(Xhat, synth.make_u0(spec.n, spec.K, spec.K, seed=1))
+    out = []
+    for t in range(iters):
+        Uprev = st.U.astype(np.float64).copy()
+        yprev = st.ytilde.copy()
+        info = st.step(spec.K, hp["alpha"], hp["beta"], eps_d, eps_c, T_min)
+        assert info["status"] == 0 and info["t"] == t
+        direct = np.linalg.norm(st.U.astype(np.float64) - Uprev) / np.sqrt(spec.K)
+        out.append((t, info, direct, not np.array_equal(yprev, st.ytilde)))
+        if info["stop"]:
+            break
+    return out
+
+
+def test_dual_gate_is_the_main_text_test_on_the_movement():
+    """Section 4.3: the dual ascent fires exactly when delta-hat < eps_d. The comparison is made
+    here on delta-hat itself (and on the directly computed movement), not on the squared form the
+    oracle evaluates, over a trajectory that crosses the threshold."""
+    eps_d = 0.05
+    traj = _trajectory_with_gate_crossing(eps_d, eps_c=1e-4, T_min=10)
+    seen = set()
+    for t, info, direct, y_changed in traj:
+        if abs(direct - eps_d) > 1e-5:                       # away from the rounding edge
+            assert info["dual"] == int(direct < eps_d), (t, direct)
+        assert info["dual"] == int(info["delta_hat"] < eps_d), (t, info["delta_hat"])
+        assert y_changed == bool(info["dual"])               # y-tilde moves only through the gate
+        seen.add(info["dual"])
+    assert seen == {0, 1}
+    # a wrong power of eps_d or of K in the threshold would open the gate at another iteration
+    first_open = next(t for t, info, _, _ in traj if info["dual"])
+    assert first_open > 0 and traj[first_open - 1][2] >= eps_d > traj[first_open][2]
+
+
+@pytest.mark.parametrize("T_min", [1, 10, 10 ** 6])
+def test_stop_predicate_is_algorithm_1_break_line(T_min):
+    """Algorithm 1's break: delta-hat < min(eps_d, eps_c), rho < eps_c and t + 1 >= T_min."""
+    eps_d, eps_c = 0.05, 1e-4
+    base = _trajectory_with_gate_crossing(eps_d, eps_c, T_min=1)
+    t_ready = base[-1][0]                                     # first iteration whose tests all pass
+    assert base[-1][1]["stop"] == 1 and t_ready + 1 > 1
+    if T_min == 10 ** 6:
+        T_min = t_ready + 3                                   # delays an otherwise-ready stop
+    traj = _trajectory_with_gate_crossing(eps_d, eps_c, T_min, iters=t_ready + 10)
+    for t, info, direct, _ in traj:
+        want = info["delta_hat"] < min(eps_d, eps_c) and info["rho"] < eps_c and t + 1 >= T_min
+        assert info["stop"] == int(want), (t, info)
+    last_t = traj[-1][0]
+    assert traj[-1][1]["stop"] == 1
+    assert last_t + 1 >= T_min and last_t == max(t_ready, T_min - 1)
 
 
 def test_descent_inequality_with_fixed_dual():
