@@ -4,7 +4,8 @@ tiny benchmark shape (config 1: n = 2000, d = 16, K = 4, seed 0) and a digest of
 The paper prints no worked numerical example, so these stored values are not the paper's: they come
 from the CPU oracle alone (this script imports nothing but `oracle` and the input generators) and
 serve two purposes: a change of the oracle's arithmetic shows up as a diff of this file, and the GPU
-path is compared with values that were fixed before it ran.
+path is compared with stored values that no GPU run can alter (the file was written after the first
+kernels existed; it pins the oracle against drift, it is not a pin of the oracle itself).
 
     python tests/golden/make_golden.py
 """

@@ -1,6 +1,7 @@
 """Stored trajectory of the tiny benchmark shape (tests/golden/tiny_trajectory.txt, written by
 tests/golden/make_golden.py from the CPU oracle alone): the oracle must still reproduce it, and the GPU
-path must match values that were fixed before it ran."""
+path must match these stored values, which only the oracle can write (a guard against drift of either
+side, not an independent pin of the oracle)."""
 import hashlib
 import importlib.util
 import os
