@@ -49,7 +49,10 @@ extern "C" {
 #define GEM_NLR_E_BREAKDOWN  -4   /* sqrt(a) <= 1e-20: W vanished (Algorithm 1, breakdown line)   */
 #define GEM_NLR_E_NONFINITE  -5   /* a, b or h is not finite                                     */
 #define GEM_NLR_E_NOT_READY  -6   /* iteration requested before X was normalized                 */
-#define GEM_NLR_E_TIMEOUT    -7   /* a bounded device-side wait (copy pipeline) ran out          */
+#define GEM_NLR_E_TIMEOUT    -7   /* a bounded device-side wait (copy pipeline) ran out; the     */
+                                  /* kernel ran to its end without the data it waited for, so    */
+                                  /* U_dev and the dual are undefined afterwards: reload them    */
+                                  /* (gem_nlr_set_state) before iterating again                  */
 #define GEM_NLR_E_TOO_LARGE  -8   /* size beyond the fixed capacity of a *_static entry point    */
 
 typedef struct gem_nlr gem_nlr_t;   /* opaque handle */
@@ -135,7 +138,13 @@ int gem_nlr_step(gem_nlr_t *h, gem_nlr_iter_info *info);
 int gem_nlr_run(gem_nlr_t *h, gem_nlr_iter_info *last, int32_t *iters_done);
 
 /* label_i = smallest j with U_ij = max_j U_ij (an all-zero row gets 0).  labels_dev: n int32.
- * Enqueued on the handle's stream; does not synchronize.                                       */
+ * Enqueued on the handle's stream; does not synchronize.
+ * This row argmax is this library's read-out, not the paper's (its appendix on rounding takes the top-K
+ * left singular vectors of U and runs K-means on the embedded rows).  It names clusters only for
+ * r == K: at an exact solution U U^T is block diagonal with U >= 0, so rows of different clusters have
+ * disjoint supports and each of the K clusters owns exactly one of the K columns.  For r > K a cluster
+ * may own several columns, and the argmax then splits it: the labels are still the row argmax, but they
+ * are column indices, not cluster indices.                                                       */
 int gem_nlr_labels(gem_nlr_t *h, int32_t *labels_dev);
 
 /* f-hat_y(U) of Eq. "normalized" at the current (U, y).  Synchronizes.                         */
@@ -188,6 +197,19 @@ int gem_nlr_run_host(const gem_nlr_params *params, const float *X_host, float *U
                      void *cuda_stream, double *a_out, gem_nlr_iter_info *last,
                      int32_t *iters_done);
 
+/* The same job with a per-phase record (a measurement helper; the paper has no counterpart).
+ * phase_ms_out: 5 doubles of host memory (may be NULL), filled from CUDA events on cuda_stream when the
+ * job succeeds: [0] host-to-device copy of X; [1] setup (mean, spectral norm, normalization, operand
+ * images), which overlaps the copy of the starting factor; [2] the iterations, including any wait for
+ * the starting factor's copy; [3] label read-out and the device-to-host copies of U and the labels;
+ * [4] the whole job from the first copy to the last.  Host-side work between the phases (handle
+ * creation, the read-backs of the setup) is inside [1] and [2]; what the caller measures around the
+ * call beyond [4] is host overhead (stream, event and pinned-record creation, their release).     */
+int gem_nlr_run_host_timed(const gem_nlr_params *params, const float *X_host, float *U_host,
+                           int32_t *labels_host, void *device_buffer_dev, size_t device_bytes,
+                           void *cuda_stream, double *a_out, gem_nlr_iter_info *last,
+                           int32_t *iters_done, double *phase_ms_out);
+
 /* Column sums without any allocation: p_dev[j] = sum_i U_dev[i * r + j], j < r (FP64 sums in a
  * fixed order, rounded once to FP32) -- the p = U^T 1 of the iteration, for a factor the caller
  * holds.  The paper has no counterpart of this entry point; it exists for callers that cannot
@@ -205,7 +227,12 @@ int gem_nlr_run_host(const gem_nlr_params *params, const float *X_host, float *U
  * nothing is launched.  n is not limited.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
- * that device current); make that first call before any stream capture begins.  All calls share
+ * that device current).  With CUDA's lazy module loading this is also the moment the driver loads
+ * this entry point's module and places the array, which may synchronize the device and can fail if
+ * the device has no memory left: make that first call once at start-up, as a warm-up, before any
+ * stream capture begins and before memory runs short.  The device that cuda_stream belongs to must
+ * be the current device on every call (the scratch address and the launch follow the current
+ * device).  All calls share
  * the one array and it keeps the previous call's partial sums: every call overwrites what it
  * reads, so nothing needs clearing, but two calls whose kernels overlap on the GPU (different
  * streams without an ordering between them) race on it -- order them.

@@ -73,6 +73,9 @@ def lib():
         L.gem_nlr_host_job_device_bytes.restype = C.c_size_t
         L.gem_nlr_run_host.argtypes = [pp, vp, vp, vp, vp, C.c_size_t, vp, C.POINTER(C.c_double),
                                        C.POINTER(IterInfo), C.POINTER(C.c_int32)]
+        L.gem_nlr_run_host_timed.argtypes = [pp, vp, vp, vp, vp, C.c_size_t, vp, C.POINTER(C.c_double),
+                                             C.POINTER(IterInfo), C.POINTER(C.c_int32), C.POINTER(C.c_double)]
+        L.gem_nlr_run_host_timed.restype = C.c_int
         L.gem_nlr_profile.argtypes = [vp, C.c_int32]
         L.gem_nlr_profile.restype = C.c_int
         L.gem_nlr_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -221,8 +224,10 @@ class GemNlr:
             raise RuntimeError(f"gem_nlr call failed: {rc} {self.last_error()}")
 
 
-def run_host(X_host, U_host, K, device_buffer, stream=None, want_labels=True, **kw):
-    """gem_nlr_run_host: numpy/pinned-torch host arrays in, U (in place) and labels out."""
+def run_host(X_host, U_host, K, device_buffer, stream=None, want_labels=True, labels=None, phase_ms=None, **kw):
+    """gem_nlr_run_host: numpy/pinned-torch host arrays in, U (in place) and labels out.  `labels` may be a
+    caller-provided host array (n int32); `phase_ms`, a list, receives the five per-phase device times of
+    gem_nlr_run_host_timed."""
     import numpy as np
     import torch
     n, d = X_host.shape
@@ -234,15 +239,19 @@ def run_host(X_host, U_host, K, device_buffer, stream=None, want_labels=True, **
     def ptr(x):
         return x.ctypes.data if isinstance(x, np.ndarray) else x.data_ptr()
 
-    labels = None
-    if want_labels:
+    if want_labels and labels is None:
         labels = (np.empty(n, np.int32) if isinstance(X_host, np.ndarray)
                   else torch.empty(n, dtype=torch.int32, pin_memory=True))
     a, info, iters = C.c_double(), IterInfo(), C.c_int32()
-    rc = lib().gem_nlr_run_host(C.byref(params), ptr(X_host), ptr(U_host),
-                                ptr(labels) if labels is not None else None,
-                                device_buffer.data_ptr(), device_buffer.numel() * device_buffer.element_size(),
-                                st.cuda_stream, C.byref(a), C.byref(info), C.byref(iters))
+    args = (C.byref(params), ptr(X_host), ptr(U_host), ptr(labels) if labels is not None else None,
+            device_buffer.data_ptr(), device_buffer.numel() * device_buffer.element_size(),
+            st.cuda_stream, C.byref(a), C.byref(info), C.byref(iters))
+    if phase_ms is None:
+        rc = lib().gem_nlr_run_host(*args)
+    else:
+        ph = (C.c_double * 5)()
+        rc = lib().gem_nlr_run_host_timed(*args, ph)
+        phase_ms[:] = list(ph)
     return rc, labels, a.value, info.as_dict(), iters.value
 
 
@@ -256,6 +265,8 @@ def column_sums_static(U, out=None, stream=None):
     n, r = U.shape
     if out is None:
         out = torch.empty(r, dtype=torch.float32, device=U.device)
+    assert out.is_cuda and out.device == U.device and out.dtype == torch.float32 and out.numel() >= r
     st = stream if stream is not None else torch.cuda.current_stream(U.device)
-    rc = lib().gem_nlr_column_sums_static(U.data_ptr(), int(n), int(r), out.data_ptr(), st.cuda_stream)
+    with torch.cuda.device(U.device):          # the entry point works on the current device
+        rc = lib().gem_nlr_column_sums_static(U.data_ptr(), int(n), int(r), out.data_ptr(), st.cuda_stream)
     return rc, out

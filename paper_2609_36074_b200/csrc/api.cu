@@ -547,6 +547,15 @@ int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U
                      int32_t* labels_host, void* device_buffer_dev, size_t device_bytes,
                      void* cuda_stream, double* a_out, gem_nlr_iter_info* last, int32_t* iters_done)
 {
+    return gem_nlr_run_host_timed(params, X_host, U_host, labels_host, device_buffer_dev, device_bytes, cuda_stream,
+                                  a_out, last, iters_done, nullptr);
+}
+
+int gem_nlr_run_host_timed(const gem_nlr_params* params, const float* X_host, float* U_host,
+                           int32_t* labels_host, void* device_buffer_dev, size_t device_bytes,
+                           void* cuda_stream, double* a_out, gem_nlr_iter_info* last, int32_t* iters_done,
+                           double* phase_ms_out)
+{
     if (!params || !X_host || !U_host || !device_buffer_dev) return GEM_NLR_E_INVALID;
     if (!valid_params(*params) || ((uintptr_t)device_buffer_dev & 255)) return GEM_NLR_E_INVALID;
     if (device_bytes < gem_nlr_host_job_device_bytes(params)) return GEM_NLR_E_WORKSPACE;
@@ -563,14 +572,26 @@ int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U
     // its transfer overlaps the setup (mean, power iteration, normalization, images), which needs X only.
     cudaStream_t side = nullptr;
     cudaEvent_t x_there = nullptr, u_there = nullptr;
+    cudaEvent_t tev[4] = {nullptr, nullptr, nullptr, nullptr};   // job start, setup done, iterations done, copies done
+    if (phase_ms_out) {
+        for (int i = 0; i < 5; ++i) phase_ms_out[i] = 0.0;
+        for (int i = 0; i < 4; ++i)
+            if (cudaEventCreate(&tev[i]) != cudaSuccess) {
+                for (int k = 0; k < i; ++k) cudaEventDestroy(tev[k]);
+                return GEM_NLR_E_CUDA;
+            }
+    }
+    auto release_tev = [&]() { for (int i = 0; i < 4; ++i) if (tev[i]) cudaEventDestroy(tev[i]); };
     if (cudaStreamCreateWithFlags(&side, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaEventCreateWithFlags(&x_there, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&x_there, phase_ms_out ? cudaEventDefault : cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&u_there, cudaEventDisableTiming) != cudaSuccess) {
         if (side) cudaStreamDestroy(side);
         if (x_there) cudaEventDestroy(x_there);
+        release_tev();
         return GEM_NLR_E_CUDA;
     }
-    auto release = [&]() { cudaStreamDestroy(side); cudaEventDestroy(x_there); cudaEventDestroy(u_there); };
+    auto release = [&]() { cudaStreamDestroy(side); cudaEventDestroy(x_there); cudaEventDestroy(u_there); release_tev(); };
+    if (tev[0]) cudaEventRecord(tev[0], st);
     if (cudaMemcpyAsync(Xd, X_host, 4 * n * P.d, cudaMemcpyHostToDevice, st) != cudaSuccess ||
         cudaEventRecord(x_there, st) != cudaSuccess ||
         cudaStreamWaitEvent(side, x_there, 0) != cudaSuccess ||
@@ -584,10 +605,12 @@ int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U
     int rc = gem_nlr_create(&h, &P, Xd, Ud, ws, make_layout(P).total, cuda_stream);
     if (rc < 0) { cudaStreamSynchronize(side); release(); return rc; }
     rc = gem_nlr_spectral_norm(h, a_out);
+    if (tev[1]) cudaEventRecord(tev[1], st);
     // nothing before this point touches U; the iterations wait for it on the caller's stream
     if (cudaStreamWaitEvent(st, u_there, 0) != cudaSuccess) rc = GEM_NLR_E_CUDA;
     int run_rc = rc;
     if (rc >= 0) run_rc = gem_nlr_run(h, last, iters_done);
+    if (tev[2]) cudaEventRecord(tev[2], st);
     if (run_rc >= 0 || run_rc == GEM_NLR_E_BREAKDOWN) {
         if (labels_host) {
             gem_nlr_labels(h, Ld);
@@ -596,7 +619,16 @@ int gem_nlr_run_host(const gem_nlr_params* params, const float* X_host, float* U
         }
         if (cudaMemcpyAsync(U_host, Ud, 4 * n * P.r, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             run_rc = GEM_NLR_E_CUDA;
+        if (tev[3]) cudaEventRecord(tev[3], st);
         if (cudaStreamSynchronize(st) != cudaSuccess) run_rc = GEM_NLR_E_CUDA;
+        if (phase_ms_out && run_rc >= 0) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, tev[0], x_there) == cudaSuccess) phase_ms_out[0] = ms;
+            if (cudaEventElapsedTime(&ms, x_there, tev[1]) == cudaSuccess) phase_ms_out[1] = ms;
+            if (cudaEventElapsedTime(&ms, tev[1], tev[2]) == cudaSuccess) phase_ms_out[2] = ms;
+            if (cudaEventElapsedTime(&ms, tev[2], tev[3]) == cudaSuccess) phase_ms_out[3] = ms;
+            if (cudaEventElapsedTime(&ms, tev[0], tev[3]) == cudaSuccess) phase_ms_out[4] = ms;
+        }
     }
     gem_nlr_destroy(h);
     cudaStreamSynchronize(side);

@@ -158,7 +158,7 @@ k_pi_fin(const double* __restrict__ part, int g, int d, double* __restrict__ w)
 
 // X-hat = FP32((X - mean) * (1/a)), evaluated in FP64.
 __global__ void __launch_bounds__(256)
-k_normalize(const float* __restrict__ X, float* __restrict__ Xhat, int64_t total, int d,
+k_normalize(const float* X, float* Xhat, int64_t total, int d,
             const double* __restrict__ mean, double inv_a)
 {
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

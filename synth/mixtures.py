@@ -93,11 +93,13 @@ def _workers() -> int:
     return max(1, min(16, os.cpu_count() or 1))
 
 
-def make_mixture(spec: MixtureSpec, out: np.ndarray | None = None):
+def make_mixture(spec: MixtureSpec, out: np.ndarray | None = None, rows: int | None = None):
     """Return (X, labels, centres): X is n x d float32 row-major, labels int32.
 
     Labels are contiguous blocks of the cluster sizes followed by a seeded row
     shuffle, so cluster membership is spread over the whole row range.
+    With `rows` only the leading rows of the same problem are generated (X and
+    labels are cut to `rows`; the values equal those of the full problem).
     """
     n, d, K = spec.n, spec.d, spec.K
     head = np.random.default_rng([spec.seed, 0])
@@ -111,6 +113,9 @@ def make_mixture(spec: MixtureSpec, out: np.ndarray | None = None):
         sigma = np.ones(K, dtype=np.float32)
     labels = np.repeat(np.arange(K, dtype=np.int32), sizes)
     np.random.default_rng([spec.seed, 1]).shuffle(labels)
+    if rows is not None:
+        n = min(n, int(rows))
+        labels = labels[:n]
     X = out if out is not None else np.empty((n, d), dtype=np.float32)
     assert X.shape == (n, d) and X.dtype == np.float32 and X.flags.c_contiguous
 
