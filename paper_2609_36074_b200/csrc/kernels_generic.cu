@@ -368,7 +368,15 @@ k_fin1(Ctl* __restrict__ ctl, const double* __restrict__ part1v, int gv, const d
     __shared__ double sred[32];
     for (int j = threadIdx.x; j < r; j += blockDim.x) {
         double v = 0.0;
-        for (int b = 0; b < gv; ++b) v += part1v[(size_t)b * (r + 2) + j];
+        int b = 0;
+        for (; b + 8 <= gv; b += 8) {             // eight records requested at once, added in record order
+            double t[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) t[k] = __ldcg(part1v + (size_t)(b + k) * (r + 2) + j);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v += t[k];
+        }
+        for (; b < gv; ++b) v += __ldcg(part1v + (size_t)b * (r + 2) + j);
         float sf = (float)v;
         s[j] = sf;
         alpha_s[j] = alpha * sf;
