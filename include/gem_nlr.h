@@ -187,6 +187,17 @@ int gem_nlr_profile_read(gem_nlr_t *h, double *ms_first_phase, double *ms_second
                          int64_t *iterations);
 int64_t gem_nlr_launch_count(gem_nlr_t *h);
 
+/* Self-test of the failure path that a healthy run never takes (no counterpart in the paper): every wait of
+ * the copy / tensor-core pipelines is bounded, and when one runs out the kernel records GEM_NLR_E_TIMEOUT
+ * and runs to its end instead of hanging.  This call launches a one-CTA kernel that waits, through the same
+ * device code, on a barrier nothing arrives on, giving up after max_polls polls (1 .. 2^20), and then waits
+ * once more with the production limit, which must return at once.  It returns GEM_NLR_E_TIMEOUT when the
+ * path works (GEM_NLR_OK would mean the wait never ran out); the handle keeps that error, as after a real
+ * time-out, and refuses further iterations until gem_nlr_set_state reloads the factor and the dual.
+ * cycles_out (2 entries of host memory, may be NULL): SM clock cycles spent in the two waits.
+ * Nothing faults, traps or spins without bound.  Synchronizes.                                     */
+int gem_nlr_selftest_wait_timeout(gem_nlr_t *h, uint32_t max_polls, int64_t *cycles_out);
+
 /* Whole job with HOST buffers: copies X_host and U_host to device_buffer_dev, runs setup, up to
  * T iterations and the label read-out, and copies U (into U_host) and the labels back.
  * device_buffer_dev must hold gem_nlr_host_job_device_bytes(params) bytes (256-byte aligned).

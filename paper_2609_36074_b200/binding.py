@@ -82,6 +82,8 @@ def lib():
         L.gem_nlr_profile_read.restype = C.c_int
         L.gem_nlr_launch_count.argtypes = [vp]
         L.gem_nlr_launch_count.restype = C.c_int64
+        L.gem_nlr_selftest_wait_timeout.argtypes = [vp, C.c_uint32, C.POINTER(C.c_int64)]
+        L.gem_nlr_selftest_wait_timeout.restype = C.c_int
         L.gem_nlr_column_sums_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp]
         L.gem_nlr_column_sums_static.restype = C.c_int
         for name in ("create", "spectral_norm", "set_normalized", "step", "run", "labels", "objective",
@@ -198,6 +200,12 @@ class GemNlr:
         a, b, n = C.c_double(), C.c_double(), C.c_int64()
         self._check(lib().gem_nlr_profile_read(self._h, C.byref(a), C.byref(b), C.byref(n)))
         return a.value, b.value, n.value
+
+    def selftest_wait_timeout(self, max_polls: int = 1024):
+        """gem_nlr_selftest_wait_timeout: returns (rc, cycles of the wait that runs out, cycles of the wait after it)."""
+        cyc = (C.c_int64 * 2)()
+        rc = lib().gem_nlr_selftest_wait_timeout(self._h, int(max_polls), cyc)
+        return rc, int(cyc[0]), int(cyc[1])
 
     def launch_count(self) -> int:
         return int(lib().gem_nlr_launch_count(self._h))

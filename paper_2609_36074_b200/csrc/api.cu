@@ -533,6 +533,22 @@ int gem_nlr_profile_read(gem_nlr_t* h, double* ms_first_phase, double* ms_second
 
 int64_t gem_nlr_launch_count(gem_nlr_t* h) { return h ? h->launches : 0; }
 
+int gem_nlr_selftest_wait_timeout(gem_nlr_t* h, uint32_t max_polls, int64_t* cycles_out)
+{
+    if (!h || max_polls < 1 || max_polls > (1u << 20)) return GEM_NLR_E_INVALID;
+    if (h->sticky_error) return h->sticky_error;
+    // two counters at the end of the (otherwise unused between iterations) setup scratch
+    long long* cyc = reinterpret_cast<long long*>(h->pb.setup());
+    CK(h, cudaMemsetAsync(cyc, 0, 2 * sizeof(long long), h->pb.stream));
+    launch_selftest_wait(h->pb, max_polls, cyc);
+    long long host_cyc[2] = {0, 0};
+    CK(h, cudaMemcpyAsync(host_cyc, cyc, sizeof(host_cyc), cudaMemcpyDeviceToHost, h->pb.stream));
+    int rc = read_ctl(h);
+    if (rc) return rc;
+    if (cycles_out) { cycles_out[0] = host_cyc[0]; cycles_out[1] = host_cyc[1]; }
+    return result_code(h, false);
+}
+
 size_t gem_nlr_host_job_device_bytes(const gem_nlr_params* params)
 {
     if (!params || !valid_params(*params)) return 0;

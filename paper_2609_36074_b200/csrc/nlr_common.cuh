@@ -98,6 +98,9 @@ void launch_tail(const Problem& pb);
 void launch_objective(const Problem& pb);                   // fills ctl->f_final for the current (U, y)
 void launch_labels(const Problem& pb, int32_t* labels);
 
+// ---- self-test of the bounded waits (selftest.cu) ------------------------------------------
+void launch_selftest_wait(const Problem& pb, uint32_t max_polls, long long* cycles_dev /* 2 entries */);
+
 // ---- setup (Section 3) -------------------------------------------------------------------
 // Returns a negative GEM_NLR_E_* or 0; writes a to *a_out.  Synchronizes the stream.
 int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, double* a_out,

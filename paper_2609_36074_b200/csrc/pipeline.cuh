@@ -56,16 +56,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 
 // Bounded wait.  abort_flag lives in shared memory and is shared by the whole CTA; it is looked at only after
 // a failed attempt (every 64th), so the common case -- the phase is already complete -- costs one instruction.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          Ctl* ctl)
+__device__ __forceinline__ void mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                Ctl* ctl, uint32_t limit)
 {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return;
         if ((i & 63u) == 63u && *abort_flag) return;
     }
     *abort_flag = 1u;
     ctl->status = GEM_NLR_E_TIMEOUT;
     ctl->stopped = 1;
+}
+
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          Ctl* ctl)
+{
+    mbar_wait_limit(bar, parity, abort_flag, ctl, kSpinLimit);
 }
 
 // Bounded wait by polling (mbarrier.test_wait never suspends the thread): for the hand-overs on the critical

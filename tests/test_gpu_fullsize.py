@@ -1,10 +1,14 @@
 """Full-size parity: the benchmark shapes at their full n, in the launch configuration bench.py
-times (automatic kernel-family selection, library-side setup), one teacher-forced iteration from
-the seeded starting factor compared with the CPU oracle on every entry of U, plus the setup
-(spectral norm, X-hat) and the label read-out.
+times (automatic kernel-family selection, library-side setup).
 
-Config 4 (n = 2e6, d = 768, K = 1000) costs the oracle about 6 TFLOP in FP64 per iteration, so it is
-checked on a reduced-n twin with the same d, K and distribution."""
+* One teacher-forced iteration from the seeded starting factor compared with the CPU oracle on every
+  entry of U, plus the setup (spectral norm, X-hat) and the label read-out: configs 2, 3, 5 against the C
+  oracle, config 4 (about 6 TFLOP of FP64 per iteration) against the row-chunked numpy restatement of the
+  iteration at its full n, and against the C oracle on a reduced-n twin.
+* Free-running gem_nlr_run for the configured number of iterations against oracle.run at full n (configs 2
+  and 5, where the oracle's cost allows it): the dual gate, the gated dual update, the stop test and the
+  periodic read-back of the control block all take part; final U, objective, rho, the dual and the labels
+  are compared.  Configs 3 and 4 run free on reduced-n twins of the same kernel families (test_gpu_tc.py)."""
 import dataclasses
 
 import numpy as np
@@ -146,3 +150,61 @@ def test_embedding_shape_full_size_every_entry():
         alt_o = Uref[diff, lab_g[diff]].astype(np.float64)
         assert ((top_o - alt_o) <= 2 * TOL_U * scale).all()
     assert diff.size <= 1e-4 * n
+
+
+# ---- free-running trajectories at full n for the configured number of iterations ----
+# eps_d is raised on config 2 so that the gate opens within its 100 iterations (at the benchmark's 0.01 it
+# stays shut that early on a random start): every branch of the iteration then runs at full size.
+@pytest.mark.parametrize("cfg,path,eps_d", [(2, "mma.tf32x3", 0.2), (5, "ffma", None)])
+def test_full_size_free_running_trajectory(cfg, path, eps_d):
+    spec = synth.config(cfg)
+    n, d, K = spec.n, spec.d, spec.K
+    need = 2.2 * 4 * n * d + 5 * 4 * n * K + (1 << 30)
+    if psutil.virtual_memory().available < need:
+        pytest.skip(f"needs about {need / 2**30:.0f} GiB of host memory")
+    if torch.cuda.mem_get_info()[0] < 4 * n * (d + 2 * K + 8) + (1 << 30):
+        pytest.skip("not enough device memory")
+    hp = dict(synth.default_hparams(K))
+    if eps_d is not None:
+        hp["eps_d"] = eps_d
+    T, T_min = spec.iters, hp["T_min"]
+    X, _, _ = synth.make_mixture(spec)
+    U0 = synth.make_u0(n, K, K)
+    Xd = torch.from_numpy(X).cuda()
+    del X
+    Ud = torch.from_numpy(U0).cuda()
+    s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"],
+                   T=T, T_min=T_min, history=1)
+    assert s.path() == path, s.path()
+    s.spectral_norm()
+    Xhat = Xd.cpu().numpy()                      # both sides iterate on the library's X-hat
+    rc, info, iters = s.run()
+    assert rc in (gem.ITER_CAP, gem.CONVERGED), (rc, s.last_error())
+    Ug = s.U.cpu().numpy()
+    ytg, tg = s.get_state()
+    ytg = ytg.cpu().numpy()
+    lab_g = s.labels().cpu().numpy()
+    hist = s.history(T)
+    s.destroy()
+    del Xd, Ud
+
+    Uo, yto, infoo, iterso, rco = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, T_min)
+    assert iters == iterso == tg and (rc == gem.CONVERGED) == bool(infoo["stop"])
+    scale = float(np.abs(Uo).max())
+    err = _chunked_max_abs_diff(Ug, Uo) / scale
+    gates = sum(h["dual_applied"] for h in hist)
+    print(f"config {cfg}: {iters} free-running iterations, U err={err:.2e}, gate fired {gates} times, "
+          f"rho={info['rho']:.3e} fhat={info['fhat']:.8f}")
+    assert err <= TOL_U, err
+    assert _rel(info["fhat"], infoo["fhat"]) <= TOL_F and _rel(info["rho"], infoo["rho"]) <= 1e-4
+    assert abs(info["delta_hat"] - infoo["delta_hat"]) <= 1e-6 and info["dual_applied"] == infoo["dual"]
+    assert float(np.abs(ytg - yto).max()) <= 1e-4 * max(float(np.abs(yto).max()), 1e-30) + 1e-9
+    if eps_d is not None:
+        assert 0 < gates < iters                 # the gate was shut at first and open later
+    lab_o = oracle.labels(Uo)
+    diff = np.nonzero(lab_g != lab_o)[0]
+    if diff.size:                                # a differing row must be a numerical tie of the oracle's own factor
+        top_o = Uo[diff, lab_o[diff]].astype(np.float64)
+        alt_o = Uo[diff, lab_g[diff]].astype(np.float64)
+        assert ((top_o - alt_o) <= 2 * TOL_U * scale).all()
+    assert diff.size <= 1e-4 * n, diff.size

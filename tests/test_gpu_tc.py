@@ -94,6 +94,37 @@ def test_tiled_tc_trajectory_is_reproducible_and_matches_oracle():
     assert rel(outs[0][1]["rho"], infoo["rho"]) <= 1e-4
 
 
+def test_tiled_tc_trajectory_on_the_embedding_shape_twin():
+    """Ten free-running iterations at d = 768, K = 1000 (the widest benchmark shape on n = 4100 rows, both
+    products on the tiled kernels, the gate open from the start) against oracle.run."""
+    n, d, K, T = 4100, 768, 1000, 10
+    spec = synth.MixtureSpec("embedding-twin", n, d, K, "equal", -1.0, "sphere0.3", T, 0)
+    X, _, _ = synth.make_mixture(spec)
+    Xhat, _, _ = oracle.normalize(X)
+    U0 = synth.make_u0(n, K, K)
+    hp = dict(synth.default_hparams(K), eps_d=0.5, T_min=4)
+    s = make_solver(Xhat, U0, K, hp, T=T, precision=1, history=1)
+    assert s.path() == "f16x3.tiled", s.path()
+    rc, info, iters = s.run()
+    assert rc == gem.ITER_CAP and iters == T, (rc, s.last_error())
+    Ug = s.U.cpu().numpy()
+    ytg = s.get_state()[0].cpu().numpy()
+    hist = s.history(T)
+    lab_g = s.labels().cpu().numpy()
+    s.destroy()
+    Uo, yto, infoo, _, _ = oracle.run(Xhat, U0, K, hp["alpha"], hp["beta"], hp["eps_d"], hp["eps_c"], T, hp["T_min"])
+    assert u_err(Ug, Uo) <= TOL_U
+    assert rel(info["fhat"], infoo["fhat"]) <= TOL_F and rel(info["rho"], infoo["rho"]) <= 1e-4
+    assert sum(h["dual_applied"] for h in hist) > 0 and info["dual_applied"] == infoo["dual"]
+    assert float(np.abs(ytg - yto).max()) <= 1e-4 * float(np.abs(yto).max()) + 1e-9
+    lab_o = oracle.labels(Uo)
+    diff = np.nonzero(lab_g != lab_o)[0]
+    if diff.size:
+        scale = float(np.abs(Uo).max())
+        assert ((Uo[diff, lab_o[diff]].astype(np.float64) - Uo[diff, lab_g[diff]]) <= 2 * TOL_U * scale).all()
+    assert diff.size <= 2
+
+
 # ---- feature counts that are not a multiple of 32: the fp16-image kernels see d rounded up (zero features in the
 # images, zero rows in Theta); includes the shapes of the paper's own scaling study (d = 50, r = 3 K) ----
 # (n, d, K, r, kernel path)
