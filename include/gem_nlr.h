@@ -126,6 +126,19 @@ int gem_nlr_spectral_norm(gem_nlr_t *h, double *a_out);
 /* Declare that X_dev already holds X-hat (normalized elsewhere); a is recorded only.           */
 int gem_nlr_set_normalized(gem_nlr_t *h, double a);
 
+/* Data-informed starting factor (appendix "Additional Computation Details", paragraph "Initialization"):
+ *     V = X-hat X-hat^T Z,  V = Q R,  U0 = Proj_Omega(Q) = sqrt(K) [Q]_+ / ||[Q]_+||_F,
+ * the orthonormalization done as Cholesky QR in feature space (M = X-hat^T Z, C = X-hat^T X-hat,
+ * M^T C M = R^T R, Q = X-hat (M R^{-1})).  On entry U_dev holds the sample matrix Z (n x r, the caller's
+ * random draw, e.g. i.i.d. N(0,1); finite entries); on return it holds U0, the dual is zero and the
+ * iteration counter is 0.  X must have been normalized.  The large products run on the general-shape FFMA
+ * kernels with FP64 accumulation of the split-K partials; the r x r factorization and the solve are FP64.
+ * Needs r <= d (the sample has rank at most d) -- GEM_NLR_E_INVALID otherwise -- and a sample that is not
+ * too ill-conditioned for Cholesky QR: a non-positive pivot returns GEM_NLR_E_BREAKDOWN (U_dev then still
+ * holds Z, and the handle stays usable: write another Z, or a starting factor of your own, and go on).
+ * Synchronizes.                                                                                     */
+int gem_nlr_init_range(gem_nlr_t *h);
+
 /* Exactly one iteration of Algorithm 1 from the current (U, y).  On return U_dev holds the new
  * normalized U and *info (may be NULL) the iteration's numbers.  Returns GEM_NLR_OK,
  * GEM_NLR_CONVERGED if the stop test fired, or an error.  Synchronizes.                        */

@@ -86,7 +86,8 @@ def lib():
         L.gem_nlr_selftest_wait_timeout.restype = C.c_int
         L.gem_nlr_column_sums_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp]
         L.gem_nlr_column_sums_static.restype = C.c_int
-        for name in ("create", "spectral_norm", "set_normalized", "step", "run", "labels", "objective",
+        L.gem_nlr_init_range.argtypes = [vp]
+        for name in ("init_range", "create", "spectral_norm", "set_normalized", "step", "run", "labels", "objective",
                      "get_state", "set_state", "history", "buffer", "destroy", "run_host"):
             getattr(L, "gem_nlr_" + name).restype = C.c_int
         _lib = L
@@ -143,6 +144,10 @@ class GemNlr:
 
     def set_normalized(self, a: float = 1.0) -> None:
         self._check(lib().gem_nlr_set_normalized(self._h, float(a)))
+
+    def init_range(self) -> int:
+        """gem_nlr_init_range: U holds Z on entry, the data-informed starting factor on return."""
+        return lib().gem_nlr_init_range(self._h)
 
     def step(self):
         info = IterInfo()

@@ -60,7 +60,9 @@ Layout make_layout(const gem_nlr_params& P)
     // partial areas are sized for the largest user among the kernel families
     size_t p1 = sizeof(double) * (size_t)(L.g1x > 8 || !tc_images ? L.g1x : 8) * dp * r;   // r > 256: up to 8 row ranges of the tiled tcgen05 first product
     size_t p1_fast = ((size_t)dp * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)dp * r + r + 4) : 0;
-    L.part1 = take(p1 > p1_fast ? p1 : p1_fast);
+    if (r <= d && p1 < sizeof(double) * 8 * (size_t)d * d) p1 = sizeof(double) * 8 * (size_t)d * d;   // X-hat^T X-hat of the data-informed start: up to 8 row chunks
+    L.part1_bytes = p1 > p1_fast ? p1 : p1_fast;
+    L.part1 = take(L.part1_bytes);
     L.part1v = take(sizeof(double) * (size_t)L.gv * (r + 2));
     size_t p2 = sizeof(double) * (size_t)L.g2x * L.g2y * (3 + G2_RT);
     size_t p2_fast = sizeof(double) * (size_t)kSMs * 4 * (4 + (size_t)r);
@@ -68,6 +70,7 @@ Layout make_layout(const gem_nlr_params& P)
     // generic family: nred1 block shares; fused reduction: one share per 16 entries of a record + r + 2 sums
     L.red1 = take(sizeof(double) * ((size_t)L.nred1 + ((size_t)dp * r + r + 2 + 15) / 16 + r + 2 + 8));
     L.setup = take(sizeof(double) * (3 * (size_t)d + 4 + (size_t)L.gs * d));
+    L.init = take(r <= d ? sizeof(double) * ((size_t)d * d + 2 * (size_t)d * r + (size_t)r * r) : 0);
     L.hist = take(P.history ? sizeof(gem_nlr_iter_info) * (size_t)(P.T > 0 ? P.T : 1) : 0);
     L.xhat = take(P.x_inplace ? 0 : sizeof(float) * (size_t)n * d);
     // tcgen05 shapes: X-hat is static, so its two-term fp16 split is built once, row-major (second product)
@@ -366,6 +369,26 @@ static int result_code(gem_nlr_t* h, bool capped)
     if (c.status < 0) { h->sticky_error = c.status; return c.status; }
     if (c.last.stop) return GEM_NLR_CONVERGED;
     return capped ? GEM_NLR_ITER_CAP : GEM_NLR_OK;
+}
+
+int gem_nlr_init_range(gem_nlr_t* h)
+{
+    if (!h) return GEM_NLR_E_INVALID;
+    if (h->sticky_error) return h->sticky_error;
+    if (!h->normalized) return GEM_NLR_E_NOT_READY;
+    if (h->pb.P.r > h->pb.P.d) return GEM_NLR_E_INVALID;      // the sample X-hat X-hat^T Z has rank <= d
+    int rc = reset_ctl(h, 0);                                 // multiplier 1, no gate pending, not stopped
+    if (rc) return rc;
+    if (!launch_range_init(h->pb)) return GEM_NLR_E_WORKSPACE;
+    launch_tail(h->pb);                                       // U0 = c [Q]_+ written out
+    rc = read_ctl(h);
+    if (rc) return rc;
+    const int status = h->host_ctl->status;
+    // the starting factor is in place: y = 0, iteration counter 0, no record of an iteration
+    CK(h, cudaMemsetAsync(h->pb.ytilde(), 0, sizeof(float) * (size_t)h->pb.P.n, h->pb.stream));
+    rc = reset_ctl(h, 0);
+    if (rc) return rc;
+    return status < 0 ? status : GEM_NLR_OK;
 }
 
 int gem_nlr_step(gem_nlr_t* h, gem_nlr_iter_info* info)

@@ -954,13 +954,24 @@ void launch_red1(const Problem& pb, int g, int ignore_stop, int scale_cf)
     pb.count(1);
 }
 
-void launch_generic_pass2_kernel(const Problem& pb)
+void launch_generic_pass2_alpha(const Problem& pb, float alpha)
 {
     const auto& P = pb.P;
     const auto& L = pb.L;
     dim3 g2(L.g2x, L.g2y);
     k_pass2_generic<<<g2, 256, 0, pb.stream>>>(pb.X, pb.theta(), pb.U, pb.ybar(), pb.p(), pb.alpha_s(),
-                                               pb.ctl(), P.n, P.d, P.r, P.alpha, pb.part2());
+                                               pb.ctl(), P.n, P.d, P.r, alpha, pb.part2());
+    pb.count();
+}
+
+void launch_generic_pass2_kernel(const Problem& pb)
+{
+    launch_generic_pass2_alpha(pb, pb.P.alpha);
+}
+
+void launch_pass1_partials(const Problem& pb, const float* A, const float* B, int da, int rb, int tiles_b, dim3 grid)
+{
+    k_pass1_generic<<<grid, 256, 0, pb.stream>>>(A, B, pb.ctl(), pb.P.n, da, rb, tiles_b, pb.part1(), 1);
     pb.count();
 }
 

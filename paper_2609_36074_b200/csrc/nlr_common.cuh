@@ -29,6 +29,8 @@ struct Ctl {
 
 struct Layout {
     size_t ctl, p, s, alpha_s, theta, thimg, ytilde, ybar, part1, part1v, part2, red1, setup, hist, xhat, total;
+    size_t init;             // FP64 scratch of the data-informed start: M, C, T, G (0 bytes when r > d)
+    size_t part1_bytes;      // size of the split-K partial area
     size_t ximg, ximgT;      // fp16 split images of X-hat (row-major and transposed), wide tensor-core shapes only (else 0 bytes)
     int dp;                  // d rounded up to a multiple of 32 when the fp16 images exist, else d: feature count of the image kernels
     int64_t n_pad;           // n rounded up to 64: the transposed images cover n_pad / 32 stages of 32 rows
@@ -79,6 +81,7 @@ struct Problem {
     double* part2() const { return reinterpret_cast<double*>(ws + L.part2); }
     double* red1() const { return reinterpret_cast<double*>(ws + L.red1); }
     double* setup() const { return reinterpret_cast<double*>(ws + L.setup); }
+    double* init() const { return reinterpret_cast<double*>(ws + L.init); }
     gem_nlr_iter_info* hist() const { return reinterpret_cast<gem_nlr_iter_info*>(ws + L.hist); }
 };
 
@@ -91,6 +94,12 @@ void launch_vector_pass(const Problem& pb);
 void launch_generic_pass1(const Problem& pb, int ignore_stop);
 void launch_fin1(const Problem& pb, int mode);
 void launch_generic_pass2_kernel(const Problem& pb);
+void launch_generic_pass2_alpha(const Problem& pb, float alpha);    // the same kernel with a given step size
+// FP64 split-K partials of A^T (c_f B) into part1 (A: n x da, B: n x rb, both row-major with their own width as
+// pitch; grid = (row chunks, da tiles x rb tiles)); ignores the stop flag.
+void launch_pass1_partials(const Problem& pb, const float* A, const float* B, int da, int rb, int tiles_b, dim3 grid);
+// Data-informed starting factor (kernels_init.cu).
+bool launch_range_init(const Problem& pb);
 // Reduction of g FP64 partials of Theta (layout [d][r] each) into Theta and the ||Theta||^2 shares.
 void launch_red1(const Problem& pb, int g, int ignore_stop, int scale_cf);   // the fused second product alone
 void launch_fin2(const Problem& pb, int gx, int gy, int cols_per);
