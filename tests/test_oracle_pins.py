@@ -474,3 +474,74 @@ def test_range_init_needs_a_full_rank_sample():
     Z = rng.standard_normal((200, 8)).astype(np.float32)          # r > d: V has rank <= d
     with pytest.raises(np.linalg.LinAlgError):
         range_init.range_init(Xhat, Z, 8)
+
+
+# ---- label read-out for r > K (appendix "Additional Computation Details", "Recover cluster labels") ----
+def _planted_factor_with_split_columns(n=600, K=4, per=3, seed=0, noise=0.0):
+    """U >= 0 with r = per * K columns whose rows are constant within each planted cluster, every cluster's mass
+    spread over its own `per` columns with different weights: U U^T is the planted block matrix."""
+    rng = np.random.default_rng(seed)
+    sizes = np.full(K, n // K)
+    sizes[: n - sizes.sum()] += 1
+    lab = np.repeat(np.arange(K), sizes)
+    rng.shuffle(lab)
+    r = per * K
+    U = np.zeros((n, r))
+    for k in range(K):
+        w = rng.uniform(0.2, 1.0, size=per)
+        w /= np.linalg.norm(w)
+        U[np.ix_(lab == k, np.arange(per * k, per * (k + 1)))] = w / np.sqrt(sizes[k])
+    if noise:
+        U = np.abs(U + noise * rng.standard_normal(U.shape) / np.sqrt(n))
+    return U.astype(np.float32), lab
+
+
+def test_spectral_labels_recover_a_partition_that_row_argmax_splits():
+    from oracle import spectral_labels as sl
+    U, lab = _planted_factor_with_split_columns()
+    labels, Y, passes = sl.spectral_labels(U, 4)
+    assert _same_partition(labels, lab.astype(np.int32))
+    # the row argmax is a valid column index but not a cluster index when r > K: the heaviest of a cluster's own
+    # columns wins for all of its rows here, so the argmax only names K of the 12 columns
+    assert set(oracle.labels(U).tolist()) <= set(range(12)) and len(set(oracle.labels(U).tolist())) == 4
+    Un, _ = _planted_factor_with_split_columns(noise=0.3, seed=3)
+    labels_n, _, _ = sl.spectral_labels(Un, 4)
+    assert _same_partition(labels_n, _planted_factor_with_split_columns(seed=3)[1].astype(np.int32))
+
+
+def test_spectral_embedding_distances_match_the_gram_route():
+    """Leading left singular vectors from the r x r Gram matrix: P_K = U Q_K S_K^{-1} with U^T U = Q S^2 Q^T.
+    Rows of the two embeddings have the same pairwise distances (signs and in-eigenspace rotations drop out)."""
+    from oracle import spectral_labels as sl
+    U, _ = _planted_factor_with_split_columns(noise=0.5, seed=1)
+    K = 4
+    Y = sl.embedding(U, K)
+    U64 = U.astype(np.float64)
+    lam, Q = np.linalg.eigh(U64.T @ U64)
+    Yg = U64 @ (Q[:, ::-1][:, :K] / np.sqrt(lam[::-1][:K]))
+    rng = np.random.default_rng(0)
+    i, j = rng.integers(0, U.shape[0], 200), rng.integers(0, U.shape[0], 200)
+    d_svd = np.linalg.norm(Y[i] - Y[j], axis=1)
+    d_gram = np.linalg.norm(Yg[i] - Yg[j], axis=1)
+    assert np.abs(d_svd - d_gram).max() <= 1e-9
+
+
+def test_lloyd_ends_at_a_fixed_point_and_does_not_raise_the_cost():
+    from oracle import spectral_labels as sl
+    rng = np.random.default_rng(2)
+    Y = np.concatenate([rng.standard_normal((80, 3)) + 4.0 * rng.standard_normal(3) for _ in range(5)])
+    seeds = sl.farthest_point_seeds(Y, 5)
+    assert len(set(seeds.tolist())) == 5 and seeds[0] == int(np.argmax((Y ** 2).sum(1)))
+    # each seed is the farthest row from the seeds before it
+    for m in range(1, 5):
+        dmin = np.min(((Y[:, None, :] - Y[seeds[:m]][None]) ** 2).sum(2), axis=1)
+        assert dmin[seeds[m]] == dmin.max()
+    labels, centres, passes = sl.lloyd(Y, Y[seeds].copy(), max_iter=100)
+    assert passes < 100
+    d2 = ((Y[:, None, :] - centres[None]) ** 2).sum(2)
+    assert np.array_equal(labels, np.argmin(d2, axis=1))
+    for k in range(5):
+        np.testing.assert_allclose(centres[k], Y[labels == k].mean(0), atol=1e-12)
+    cost = lambda lab, C: float(((Y - C[lab]) ** 2).sum())
+    lab0 = np.argmin(((Y[:, None, :] - Y[seeds][None]) ** 2).sum(2), axis=1)
+    assert cost(labels, centres) <= cost(lab0, Y[seeds]) + 1e-12
