@@ -160,6 +160,23 @@ int gem_nlr_run(gem_nlr_t *h, gem_nlr_iter_info *last, int32_t *iters_done);
  * are column indices, not cluster indices.                                                       */
 int gem_nlr_labels(gem_nlr_t *h, int32_t *labels_dev);
 
+/* The paper's own read-out (appendix "Additional Computation Details", paragraph "Recover cluster labels
+ * from U matrix"), for any r >= K: the leading K left singular vectors of U as a spectral embedding, then
+ * K-means on its rows.  The singular vectors come from the r x r Gram matrix (U^T U = Q S^2 Q^T,
+ * P_K = U Q_K S_K^{-1}; FP64, Jacobi).  The paper fixes neither the seeding nor the stopping rule of its
+ * K-means; here both are deterministic: farthest-point seeding (first centre = the row of largest norm, each
+ * further centre the row farthest from its nearest centre, lowest row index on ties), then Lloyd passes
+ * (nearest centre, lowest centre index on ties; a centre without rows stays) until no label changes or
+ * max_iter passes.  Label k is the k-th seeded centre.  labels_dev: n int32 (output).  scratch_dev: caller-owned
+ * device memory, 256-byte aligned, at least gem_nlr_labels_spectral_scratch_bytes (about 4 n (K + 1) bytes:
+ * the embedding); it also uses the handle's split-K partial area, so it must not run concurrently with an
+ * iteration.  *passes_out (may be NULL): assignment passes made.  Needs r <= 2048.  Returns GEM_NLR_OK,
+ * GEM_NLR_E_BREAKDOWN if U has numerical rank below K, or an argument / CUDA error.  Reads back 8 bytes per
+ * Lloyd pass; synchronizes.                                                                          */
+size_t gem_nlr_labels_spectral_scratch_bytes(const gem_nlr_params *params);
+int gem_nlr_labels_spectral(gem_nlr_t *h, int32_t *labels_dev, void *scratch_dev, size_t scratch_bytes,
+                            int32_t max_iter, int32_t *passes_out);
+
 /* f-hat_y(U) of Eq. "normalized" at the current (U, y).  Synchronizes.                         */
 int gem_nlr_objective(gem_nlr_t *h, double *fhat_out);
 

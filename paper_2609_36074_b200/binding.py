@@ -87,6 +87,10 @@ def lib():
         L.gem_nlr_column_sums_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp]
         L.gem_nlr_column_sums_static.restype = C.c_int
         L.gem_nlr_init_range.argtypes = [vp]
+        L.gem_nlr_labels_spectral_scratch_bytes.argtypes = [pp]
+        L.gem_nlr_labels_spectral_scratch_bytes.restype = C.c_size_t
+        L.gem_nlr_labels_spectral.argtypes = [vp, vp, vp, C.c_size_t, C.c_int32, C.POINTER(C.c_int32)]
+        L.gem_nlr_labels_spectral.restype = C.c_int
         for name in ("init_range", "create", "spectral_norm", "set_normalized", "step", "run", "labels", "objective",
                      "get_state", "set_state", "history", "buffer", "destroy", "run_host"):
             getattr(L, "gem_nlr_" + name).restype = C.c_int
@@ -165,6 +169,18 @@ class GemNlr:
             out = torch.empty(self.params.n, dtype=torch.int32, device=self.U.device)
         self._check(lib().gem_nlr_labels(self._h, out.data_ptr()))
         return out
+
+    def labels_spectral(self, out=None, max_iter: int = 50):
+        """gem_nlr_labels_spectral: (rc, labels, assignment passes); the scratch is a torch allocation."""
+        import torch
+        if out is None:
+            out = torch.empty(self.params.n, dtype=torch.int32, device=self.U.device)
+        nbytes = int(lib().gem_nlr_labels_spectral_scratch_bytes(C.byref(self.params)))
+        scratch = torch.empty(nbytes, dtype=torch.uint8, device=self.U.device)
+        passes = C.c_int32()
+        rc = lib().gem_nlr_labels_spectral(self._h, out.data_ptr(), scratch.data_ptr(), nbytes, int(max_iter),
+                                           C.byref(passes))
+        return rc, out, passes.value
 
     def objective(self) -> float:
         f = C.c_double()

@@ -448,6 +448,25 @@ int gem_nlr_labels(gem_nlr_t* h, int32_t* labels_dev)
     return GEM_NLR_OK;
 }
 
+size_t gem_nlr_labels_spectral_scratch_bytes(const gem_nlr_params* params)
+{
+    if (!params || !valid_params(*params)) return 0;
+    return readout_scratch_bytes(*params);
+}
+
+int gem_nlr_labels_spectral(gem_nlr_t* h, int32_t* labels_dev, void* scratch_dev, size_t scratch_bytes,
+                            int32_t max_iter, int32_t* passes_out)
+{
+    if (!h || !labels_dev || !scratch_dev || max_iter < 1) return GEM_NLR_E_INVALID;
+    if (((uintptr_t)scratch_dev & 255) != 0) return GEM_NLR_E_INVALID;
+    if (scratch_bytes < readout_scratch_bytes(h->pb.P)) return GEM_NLR_E_WORKSPACE;
+    if (h->pb.P.r > 2048) return GEM_NLR_E_INVALID;          // one-CTA eigen-decomposition of the r x r Gram matrix
+    int rc = run_spectral_labels(h->pb, labels_dev, (char*)scratch_dev, max_iter, passes_out,
+                                 reinterpret_cast<unsigned long long*>(h->host_scratch));
+    if (rc == GEM_NLR_E_CUDA) return cuda_fail(h, cudaGetLastError(), "labels_spectral");
+    return rc;
+}
+
 int gem_nlr_objective(gem_nlr_t* h, double* fhat_out)
 {
     if (!h || !fhat_out) return GEM_NLR_E_INVALID;

@@ -25,6 +25,12 @@ k_red_f64(const double* __restrict__ part, int g, int64_t count, double* __restr
     }
 }
 
+void launch_red_f64(const Problem& pb, const double* part, int g, int64_t count, double* out)
+{
+    k_red_f64<<<kSMs, 256, 0, pb.stream>>>(part, g, count, out);
+    pb.count(1);
+}
+
 // One CTA.  M (d x r), C (d x d) FP64 row-major in; T = C M, G = M^T T, Cholesky G = R^T R in place (upper
 // triangle of G), B = M R^{-1} written as FP32 into theta (d x r row-major, what the second product reads).
 // A pivot that is not positive relative to the largest diagonal entry of G (the sample has no full column

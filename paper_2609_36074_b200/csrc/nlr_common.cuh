@@ -100,6 +100,11 @@ void launch_generic_pass2_alpha(const Problem& pb, float alpha);    // the same 
 void launch_pass1_partials(const Problem& pb, const float* A, const float* B, int da, int rb, int tiles_b, dim3 grid);
 // Data-informed starting factor (kernels_init.cu).
 bool launch_range_init(const Problem& pb);
+void launch_red_f64(const Problem& pb, const double* part, int g, int64_t count, double* out);
+// Spectral label read-out for r >= K (kernels_readout.cu): leading K left singular vectors + K-means.
+size_t readout_scratch_bytes(const gem_nlr_params& P);
+int run_spectral_labels(const Problem& pb, int32_t* labels, char* scratch, int max_iter, int32_t* passes_out,
+                        unsigned long long* pinned_host /* >= 16 bytes */);
 // Reduction of g FP64 partials of Theta (layout [d][r] each) into Theta and the ||Theta||^2 shares.
 void launch_red1(const Problem& pb, int g, int ignore_stop, int scale_cf);   // the fused second product alone
 void launch_fin2(const Problem& pb, int gx, int gy, int cols_per);
