@@ -217,6 +217,36 @@ int gem_nlr_profile_read(gem_nlr_t *h, double *ms_first_phase, double *ms_second
                          int64_t *iterations);
 int64_t gem_nlr_launch_count(gem_nlr_t *h);
 
+/* ---- Row-sharded runs over several GPUs (one process and one handle per GPU) ---------------------------
+ * The iteration shards by rows: rank g holds rows_g of X, U and the dual (n in its gem_nlr_params is its own
+ * row count), and the small replicated quantities are summed over the ranks twice per iteration -- after the
+ * first product Theta (d x r), s (r), sum q^2, sum ytilde q; after the second a, b, h and the column sums of
+ * W (r) -- plus once per application of X_c^T X_c during setup and once for the column mean.  The library
+ * does not link a communication library: the caller supplies two callbacks (with torch.distributed / NCCL
+ * behind them in the Python binding).  The sums themselves are taken by this library's kernels, in rank
+ * order, from the gathered per-rank records, so every rank obtains bit-identical replicated values and the
+ * result does not depend on a library's reduction order.  The paper runs on one GPU; this is the scale-out
+ * its largest data sets call for.
+ *
+ * gem_nlr_gather_fn: all ranks call it with the same byte count; when the work it enqueues on cuda_stream
+ * has completed, recv_dev holds the world records of `bytes` bytes each, back to back in rank order
+ * (an all-gather; send_dev and recv_dev are device memory of this rank).  Returns 0 on success.
+ * gem_nlr_host_sum_fn: replaces buf_host[0 .. count) by its sum over the ranks, added in rank order, on
+ * every rank (host memory; blocking).  Returns 0 on success.
+ *
+ * gem_nlr_shard_attach: call after gem_nlr_create and before anything else.  n_global = total rows.
+ * exchange_dev: device memory of gem_nlr_shard_exchange_bytes(params, world) bytes, 256-byte aligned,
+ * caller-owned, alive until destroy.  Afterwards gem_nlr_spectral_norm, _step, _run, _objective and _labels
+ * work as on one GPU (every rank must make the same calls in the same order; rho, the gate and the stop test
+ * are global and identical on all ranks; labels are those of the rank's own rows).  gem_nlr_init_range,
+ * gem_nlr_labels_spectral and gem_nlr_run_host are single-GPU calls and return GEM_NLR_E_INVALID on a
+ * sharded handle.                                                                                       */
+typedef int (*gem_nlr_gather_fn)(void *ctx, const void *send_dev, void *recv_dev, size_t bytes, void *cuda_stream);
+typedef int (*gem_nlr_host_sum_fn)(void *ctx, double *buf_host, int64_t count);
+size_t gem_nlr_shard_exchange_bytes(const gem_nlr_params *params, int32_t world);
+int gem_nlr_shard_attach(gem_nlr_t *h, int32_t rank, int32_t world, int64_t n_global, gem_nlr_gather_fn gather,
+                         gem_nlr_host_sum_fn host_sum, void *ctx, void *exchange_dev, size_t exchange_bytes);
+
 /* Self-test of the failure path that a healthy run never takes (no counterpart in the paper): every wait of
  * the copy / tensor-core pipelines is bounded, and when one runs out the kernel records GEM_NLR_E_TIMEOUT
  * and runs to its end instead of hanging.  This call launches a one-CTA kernel that waits, through the same

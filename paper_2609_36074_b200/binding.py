@@ -86,6 +86,10 @@ def lib():
         L.gem_nlr_selftest_wait_timeout.restype = C.c_int
         L.gem_nlr_column_sums_static.argtypes = [vp, C.c_int64, C.c_int32, vp, vp]
         L.gem_nlr_column_sums_static.restype = C.c_int
+        L.gem_nlr_shard_exchange_bytes.argtypes = [pp, C.c_int32]
+        L.gem_nlr_shard_exchange_bytes.restype = C.c_size_t
+        L.gem_nlr_shard_attach.argtypes = [vp, C.c_int32, C.c_int32, C.c_int64, vp, vp, vp, vp, C.c_size_t]
+        L.gem_nlr_shard_attach.restype = C.c_int
         L.gem_nlr_init_range.argtypes = [vp]
         L.gem_nlr_labels_spectral_scratch_bytes.argtypes = [pp]
         L.gem_nlr_labels_spectral_scratch_bytes.restype = C.c_size_t

@@ -110,6 +110,7 @@ struct gem_nlr {
     TcgPlan tcg;
     Tcg1Plan tcg1;
     bool use_tcg1;         // first product by the tiled tcgen05 kernel (vector pass separate)
+    ShardInfo shard;       // row-sharded run: rank, world, callbacks (world <= 1: single GPU)
     char err[256];
     int64_t launches;      // kernels launched by this handle
     int pi_iters;          // power iterations taken by the last setup
@@ -141,6 +142,7 @@ static int reset_ctl(gem_nlr_t* h, int32_t t)
     c.c_f = 1.0f;
     c.t = t;
     c.hist_cap = h->pb.P.history ? (h->pb.P.T > 0 ? h->pb.P.T : 1) : 0;
+    c.shard_world = h->shard.world;
     *h->host_ctl = c;
     CK(h, cudaMemcpyAsync(h->pb.ctl(), h->host_ctl, sizeof(Ctl), cudaMemcpyHostToDevice, h->pb.stream));
     CK(h, cudaStreamSynchronize(h->pb.stream));   // host_ctl is reused for read-backs
@@ -162,6 +164,10 @@ static int ensure_loaded(gem_nlr_t* h)
 {
     if (!h->loaded) {
         launch_init_colsum(h->pb);
+        if (h->pb.shard) {
+            const int rc = shard_exchange_second(h->pb, 1);
+            if (rc) return rc;
+        }
         h->loaded = true;
     }
     return GEM_NLR_OK;
@@ -169,8 +175,10 @@ static int ensure_loaded(gem_nlr_t* h)
 
 // One iteration = vector pass + first product (+ reductions), then the fused second product
 // and its scalar reduction.  With profiling on, events bracket the two phases.
-static void launch_iteration(gem_nlr_t* h)
+static int launch_iteration(gem_nlr_t* h)
 {
+    const bool sharded = h->pb.shard != nullptr;
+    int xrc = GEM_NLR_OK;
     const bool prof = h->profile && h->ev_used + 3 <= h->ev_cap;
     cudaEvent_t* e = prof ? h->ev + h->ev_used : nullptr;
     if (prof) cudaEventRecord(e[0], h->pb.stream);
@@ -186,18 +194,32 @@ static void launch_iteration(gem_nlr_t* h)
         else launch_generic_pass1(h->pb, 0);
         launch_fin1(h->pb, 0);
     }
+    // row-sharded: the kernels above parked this rank's sums; combine all ranks' and take the scalar step
+    if (sharded) xrc = shard_exchange_first((h->use_tc1 || h->use_tcg1 || h->use_tc || h->use_tcg) ? h->pbp : h->pb, 0);
+    if (xrc) return xrc;
     if (prof) cudaEventRecord(e[1], h->pb.stream);
     if (h->use_tc || h->use_ffma || h->use_tcg) {
         if (h->use_tcg) tcg_launch_second(h->pbp, h->tcg);
         else if (h->use_tc) tc_launch_second(h->pbp, h->tc);
         else if (h->use_mma) mma_launch_second(h->pb, h->ffma);
         else ffma_launch_second(h->pb, h->ffma);
+        if (sharded) xrc = shard_exchange_second(h->pb, 0);
         if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
-        return;
+        return xrc;
     }
     launch_generic_pass2_kernel(h->pb);
     if (prof) { cudaEventRecord(e[2], h->pb.stream); h->ev_used += 3; }
     launch_fin2(h->pb, h->pb.L.g2x, h->pb.L.g2y, G2_RT);
+    if (sharded) xrc = shard_exchange_second(h->pb, 0);
+    return xrc;
+}
+
+// Finishes the last iteration (dual step, rho, stop test) and writes the pending multiplier into U.
+static int launch_tail_any(gem_nlr_t* h)
+{
+    launch_tail(h->pb);
+    if (h->pb.shard) return shard_exchange_first(h->pb, 1);
+    return GEM_NLR_OK;
 }
 
 static void drain_profile(gem_nlr_t* h)
@@ -371,11 +393,48 @@ static int result_code(gem_nlr_t* h, bool capped)
     return capped ? GEM_NLR_ITER_CAP : GEM_NLR_OK;
 }
 
+size_t gem_nlr_shard_exchange_bytes(const gem_nlr_params* params, int32_t world)
+{
+    if (!params || !valid_params(*params) || world < 1) return 0;
+    const Layout L = make_layout(*params);
+    return sizeof(double) * shard_record_doubles(*params, L.dp) * (size_t)(world + 1);
+}
+
+int gem_nlr_shard_attach(gem_nlr_t* h, int32_t rank, int32_t world, int64_t n_global, gem_nlr_gather_fn gather,
+                         gem_nlr_host_sum_fn host_sum, void* ctx, void* exchange_dev, size_t exchange_bytes)
+{
+    if (!h || world < 1 || rank < 0 || rank >= world || n_global < h->pb.P.n || !gather || !host_sum || !exchange_dev)
+        return GEM_NLR_E_INVALID;
+    if (((uintptr_t)exchange_dev & 255) || h->normalized || h->t_host != 0) return GEM_NLR_E_INVALID;
+    if (exchange_bytes < gem_nlr_shard_exchange_bytes(&h->pb.P, world)) return GEM_NLR_E_WORKSPACE;
+    h->shard.rank = rank;
+    h->shard.world = world;
+    h->shard.n_global = n_global;
+    h->shard.gather = gather;
+    h->shard.host_sum = host_sum;
+    h->shard.ctx = ctx;
+    h->shard.xbuf = reinterpret_cast<double*>(exchange_dev);
+    h->shard.xcount = shard_record_doubles(h->pb.P, h->pb.L.dp);
+    // the penalty weight and rho refer to all rows
+    h->pb.gamma = (double)h->pb.P.beta / (double)n_global;
+    h->pb.gamma_f = (float)h->pb.gamma;
+    h->pbp.gamma = h->pb.gamma;
+    h->pbp.gamma_f = h->pb.gamma_f;
+    if (world == 1) {                                         // one rank: nothing to exchange, the single-GPU path as it is
+        h->shard.world = 0;
+        return GEM_NLR_OK;
+    }
+    h->pb.shard = &h->shard;
+    h->pbp.shard = &h->shard;
+    return reset_ctl(h, 0);                                   // the control block now says "sharded"
+}
+
 int gem_nlr_init_range(gem_nlr_t* h)
 {
     if (!h) return GEM_NLR_E_INVALID;
     if (h->sticky_error) return h->sticky_error;
     if (!h->normalized) return GEM_NLR_E_NOT_READY;
+    if (h->pb.shard) return GEM_NLR_E_INVALID;                // single-GPU call
     if (h->pb.P.r > h->pb.P.d) return GEM_NLR_E_INVALID;      // the sample X-hat X-hat^T Z has rank <= d
     int rc = reset_ctl(h, 0);                                 // multiplier 1, no gate pending, not stopped
     if (rc) return rc;
@@ -398,9 +457,10 @@ int gem_nlr_step(gem_nlr_t* h, gem_nlr_iter_info* info)
     if (!h->normalized) return GEM_NLR_E_NOT_READY;
     int rc = clear_stop(h);
     if (rc) return rc;
-    ensure_loaded(h);
-    launch_iteration(h);
-    launch_tail(h->pb);
+    rc = ensure_loaded(h);
+    if (rc == GEM_NLR_OK) rc = launch_iteration(h);
+    if (rc == GEM_NLR_OK) rc = launch_tail_any(h);
+    if (rc) return rc;
     rc = read_ctl(h);
     if (rc) return rc;
     if (info) *info = h->host_ctl->last;
@@ -414,12 +474,14 @@ int gem_nlr_run(gem_nlr_t* h, gem_nlr_iter_info* last, int32_t* iters_done)
     if (!h->normalized) return GEM_NLR_E_NOT_READY;
     int rc = clear_stop(h);
     if (rc) return rc;
-    ensure_loaded(h);
+    rc = ensure_loaded(h);
+    if (rc) return rc;
     const int32_t T = h->pb.P.T, T_min = h->pb.P.T_min;
     const int32_t t0 = h->t_host;
     int since_check = 0;
     for (int32_t t = t0; t < T; ++t) {
-        launch_iteration(h);
+        rc = launch_iteration(h);
+        if (rc) return rc;
         ++since_check;
         // The stop test of iteration t is evaluated by the first kernels of iteration t + 1, so a
         // flag seen here is at most one iteration old; kernels launched after a stop return at once.
@@ -431,7 +493,8 @@ int gem_nlr_run(gem_nlr_t* h, gem_nlr_iter_info* last, int32_t* iters_done)
             if (h->host_ctl->stopped) break;
         }
     }
-    launch_tail(h->pb);
+    rc = launch_tail_any(h);
+    if (rc) return rc;
     rc = read_ctl(h);
     if (rc) return rc;
     if (h->profile) drain_profile(h);
@@ -461,6 +524,7 @@ int gem_nlr_labels_spectral(gem_nlr_t* h, int32_t* labels_dev, void* scratch_dev
     if (((uintptr_t)scratch_dev & 255) != 0) return GEM_NLR_E_INVALID;
     if (scratch_bytes < readout_scratch_bytes(h->pb.P)) return GEM_NLR_E_WORKSPACE;
     if (h->pb.P.r > 2048) return GEM_NLR_E_INVALID;          // one-CTA eigen-decomposition of the r x r Gram matrix
+    if (h->pb.shard) return GEM_NLR_E_INVALID;               // single-GPU call
     int rc = run_spectral_labels(h->pb, labels_dev, (char*)scratch_dev, max_iter, passes_out,
                                  reinterpret_cast<unsigned long long*>(h->host_scratch));
     if (rc == GEM_NLR_E_CUDA) return cuda_fail(h, cudaGetLastError(), "labels_spectral");
@@ -471,9 +535,14 @@ int gem_nlr_objective(gem_nlr_t* h, double* fhat_out)
 {
     if (!h || !fhat_out) return GEM_NLR_E_INVALID;
     if (!h->normalized) return GEM_NLR_E_NOT_READY;
-    ensure_loaded(h);
+    int rc = ensure_loaded(h);
+    if (rc) return rc;
     launch_objective(h->pb);
-    int rc = read_ctl(h);
+    if (h->pb.shard) {
+        rc = shard_exchange_first(h->pb, 2);
+        if (rc) return rc;
+    }
+    rc = read_ctl(h);
     if (rc) return rc;
     *fhat_out = h->host_ctl->f_final;
     return GEM_NLR_OK;

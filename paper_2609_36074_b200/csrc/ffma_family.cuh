@@ -18,6 +18,9 @@ bool ffma_plan(const Problem& pb, FfmaPlan* plan);
 void ffma_launch_first(const Problem& pb, const FfmaPlan& plan, int mode);
 // Reduction of g per-CTA partial records [d*r Theta | r s | sum q^2 | sum ytilde q] (FP64) + scalar step.
 void red1_fused_launch(const Problem& pb, int g, int mode);
+// The same reduction over the gathered records of a row-sharded run (one per rank, rank order), followed by the
+// scalar step on the combined sums; n_global is the row count over all ranks.
+void red1_combine_launch(const Problem& pb, const double* records, int world, int64_t n_global, int mode);
 // Fused second product, statistics, scalar step (multiplier, movement, gate, p).
 void ffma_launch_second(const Problem& pb, const FfmaPlan& plan);
 

@@ -13,11 +13,13 @@ namespace gemnlr {
 // reset to 1), 2: objective evaluation only.
 __device__ __forceinline__ void fin1_scalars(Ctl* ctl, double qq, double yq, double t2, int64_t n,
                                              double gamma, double eps_c, int T_min,
-                                             gem_nlr_iter_info* hist, int mode)
+                                             gem_nlr_iter_info* hist, int mode, bool combined = false)
 {
     ctl->qq = qq;
     ctl->yq = yq;
     if (mode != 1) ctl->theta2 = t2;
+    // row-sharded run: these are one rank's sums; they stay parked until the exchange has combined all ranks'
+    if (ctl->shard_world > 1 && !combined) return;
     if (ctl->tail_pending) {
         gem_nlr_iter_info rec = ctl->last;
         rec.rho = sqrt(qq / (double)n);
@@ -45,8 +47,14 @@ __device__ __forceinline__ void fin1_scalars(Ctl* ctl, double qq, double yq, dou
 // Delta = max{c^2 a + b - 2 c h, 0}; delta_hat = sqrt(Delta)/sqrt(K); gate = Delta < eps_d^2 K.
 // Returns false on breakdown / non-finite statistics; *c_out = FP64(c_f) otherwise.
 __device__ __forceinline__ bool fin2_scalars(Ctl* ctl, double a, double b, double h, int K,
-                                             double eps_d, double* c_out)
+                                             double eps_d, double* c_out, bool combined = false)
 {
+    if (ctl->shard_world > 1 && !combined) {
+        // row-sharded run: park this rank's sums; with c = 1 the caller stores its plain column sums in p
+        ctl->sa = a; ctl->sb = b; ctl->sh = h;
+        *c_out = 1.0;
+        return true;
+    }
     gem_nlr_iter_info rec;
     rec.t = ctl->t;
     rec.dual_applied = 0;

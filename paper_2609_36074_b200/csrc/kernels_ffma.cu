@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(256)
 k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, Ctl* __restrict__ ctl,
              float* __restrict__ theta, double* __restrict__ red, float* __restrict__ s,
              float* __restrict__ alpha_s, int64_t n, float alpha, double gamma, double eps_c, int T_min,
-             gem_nlr_iter_info* __restrict__ hist, int mode, int ignore_stop)
+             gem_nlr_iter_info* __restrict__ hist, int mode, int ignore_stop, int combined)
 {
     if (!ignore_stop && ctl->stopped) return;
     __shared__ double sl[16][RED1_EB];
@@ -338,7 +338,7 @@ k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, 
 #pragma unroll
         for (int k = 1; k < 16; ++k) tot += sl[k][e_local];
         if (e < dr) {
-            theta[e] = (float)tot;
+            if (mode != 1) theta[e] = (float)tot;          // the tail keeps Theta: its records carry no fresh product
             t2 = tot * tot;
         } else {
             extra[e - dr] = tot;
@@ -364,7 +364,7 @@ k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, 
     tt = block_sum<256>(tt, sred);
     if (threadIdx.x == 0) {
         ctl->counter[0] = 0;
-        fin1_scalars(ctl, __ldcg(extra + r), __ldcg(extra + r + 1), tt, n, gamma, eps_c, T_min, hist, mode);
+        fin1_scalars(ctl, __ldcg(extra + r), __ldcg(extra + r + 1), tt, n, gamma, eps_c, T_min, hist, mode, combined != 0);
     }
 }
 
@@ -633,7 +633,16 @@ void red1_fused_launch(const Problem& pb, int g, int mode)
     const int dr = pb.P.d * pb.P.r;
     ffma::k_red1_fused<<<(dr + pb.P.r + 2 + ffma::RED1_EB - 1) / ffma::RED1_EB, 256, 0, pb.stream>>>(
         pb.part1(), g, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
-        pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0);
+        pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0, 0);
+    pb.count(1);
+}
+
+void red1_combine_launch(const Problem& pb, const double* records, int world, int64_t n_global, int mode)
+{
+    const int dr = pb.P.d * pb.P.r;
+    ffma::k_red1_fused<<<(dr + pb.P.r + 2 + ffma::RED1_EB - 1) / ffma::RED1_EB, 256, 0, pb.stream>>>(
+        records, world, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
+        n_global, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, mode != 0, 1);
     pb.count(1);
 }
 

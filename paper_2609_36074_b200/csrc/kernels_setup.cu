@@ -236,10 +236,23 @@ int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, dou
     double* part = wdev + d;                // [g][d]
     cudaStream_t st = pb.stream;
 
+    std::vector<double> hostv(d);
     if (P.center) {
         k_colmean<<<g, 256, 0, st>>>(X_in, P.n, d, part);
         k_colmean_fin<<<(d + 255) / 256, 256, 0, st>>>(part, g, d, P.n, mean);
         pb.count(2);
+        if (pb.shard) {
+            // global mean = (sum over ranks of the local column sums) / n_global, summed on the host in rank order
+            if (cudaMemcpyAsync(hostv.data(), mean, sizeof(double) * d, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+                cudaStreamSynchronize(st) != cudaSuccess)
+                return GEM_NLR_E_CUDA;
+            for (int j = 0; j < d; ++j) hostv[j] *= (double)P.n;
+            if (pb.shard->host_sum(pb.shard->ctx, hostv.data(), d) != 0) return GEM_NLR_E_CUDA;
+            for (int j = 0; j < d; ++j) hostv[j] /= (double)pb.shard->n_global;
+            if (cudaMemcpyAsync(mean, hostv.data(), sizeof(double) * d, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+                cudaStreamSynchronize(st) != cudaSuccess)
+                return GEM_NLR_E_CUDA;
+        }
     } else {
         cudaMemsetAsync(mean, 0, sizeof(double) * d, st);
     }
@@ -281,6 +294,8 @@ int run_spectral_norm(const Problem& pb, const float* X_in, float* Xhat_out, dou
         if (cudaMemcpyAsync(w.data(), wdev, sizeof(double) * d, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return GEM_NLR_E_CUDA;
         if (cudaStreamSynchronize(st) != cudaSuccess) return GEM_NLR_E_CUDA;
+        // row-sharded: X_c^T X_c v is the sum of the ranks' products (every rank then runs the same recurrence)
+        if (pb.shard && pb.shard->host_sum(pb.shard->ctx, w.data(), d) != 0) return GEM_NLR_E_CUDA;
         double ak = 0.0;
         for (int j = 0; j < d; ++j) ak += vk[j] * w[j];
         if (!isfinite(ak)) return GEM_NLR_E_NONFINITE;

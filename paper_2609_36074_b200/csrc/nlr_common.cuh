@@ -25,6 +25,12 @@ struct Ctl {
     double  f_final;        // objective at the current iterate when the stop test fired
     gem_nlr_iter_info last; // latest iteration (rho/stop filled in when its tail has run)
     uint32_t counter[4];    // arrival counters for last-block reductions (always left at zero)
+    // Row-sharded runs (several GPUs, each with a block of rows): with shard_world > 1 the scalar steps inside the
+    // iteration kernels only park their local sums here (and in the Theta, s, p buffers); the sums of all ranks
+    // are combined, in rank order, by the exchange kernels, which then take the scalar step on every rank alike.
+    int32_t shard_world;    // 0 or 1: not sharded
+    int32_t pad_;
+    double  sa, sb, sh;     // parked local a, b, h
 };
 
 struct Layout {
@@ -48,7 +54,19 @@ constexpr int G2_TM = 64, G2_RT = 64, G2_DT = 32;    // generic pass-2 tile
 
 Layout make_layout(const gem_nlr_params& P);
 
+// Host-side description of a row-sharded run (owned by the handle).
+struct ShardInfo {
+    int rank, world;
+    int64_t n_global;                       // rows over all ranks: gamma = beta / n_global, rho = ||q|| / sqrt(n_global)
+    gem_nlr_gather_fn gather;               // all-gather of equal-sized device records, in rank order, on a stream
+    gem_nlr_host_sum_fn host_sum;           // in-place sum of a host FP64 vector over the ranks, in rank order
+    void* ctx;
+    double* xbuf;                           // device exchange area: [count] send, then [world][count] receive
+    size_t xcount;                          // doubles per record the area was sized for
+};
+
 struct Problem {
+    const ShardInfo* shard;                 // null: single GPU
     gem_nlr_params P;
     int dx;          // features per row of X as stored (row pitch).  P.d equals dx except in the view the
                      // fp16-image tensor-core kernels get, where P.d is dx rounded up to a multiple of 32:
@@ -111,6 +129,15 @@ void launch_fin2(const Problem& pb, int gx, int gy, int cols_per);
 void launch_tail(const Problem& pb);
 void launch_objective(const Problem& pb);                   // fills ctl->f_final for the current (U, y)
 void launch_labels(const Problem& pb, int32_t* labels);
+
+// ---- row-sharded runs (kernels_shard.cu): exchange of the small replicated quantities ----------
+// After the first phase (local Theta, s, sum q^2, sum ytilde q parked): gather, combine in rank order, scalar step
+// with the mode of the deferred call (0 iteration, 1 tail, 2 objective).  Returns a GEM_NLR_* code.
+int shard_exchange_first(const Problem& pb, int mode);
+// After the second product (local a, b, h parked, local column sums in p): gather, combine, multiplier, gate, p.
+// colsum_only: just p = sum of the ranks' column sums (a freshly loaded factor).
+int shard_exchange_second(const Problem& pb, int colsum_only);
+size_t shard_record_doubles(const gem_nlr_params& P, int dp);
 
 // ---- self-test of the bounded waits (selftest.cu) ------------------------------------------
 void launch_selftest_wait(const Problem& pb, uint32_t max_polls, long long* cycles_dev /* 2 entries */);
