@@ -63,17 +63,18 @@ def _peaks():
 # Keyed by (n, d, r, kernel path) -> {phase: (bytes, profile file)}; anything else reports null.
 NCU_TRAFFIC = {
     (1_000_000, 128, 16, "mma.tf32x3"): {
-        "second": (640.0e6, "profiles/mma_tf32x3_128x16_config2_medium.md"),
-        "first": (585.6e6, "profiles/mma_tf32x3_128x16_config2_medium.md")},
+        "second": (635.9e6, "profiles/mma_tf32x3_128x16_config2_medium.md"),
+        "first": (587.1e6, "profiles/mma_tf32x3_128x16_config2_medium.md")},
     (10_000_000, 64, 100, "f16x3"): {
         "second": (10.36e9, "profiles/tcgen05_64x100_config3_many_cluster.md"),
-        "first": (6.72e9, "profiles/tcgen05_64x100_config3_many_cluster.md")},
+        "first": (7.29e9, "profiles/tcgen05_64x100_config3_many_cluster.md")},
+    # first phase of the tiled family: the first-product kernel alone (the separate vector pass reads U once more)
     (2_000_000, 768, 1000, "f16x3.tiled"): {
-        "second": (21.52e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md"),
-        "first": (14.6e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md")},
+        "second": (21.57e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md"),
+        "first": (18.90e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md")},
     (100_000_000, 32, 8, "ffma"): {
-        "second": (19.49e9, "profiles/ffma_32x8_config5_massive.md"),
-        "first": (17.2e9, "profiles/ffma_32x8_config5_massive.md")},
+        "second": (19.50e9, "profiles/ffma_32x8_config5_massive.md"),
+        "first": (16.81e9, "profiles/ffma_32x8_config5_massive.md")},
 }
 
 
