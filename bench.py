@@ -298,8 +298,10 @@ def bench_config(cfg, args, dev, rank, world, local, with_cpu, with_e2e):
     U0_host = torch.empty((n, r), dtype=torch.float32, pin_memory=True)
     synth.make_u0(n, r, K, seed=rspec.seed, out=U0_host.numpy())
 
+    # x_inplace = 2: the data buffer may be given up after setup (the tensor-core shapes then keep the row-major fp16
+    # image pair in it instead of X-hat plus a separate pair in the workspace)
     kw = dict(alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"], T=T, T_min=T,
-              precision=args.precision)
+              precision=args.precision, x_inplace=2)
     Xd = X_host.to(dev, non_blocking=True)
     U0d = U0_host.to(dev, non_blocking=True)
     Ud = torch.empty_like(U0d)

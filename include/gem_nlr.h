@@ -70,7 +70,12 @@ typedef struct {
     double   eps_d;         /* dual gate:  max{c^2 a + b - 2 c h, 0} < eps_d^2 K                 */
     double   eps_c;         /* stop: gate and delta-hat < eps_c and rho < eps_c                  */
     int32_t  center;        /* 1: subtract the column mean before the spectral norm (paper)      */
-    int32_t  x_inplace;     /* 1: X_dev is overwritten by X-hat; 0: X-hat lives in the workspace */
+    int32_t  x_inplace;     /* 1: X_dev is overwritten by X-hat; 0: X-hat lives in the workspace; */
+                            /* 2: X_dev may be given up: as 1, and where both products read only  */
+                            /* the fp16 operand images the row-major image pair is built over     */
+                            /* X-hat after setup (same bytes), so the workspace holds only the    */
+                            /* transposed pair; gem_nlr_objective, gem_nlr_init_range and buffer 5 */
+                            /* then return GEM_NLR_E_INVALID (they read X-hat itself)             */
     int32_t  pi_max_iters;  /* power-iteration cap for ||X_c||_2 (<=0: 100)                      */
     double   pi_tol;        /* stop when |sigma_k - sigma_{k-1}| <= pi_tol * sigma_k (<=0: 1e-7) */
     uint64_t pi_seed;       /* seed of the starting vector                                       */

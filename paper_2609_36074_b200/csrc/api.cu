@@ -22,6 +22,7 @@ static bool valid_params(const gem_nlr_params& P)
     if (!(P.alpha > 0.f) || !(P.beta > 0.f)) return false;
     if (P.T < 0 || P.T_min < 0 || P.eps_d < 0.0 || P.eps_c < 0.0) return false;
     if (P.precision < -1 || P.precision > 3) return false;
+    if (P.x_inplace < 0 || P.x_inplace > 2) return false;
     return true;
 }
 
@@ -45,6 +46,15 @@ Layout make_layout(const gem_nlr_params& P)
     const bool tc_images = (P.precision == -1 || P.precision == 1) && r >= 32 && n >= 4096;
     const int dp = tc_images ? (d + 31) / 32 * 32 : d;
     L.dp = dp;
+    L.has_img = tc_images ? 1 : 0;
+    // x_inplace == 2: X-hat itself may be given up after setup.  Where both products read only the fp16 images (the
+    // shapes below: the resident-Theta pair and the tiled pair) the row-major image pair takes X-hat's place, which
+    // has exactly its size when d needs no padding.  The rule is deliberately narrower than the kernels' own shape
+    // tests; gem_nlr_create checks it against the kernels actually chosen.
+    const bool pair_small = d % 32 == 0 && d >= 32 && d <= 256 && r % 4 == 0 && r <= 128 && (size_t)d * r <= 16384;
+    const bool pair_tiled = d % 32 == 0 && d >= 256 && d <= 1536 && r % 4 == 0 && r > 256 && r <= 1536 &&
+                            ((r + 127) / 128) * ((d + 255) / 256) <= kSMs;
+    L.img_inplace = (P.x_inplace == 2 && tc_images && (pair_small || pair_tiled)) ? 1 : 0;
     L.nred1 = (int)ceil_div((int64_t)dp * r, 64);
 
     size_t off = 0;
@@ -77,7 +87,7 @@ Layout make_layout(const gem_nlr_params& P)
     // and transposed in blocks of fb features x 32 rows (first product): about 2 x 2 x n x d halves.
     L.n_pad = (n + 63) / 64 * 64;
     L.fb = dp >= 256 ? 256 : dp;
-    L.ximg = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)n * dp : 0);
+    L.ximg = take(tc_images && !L.img_inplace ? sizeof(uint16_t) * 2 * (size_t)n * dp : 0);
     L.ximgT = take(tc_images ? sizeof(uint16_t) * 2 * (size_t)(L.n_pad / 32) * ((dp + L.fb - 1) / L.fb) * L.fb * 32 : 0);
     L.total = off;
     return L;
@@ -110,6 +120,7 @@ struct gem_nlr {
     TcgPlan tcg;
     Tcg1Plan tcg1;
     bool use_tcg1;         // first product by the tiled tcgen05 kernel (vector pass separate)
+    bool x_consumed;       // x_inplace == 2 in effect: after setup the X buffer holds the row-major fp16 images, not X-hat
     ShardInfo shard;       // row-sharded run: rank, world, callbacks (world <= 1: single GPU)
     char err[256];
     int64_t launches;      // kernels launched by this handle
@@ -326,6 +337,19 @@ int gem_nlr_create(gem_nlr_t** out, const gem_nlr_params* params, float* X_dev, 
             }
         }
     }
+    if (L.img_inplace) {
+        const bool both = (h->use_tc1 && h->use_tc && h->tc.f16) || (h->use_tcg1 && h->use_tcg);
+        if (both) {
+            h->x_consumed = true;
+        } else {
+            // the kernels chosen for this shape still read X-hat: keep it, build no images, iterate on the
+            // general-shape kernels (correct for every shape; the layout holds no room for separate images)
+            h->use_tc = h->use_tc1 = h->use_tcg = h->use_tcg1 = false;
+            h->pb.L.has_img = h->pbp.L.has_img = 0;
+            h->pb.L.img_inplace = h->pbp.L.img_inplace = 0;
+            h->path = h->use_mma ? "mma.tf32x3" : h->use_ffma ? "ffma" : "generic";
+        }
+    }
     if (cudaMallocHost((void**)&h->host_ctl, sizeof(Ctl)) != cudaSuccess ||
         cudaMallocHost((void**)&h->host_scratch, 64) != cudaSuccess) {
         if (h->host_ctl) cudaFreeHost(h->host_ctl);
@@ -435,6 +459,7 @@ int gem_nlr_init_range(gem_nlr_t* h)
     if (h->sticky_error) return h->sticky_error;
     if (!h->normalized) return GEM_NLR_E_NOT_READY;
     if (h->pb.shard) return GEM_NLR_E_INVALID;                // single-GPU call
+    if (h->x_consumed) return GEM_NLR_E_INVALID;              // X-hat itself was given up (x_inplace == 2)
     if (h->pb.P.r > h->pb.P.d) return GEM_NLR_E_INVALID;      // the sample X-hat X-hat^T Z has rank <= d
     int rc = reset_ctl(h, 0);                                 // multiplier 1, no gate pending, not stopped
     if (rc) return rc;
@@ -535,6 +560,7 @@ int gem_nlr_objective(gem_nlr_t* h, double* fhat_out)
 {
     if (!h || !fhat_out) return GEM_NLR_E_INVALID;
     if (!h->normalized) return GEM_NLR_E_NOT_READY;
+    if (h->x_consumed) return GEM_NLR_E_INVALID;              // the stand-alone evaluation reads X-hat itself
     int rc = ensure_loaded(h);
     if (rc) return rc;
     launch_objective(h->pb);
@@ -592,7 +618,10 @@ int gem_nlr_buffer(gem_nlr_t* h, int32_t which, void** ptr_dev)
         case 2: *ptr_dev = h->pb.s(); break;
         case 3: *ptr_dev = h->pb.ytilde(); break;
         case 4: *ptr_dev = h->pb.ybar(); break;
-        case 5: *ptr_dev = h->pb.X; break;
+        case 5:
+            if (h->x_consumed && h->normalized) return GEM_NLR_E_INVALID;
+            *ptr_dev = h->pb.X;
+            break;
         default: return GEM_NLR_E_INVALID;
     }
     return GEM_NLR_OK;
@@ -664,7 +693,7 @@ size_t gem_nlr_host_job_device_bytes(const gem_nlr_params* params)
 {
     if (!params || !valid_params(*params)) return 0;
     gem_nlr_params P = *params;
-    P.x_inplace = 1;
+    P.x_inplace = 2;                                          // the device copy of X belongs to the job
     const size_t n = (size_t)P.n;
     return align_up(4 * n * P.d, 256) + align_up(4 * n * P.r, 256) + align_up(4 * n, 256) +
            make_layout(P).total;
@@ -687,7 +716,7 @@ int gem_nlr_run_host_timed(const gem_nlr_params* params, const float* X_host, fl
     if (!valid_params(*params) || ((uintptr_t)device_buffer_dev & 255)) return GEM_NLR_E_INVALID;
     if (device_bytes < gem_nlr_host_job_device_bytes(params)) return GEM_NLR_E_WORKSPACE;
     gem_nlr_params P = *params;
-    P.x_inplace = 1;
+    P.x_inplace = 2;                                          // the device copy of X belongs to the job
     const size_t n = (size_t)P.n;
     char* base = (char*)device_buffer_dev;
     float* Xd = (float*)base;

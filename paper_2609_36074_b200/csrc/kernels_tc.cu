@@ -485,8 +485,8 @@ bool tc_plan(const Problem& pb, TcPlan* pl, float* img_storage)
     pl->img_lo = f16 ? reinterpret_cast<float*>(reinterpret_cast<uint16_t*>(img_storage) + (size_t)NB * 32 * NP)
                      : img_storage + (size_t)NB * 32 * NP;
     if (f16) {
-        if (!make_tensor_map_2d_f16(&pl->tmX, pb.ximg(0), pb.P.n, d, d, tc::TILE_M, 32)) return false;
-        if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, d, tc::TILE_M, 32)) return false;
+        if (!make_tensor_map_2d_f16(&pl->tmX, pb.ximg(0), pb.P.n, d, pb.ximg_pitch(), tc::TILE_M, 32)) return false;
+        if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, pb.ximg_pitch(), tc::TILE_M, 32)) return false;
     } else {
         if (!make_tensor_map_2d(&pl->tmX, pb.X, pb.P.n, d, tc::TILE_M, 32)) return false;
         pl->tmX2 = pl->tmX;

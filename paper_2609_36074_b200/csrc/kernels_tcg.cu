@@ -105,6 +105,53 @@ k_ximg_build(const float* __restrict__ X, int64_t n, int dx, int d, int64_t n_pa
     }
 }
 
+// The same images when X-hat itself may be given up (x_inplace == 2, d a multiple of 32): the row-major pair is
+// written over X-hat, row by row (row i: d halves of h1 followed by d halves of h2 in the 4 d bytes of its FP32
+// row, so each image has a row pitch of 2 d halves).  A block owns whole stages of 32 rows: it reads all of their
+// FP32 entries into shared memory before it writes any of their bytes.
+__global__ void __launch_bounds__(256)
+k_ximg_build_inplace(float* X, int64_t n, int d, int64_t n_pad, int fb, __half* __restrict__ h1T, __half* __restrict__ h2T)
+{
+    extern __shared__ float xs[];                          // [32][d + 1]
+    const int pitch = d + 1;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    __half* X16 = reinterpret_cast<__half*>(X);
+    const int64_t n_stages = n_pad / 32;
+    const int nnb = (d + fb - 1) / fb;
+    for (int64_t st = blockIdx.x; st < n_stages; st += gridDim.x) {
+        const int64_t row0 = st * 32;
+        for (int idx = threadIdx.x; idx < 32 * d; idx += 256) {
+            const int rr = idx / d, f = idx - rr * d;
+            xs[rr * pitch + f] = (row0 + rr < n) ? X[(row0 + rr) * d + f] * 32768.0f : 0.f;
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < 32 * d; idx += 256) {
+            const int rr = idx / d, f = idx - rr * d;
+            if (row0 + rr < n) {
+                const float v = xs[rr * pitch + f];
+                const __half a = __float2half_rn(v);
+                const __half b = __float2half_rn(v - __half2float(a));
+                X16[(row0 + rr) * 2 * d + f] = a;
+                X16[(row0 + rr) * 2 * d + d + f] = b;
+            }
+        }
+        for (int f0 = 0; f0 < d; f0 += 32) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int f = f0 + ty + 8 * i;
+                const float v = xs[tx * pitch + f];        // row tx of the stage, feature f
+                const __half a = __float2half_rn(v);
+                const __half b = __float2half_rn(v - __half2float(a));
+                const int nbk = f / fb, m = f - nbk * fb, kk = tx;
+                const size_t off = (((size_t)st * nnb + nbk) * fb + m) * 32 + (size_t)((((kk >> 3) ^ ((m >> 1) & 3)) << 3) + (kk & 7));
+                h1T[off] = a;
+                h2T[off] = b;
+            }
+        }
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
             const __half* __restrict__ img_h1, const __half* __restrict__ img_h2, float* __restrict__ U,
@@ -622,8 +669,8 @@ bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
     if (pl->smem2 > 227 * 1024 - 1024) return false;
     pl->img_h1 = img_storage;
     pl->img_h2 = reinterpret_cast<uint16_t*>(img_storage) + (size_t)d * RP;
-    if (!make_tensor_map_2d_f16(&pl->tmX1, pb.ximg(0), pb.P.n, d, d, tcg::TILE_M, tcg::KC)) return false;
-    if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, d, tcg::TILE_M, tcg::KC)) return false;
+    if (!make_tensor_map_2d_f16(&pl->tmX1, pb.ximg(0), pb.P.n, d, pb.ximg_pitch(), tcg::TILE_M, tcg::KC)) return false;
+    if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, pb.ximg_pitch(), tcg::TILE_M, tcg::KC)) return false;
     const int64_t items = (pb.P.n + tcg::TILE_M - 1) / tcg::TILE_M * NCB;
     pl->g2 = (int)(items < kSMs ? items : kSMs);
     if (cudaFuncSetAttribute(tcg::k_pass2_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
@@ -634,6 +681,15 @@ bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
 void tcg_prepare(const Problem& pb)
 {
     cudaMemsetAsync(pb.ximgT(0), 0, sizeof(uint16_t) * 2 * pb.ximgT_halves(), pb.stream);
+    if (pb.L.img_inplace) {
+        const size_t sm = sizeof(float) * 32 * (size_t)(pb.P.d + 1);
+        cudaFuncSetAttribute(tcg::k_ximg_build_inplace, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        const int64_t stages = pb.L.n_pad / 32;
+        tcg::k_ximg_build_inplace<<<(int)(stages < kSMs ? stages : kSMs), 256, sm, pb.stream>>>(
+            pb.X, pb.P.n, pb.P.d, pb.L.n_pad, pb.L.fb, reinterpret_cast<__half*>(pb.ximgT(0)), reinterpret_cast<__half*>(pb.ximgT(1)));
+        pb.count(1);
+        return;
+    }
     const dim3 grid((unsigned)((pb.L.n_pad + 31) / 32), (unsigned)((pb.P.d + 31) / 32));
     tcg::k_ximg_build<<<grid, 256, 0, pb.stream>>>(pb.X, pb.P.n, pb.dx, pb.P.d, pb.L.n_pad, pb.L.fb,
                                                    reinterpret_cast<__half*>(pb.ximg(0)), reinterpret_cast<__half*>(pb.ximg(1)),

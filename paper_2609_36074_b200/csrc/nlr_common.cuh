@@ -38,6 +38,9 @@ struct Layout {
     size_t init;             // FP64 scratch of the data-informed start: M, C, T, G (0 bytes when r > d)
     size_t part1_bytes;      // size of the split-K partial area
     size_t ximg, ximgT;      // fp16 split images of X-hat (row-major and transposed), wide tensor-core shapes only (else 0 bytes)
+    int has_img;             // the fp16 images of X-hat exist (tensor-core shapes)
+    int img_inplace;         // x_inplace == 2 and both products read images only: the row-major image pair is built over
+                             // X-hat in the caller's X buffer (row i: d halves of h1, then d halves of h2) and ximg is 0 bytes
     int dp;                  // d rounded up to a multiple of 32 when the fp16 images exist, else d: feature count of the image kernels
     int64_t n_pad;           // n rounded up to 64: the transposed images cover n_pad / 32 stages of 32 rows
     int fb;                  // features per block of the transposed images: 256, or d when d < 256
@@ -87,11 +90,16 @@ struct Problem {
     float* alpha_s() const { return reinterpret_cast<float*>(ws + L.alpha_s); }
     float* theta() const { return reinterpret_cast<float*>(ws + L.theta); }
     // fp16 split images of X-hat (wide tensor-core shapes): h1 then h2, row-major n x d; transposed d x n_pad
-    uint16_t* ximg(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximg) + (size_t)which * P.n * P.d; }
+    uint16_t* ximg(int which) const
+    {
+        if (L.img_inplace) return reinterpret_cast<uint16_t*>(X) + (size_t)which * P.d;
+        return reinterpret_cast<uint16_t*>(ws + L.ximg) + (size_t)which * P.n * P.d;
+    }
+    int64_t ximg_pitch() const { return L.img_inplace ? 2 * (int64_t)P.d : (int64_t)P.d; }   // halves between rows of an image
     // transposed images: [n_pad / 32 stages][ceil(d / fb) blocks][fb features][32 rows] halves each
     size_t ximgT_halves() const { return (size_t)(L.n_pad / 32) * ((P.d + L.fb - 1) / L.fb) * L.fb * 32; }
     uint16_t* ximgT(int which) const { return reinterpret_cast<uint16_t*>(ws + L.ximgT) + (size_t)which * ximgT_halves(); }
-    bool has_ximg() const { return L.ximgT > L.ximg; }
+    bool has_ximg() const { return L.has_img != 0; }
     float* ytilde() const { return reinterpret_cast<float*>(ws + L.ytilde); }
     float* ybar() const { return reinterpret_cast<float*>(ws + L.ybar); }
     double* part1() const { return reinterpret_cast<double*>(ws + L.part1); }

@@ -170,3 +170,54 @@ def test_padded_feature_count_full_run_with_setup():
     assert u_err(s.U.cpu().numpy(), Uo) <= 5e-4          # the two sides normalise with their own a (1e-5 apart)
     assert rel(info["fhat"], infoo["fhat"]) <= 1e-4 and rel(info["rho"], infoo["rho"]) <= 1e-3
     s.destroy()
+
+
+# ---- x_inplace = 2: X-hat is given up after setup, the row-major fp16 images are built over it ----
+@pytest.mark.parametrize("n,d,K,path", [(8200, 64, 100, "f16x3"), (4300, 288, 600, "f16x3.tiled"), (4200, 768, 1000, "f16x3.tiled"),
+                                        (4500, 96, 36, "f16x3")])
+def test_images_built_over_xhat_give_identical_iterates(n, d, K, path):
+    import torch
+    from paper_2609_36074_b200.binding import make_params
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 1)
+    X, _, _ = synth.make_mixture(spec)
+    U0 = synth.make_u0(n, K, K, seed=1)
+    hp = dict(synth.default_hparams(K), eps_d=0.2)
+    outs = []
+    for mode in (1, 2):
+        Xd, Ud = torch.from_numpy(X.copy()).cuda(), torch.from_numpy(U0.copy()).cuda()
+        s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"], T=6, T_min=2,
+                       x_inplace=mode)
+        assert s.path() == path, s.path()
+        a = s.spectral_norm()
+        rc, info, iters = s.run()
+        assert rc >= 0 and iters == 6, (rc, s.last_error())
+        outs.append((a, s.U.cpu().numpy().copy(), info, s.labels().cpu().numpy()))
+        if mode == 2:
+            with pytest.raises(RuntimeError):
+                s.objective()                                   # reads X-hat itself: refused once it is given up
+            assert s.init_range() == gem.E_INVALID
+        s.destroy()
+    assert outs[0][0] == outs[1][0] and outs[0][2] == outs[1][2]
+    assert np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][3], outs[1][3])
+    kw = dict(alpha=hp["alpha"], beta=hp["beta"], T=6, T_min=2)
+    ws1 = gem.workspace_bytes(make_params(n, d, K, x_inplace=1, **kw))
+    ws2 = gem.workspace_bytes(make_params(n, d, K, x_inplace=2, **kw))
+    assert ws1 - ws2 >= 4 * n * d                               # the row-major pair no longer sits in the workspace
+
+
+def test_giving_up_xhat_is_only_a_permission():
+    """Shapes whose kernels still read X-hat keep it: x_inplace = 2 then behaves like 1."""
+    import torch
+    n, d, K = 5000, 32, 8                                       # FFMA family: no operand images at all
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 0)
+    X, _, _ = synth.make_mixture(spec)
+    U0 = synth.make_u0(n, K, K)
+    hp = synth.default_hparams(K)
+    Xd, Ud = torch.from_numpy(X.copy()).cuda(), torch.from_numpy(U0.copy()).cuda()
+    s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], T=3, x_inplace=2)
+    s.spectral_norm()
+    f = s.objective()
+    Xhat, _, _ = oracle.normalize(X)
+    assert np.abs(Xd.cpu().numpy() - Xhat).max() <= 2e-6 * np.abs(Xhat).max()
+    assert abs(f - oracle.objective(Xhat, U0, np.zeros(n, np.float32), hp["beta"])) <= 1e-5 * abs(f)
+    s.destroy()
