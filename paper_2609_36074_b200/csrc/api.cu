@@ -44,7 +44,11 @@ Layout make_layout(const gem_nlr_params& P)
     // feature count rounded up to a multiple of 32 (zero features in the images), so Theta, its partial records
     // and the reduction are sized for dp x r.
     const bool tc_images = (P.precision == -1 || P.precision == 1) && r >= 32 && n >= 4096;
-    const int dp = tc_images ? (d + 31) / 32 * 32 : d;
+    int dp = tc_images ? (d + 31) / 32 * 32 : d;
+    // Wide factors (r > 128) have no resident-Theta first product; the tiled one works on 256-feature blocks.  For
+    // 128 < d < 256 (the paper's d = 200 with r = 150 .. 300) the images are padded to 256 features: at most twice
+    // the tensor-core work, against a first product on the FFMA fallback otherwise.
+    if (tc_images && r > 128 && dp > 128 && dp < 256) dp = 256;
     L.dp = dp;
     L.has_img = tc_images ? 1 : 0;
     // x_inplace == 2: X-hat itself may be given up after setup.  Where both products read only the fp16 images (the
@@ -64,7 +68,14 @@ Layout make_layout(const gem_nlr_params& P)
     L.s = take(sizeof(float) * r);
     L.alpha_s = take(sizeof(float) * r);
     L.theta = take(sizeof(float) * (size_t)dp * r);
-    L.thimg = take(sizeof(float) * 2 * (size_t)((d + 31) / 32 * 32) * (r > 256 ? (r + 255) / 256 * 256 : (r + 15) / 16 * 16));
+    // Theta^T operand images: the resident-Theta kernels keep 2 x dp x pad16(r) floats (TF32 split) or halves; the tiled
+    // kernel 2 x dp x pad256(r) halves, also for r <= 256 when the resident form does not fit in shared memory
+    {
+        const size_t d32 = (size_t)((dp + 31) / 32 * 32);
+        size_t cols = r > 256 ? (size_t)((r + 255) / 256 * 256) : (size_t)((r + 15) / 16 * 16);
+        if (tc_images && cols < 128) cols = 128;
+        L.thimg = take(sizeof(float) * 2 * d32 * cols);
+    }
     L.ytilde = take(sizeof(float) * (size_t)n);
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families

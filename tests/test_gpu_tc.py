@@ -58,7 +58,8 @@ def test_tc_trajectory_matches_oracle_and_is_reproducible(n, d, K):
 
 # ---- tiled tcgen05 kernels (wide d and r: 256-column blocks, d streamed in 32-feature chunks, fp16 split) ----
 # one and several column blocks, r not a multiple of 16, ragged last row tile, more items than CTAs
-TCG_SHAPES = [(4200, 64, 300), (4100, 768, 1000), (5000, 64, 520), (21000, 32, 260), (4200, 288, 600)]
+# (4100, 1024, 48): a narrow factor whose resident Theta images do not fit in shared memory, so it takes the tiled kernels
+TCG_SHAPES = [(4200, 64, 300), (4100, 768, 1000), (5000, 64, 520), (21000, 32, 260), (4200, 288, 600), (4100, 1024, 48)]
 
 
 @pytest.mark.parametrize("n,d,K", TCG_SHAPES)
@@ -129,7 +130,8 @@ def test_tiled_tc_trajectory_on_the_embedding_shape_twin():
 # images, zero rows in Theta); includes the shapes of the paper's own scaling study (d = 50, r = 3 K) ----
 # (n, d, K, r, kernel path)
 PADDED_D_SHAPES = [(5000, 50, 60, 60, "f16x3"), (6001, 50, 20, 60, "f16x3"), (4500, 200, 100, 100, "f16x3"), (4400, 256, 128, 128, "f16x3.tiled"),
-                   (4300, 300, 400, 400, "f16x3.tiled"), (4200, 110, 300, 300, "generic+f16x3.tiled")]
+                   (4300, 300, 400, 400, "f16x3.tiled"), (4200, 110, 300, 300, "generic+f16x3.tiled"),
+                   (4300, 200, 100, 152, "f16x3.tiled"), (4200, 200, 100, 300, "f16x3.tiled")]
 
 
 @pytest.mark.parametrize("n,d,K,r,path", PADDED_D_SHAPES)
