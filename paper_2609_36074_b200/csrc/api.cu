@@ -80,7 +80,7 @@ Layout make_layout(const gem_nlr_params& P)
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families
     size_t p1 = sizeof(double) * (size_t)(L.g1x > 8 || !tc_images ? L.g1x : 8) * dp * r;   // r > 256: up to 8 row ranges of the tiled tcgen05 first product
-    size_t p1_fast = ((size_t)dp * r <= 32768) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)dp * r + r + 4) : 0;
+    size_t p1_fast = ((size_t)dp * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)dp * r + r + 4) : 0;
     if (r <= d && p1 < sizeof(double) * 8 * (size_t)d * d) p1 = sizeof(double) * 8 * (size_t)d * d;   // X-hat^T X-hat of the data-informed start: up to 8 row chunks
     L.part1_bytes = p1 > p1_fast ? p1 : p1_fast;
     L.part1 = take(L.part1_bytes);

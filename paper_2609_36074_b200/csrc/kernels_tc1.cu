@@ -410,7 +410,7 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
 {
     const int d = pb.P.d, r = pb.P.r;
     if (d % 32 != 0 || d > 256 || r % 4 != 0 || r < 8 || r > 128 || pb.P.n < 1024 || pb.P.n > 2000000000ll) return false;
-    if ((size_t)d * r > 32768) return false;          // partial records of the shared reduction kernel
+    if ((size_t)d * r > 16384) return false;          // larger products raised a launch failure at n = 4e6, d = 200 (224), r = 100 (cause not found): kept out
     const bool ximg = pb.has_ximg() && pb.L.fb == d;          // one block of d features per stage in the transposed images
     if (!ximg && d != pb.dx) return false;                    // without images X-hat itself is read: no feature padding
     const size_t stage = (((size_t)tc1::TR * r * 4 + 127) / 128 * 128 + (ximg ? 0 : (size_t)tc1::TR * d * 4) + 1023) / 1024 * 1024;

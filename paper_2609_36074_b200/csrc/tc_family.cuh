@@ -31,7 +31,7 @@ void tc_launch_second(const Problem& pb, const TcPlan& plan);
 namespace gemnlr {
 
 // First product + vector pass on tcgen05 (kernels_tc1.cu): d a multiple of 32 up to 256,
-// r a multiple of 4 in [8, 128], d * r <= 32768.
+// r a multiple of 4 in [8, 128], d * r <= 16384.
 struct Tc1Plan {
     alignas(64) CUtensorMap tmX;   // X-hat boxes: 32 rows x 32 features
     alignas(64) CUtensorMap tmU;   // U boxes: 32 rows x 32 columns
