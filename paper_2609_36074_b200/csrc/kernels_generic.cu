@@ -359,7 +359,7 @@ k_red1(const double* __restrict__ part, int g, int64_t dr, const Ctl* __restrict
 // ||Theta||^2; finishes the previous iteration (rho, stop test, history record).
 // mode 0: start of an iteration, 1: tail (also resets the multiplier after the U buffer was
 // rescaled), 2: objective evaluation only.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_fin1(Ctl* __restrict__ ctl, const double* __restrict__ part1v, int gv, const double* __restrict__ red,
        int nred, int r, int64_t n, float alpha, double gamma, double eps_c, int T_min,
        float* __restrict__ s, float* __restrict__ alpha_s, gem_nlr_iter_info* __restrict__ hist, int mode)
@@ -388,9 +388,9 @@ k_fin1(Ctl* __restrict__ ctl, const double* __restrict__ part1v, int gv, const d
     }
     if (mode != 1)
         for (int b = threadIdx.x; b < nred; b += blockDim.x) t2 += red[b];
-    qq = block_sum<256>(qq, sred);
-    yq = block_sum<256>(yq, sred);
-    t2 = block_sum<256>(t2, sred);
+    qq = block_sum<1024>(qq, sred);
+    yq = block_sum<1024>(yq, sred);
+    t2 = block_sum<1024>(t2, sred);
     if (threadIdx.x == 0) fin1_scalars(ctl, qq, yq, t2, n, gamma, eps_c, T_min, hist, mode);
 }
 
@@ -917,7 +917,7 @@ void launch_vector_pass(const Problem& pb)
 static void launch_fin1_g(const Problem& pb, int mode, int gv)
 {
     const auto& P = pb.P;
-    k_fin1<<<1, 256, 0, pb.stream>>>(pb.ctl(), pb.part1v(), gv, pb.red1(), pb.L.nred1, P.r, P.n,
+    k_fin1<<<1, 1024, 0, pb.stream>>>(pb.ctl(), pb.part1v(), gv, pb.red1(), pb.L.nred1, P.r, P.n,
                                      P.alpha, pb.gamma, P.eps_c, P.T_min, pb.s(), pb.alpha_s(),
                                      pb.hist(), mode);
     pb.count();
