@@ -324,7 +324,6 @@ def bench_config(cfg, args, dev, rank, world, local, with_cpu, with_e2e):
 
     for _ in range(args.warmup):
         one_step()
-    solver.profile(True)
     launches0 = solver.launch_count()
     torch.cuda.synchronize()
     replicas.barrier()
@@ -339,6 +338,13 @@ def bench_config(cfg, args, dev, rank, world, local, with_cpu, with_e2e):
     clocks = sampler.finish()
     ms = ev[2].elapsed_time(ev[3])
     launches = solver.launch_count() - launches0
+    # Per-phase split: the same steps once more with CUDA events around the two phases of every iteration.  The events
+    # are kept out of the timed region above because they cost the short iterations 3-7 % (config 2: 300 event
+    # records per 23 ms step); the phase times below therefore add up to slightly more than the iteration time.
+    solver.profile(True)
+    for _ in range(max(1, min(args.steps, 2))):
+        one_step()
+    torch.cuda.synchronize()
     ms_p1, ms_p2, prof_iters = solver.profile_read()
     solver.profile(False)
     ms = replicas.max_over_ranks(ms, dev)
@@ -417,7 +423,9 @@ def bench_config(cfg, args, dev, rank, world, local, with_cpu, with_e2e):
         "value": value, "ms_per_step": ms / args.steps,
         "config": {"workload": workload_name(spec, r, T),
                    "l2": "inputs larger than L2" if 4 * n * d > 126e6 else "inputs fit in L2 (latency-bound case)",
-                   "kernel_path": path, "replicas": world, "alpha": hp["alpha"], "beta": hp["beta"]},
+                   "kernel_path": path, "replicas": world, "alpha": hp["alpha"], "beta": hp["beta"],
+                   "phase_timing": "roofline phases from a second pass of the same steps with CUDA events around "
+                                   "each phase; value and roofline.iteration from the timed steps without them"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
         "cpu_baseline": cpu,
         "setup": {"spectral_norm_ms": setup_ms, "a": a, "labels_ms": labels_ms},

@@ -317,6 +317,8 @@ k_red1_fused(const double* __restrict__ part, int g, int stride, int dr, int r, 
              float* __restrict__ alpha_s, int64_t n, float alpha, double gamma, double eps_c, int T_min,
              gem_nlr_iter_info* __restrict__ hist, int mode, int ignore_stop, int combined)
 {
+    grid_dep_launch();
+    grid_dep_wait();                        // the partial records of the first-product kernel before this one
     if (!ignore_stop && ctl->stopped) return;
     __shared__ double sl[16][RED1_EB];
     __shared__ double sred[32];
@@ -631,9 +633,9 @@ bool ffma_plan(const Problem& pb, FfmaPlan* pl)
 void red1_fused_launch(const Problem& pb, int g, int mode)
 {
     const int dr = pb.P.d * pb.P.r;
-    ffma::k_red1_fused<<<(dr + pb.P.r + 2 + ffma::RED1_EB - 1) / ffma::RED1_EB, 256, 0, pb.stream>>>(
-        pb.part1(), g, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
-        pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0, 0);
+    launch_pdl(ffma::k_red1_fused, dim3((dr + pb.P.r + 2 + ffma::RED1_EB - 1) / ffma::RED1_EB), dim3(256), 0, pb.stream,
+               (const double*)pb.part1(), g, dr + pb.P.r + 2, dr, pb.P.r, pb.ctl(), pb.theta(), pb.red1(), pb.s(), pb.alpha_s(),
+               pb.P.n, pb.P.alpha, pb.gamma, pb.P.eps_c, pb.P.T_min, pb.hist(), mode, 0, 0);
     pb.count(1);
 }
 

@@ -42,6 +42,8 @@ k_pass1_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ U
     static_assert(XB % 1024 == 0 && UB % 1024 == 0 && D % 32 == 0 && R % 8 == 0, "stage alignment");
     static_assert(NCW * D * R * 4 <= NST * STAGE, "reduction scratch fits in the stage ring");
 
+    grid_dep_launch();
+    grid_dep_wait();                        // the previous kernel's U, p and control block
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -274,6 +276,8 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
     constexpr int PS = 4 + R;
     static_assert(XB % 1024 == 0 && D % 32 == 0 && R % 8 == 0 && NT <= 2, "shape");
 
+    grid_dep_launch();
+    grid_dep_wait();                        // Theta, s and the control block of the reduction kernel before this one
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -494,14 +498,14 @@ struct Shape {
     }
     static void pass1(const Problem& pb, const FfmaPlan& pl)
     {
-        k_pass1_mma<D, R, TM1, NST1><<<pl.g1, NTHREADS, smem1, pb.stream>>>(
-            pl.tm1, pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.gamma, pb.part1());
+        launch_pdl(k_pass1_mma<D, R, TM1, NST1>, dim3(pl.g1), dim3(NTHREADS), smem1, pb.stream,
+                   pl.tm1, pb.U, pb.ytilde(), pb.ybar(), pb.ctl(), pb.p(), pb.P.n, pb.gamma, pb.part1());
     }
     static void pass2(const Problem& pb, const FfmaPlan& pl)
     {
-        k_pass2_mma<D, R, NST2><<<pl.g2, NTHREADS, smem2, pb.stream>>>(
-            pl.tm2, pb.theta(), pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, pb.P.alpha, pb.P.K,
-            pb.P.eps_d, pb.part2(), pb.p());
+        launch_pdl(k_pass2_mma<D, R, NST2>, dim3(pl.g2), dim3(NTHREADS), smem2, pb.stream,
+                   pl.tm2, pb.theta(), pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, pb.P.alpha, pb.P.K,
+                   pb.P.eps_d, pb.part2(), pb.p());
     }
 };
 

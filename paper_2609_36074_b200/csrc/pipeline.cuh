@@ -146,6 +146,30 @@ __device__ __forceinline__ void mbar_wait_relaxed(uint32_t bar, uint32_t parity,
     ctl->stopped = 1;
 }
 
+// Programmatic dependent launch.  A kernel launched with launch_pdl() may become resident while its predecessor in
+// the stream is still running; grid_dep_wait() returns once that predecessor has completed and its writes are
+// visible (it returns at once when the kernel was launched the ordinary way).  grid_dep_launch() lets the next
+// kernel in the stream start becoming resident.  Used by the three kernels of the skinny-shape iteration, whose
+// launch latencies are a few per cent of a 0.23 ms iteration.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Tile load: box of the tensor map at element coordinates (x = column, y = row).  x * 4 bytes
 // must be a multiple of 16.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar)
