@@ -50,8 +50,9 @@ extern "C" {
 #define GEM_NLR_E_NONFINITE  -5   /* a, b or h is not finite                                     */
 #define GEM_NLR_E_NOT_READY  -6   /* iteration requested before X was normalized                 */
 #define GEM_NLR_E_TIMEOUT    -7   /* a bounded device-side wait (copy pipeline) ran out; the     */
-                                  /* kernel ran to its end without the data it waited for, so    */
-                                  /* U_dev and the dual are undefined afterwards: reload them    */
+                                  /* kernel ran to its end without the data it waited for (most  */
+                                  /* kernels stop storing into U_dev then), so U_dev and the     */
+                                  /* dual are undefined afterwards: reload them                  */
                                   /* (gem_nlr_set_state) before iterating again                  */
 #define GEM_NLR_E_TOO_LARGE  -8   /* size beyond the fixed capacity of a *_static entry point    */
 

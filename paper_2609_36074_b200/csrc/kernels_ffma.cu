@@ -450,6 +450,7 @@ k_pass2_ffma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
             const float yb0 = v0 ? ybar[row0] : 0.f;
             const float yb1 = v1 ? ybar[row0 + 1] : 0.f;
             mbar_wait(full_bar(s), (it / NST) & 1, &abort_flag, ctl);
+            const bool dead = abort_flag != 0;          // a wait ran out: the tile's data cannot be trusted, U is left as it is
             float acc[2][4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) { acc[0][b] = 0.f; acc[1][b] = 0.f; }
@@ -495,8 +496,8 @@ k_pass2_ffma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
                     csum[b] += wd;
                     wn[a][b] = w;
                 }
-            if (v0) *up0 = make_float4(wn[0][0], wn[0][1], wn[0][2], wn[0][3]);
-            if (v1) *up1 = make_float4(wn[1][0], wn[1][1], wn[1][2], wn[1][3]);
+            if (v0 && !dead) *up0 = make_float4(wn[0][0], wn[0][1], wn[0][2], wn[0][3]);
+            if (v1 && !dead) *up1 = make_float4(wn[1][0], wn[1][1], wn[1][2], wn[1][3]);
         }
     }
     __syncthreads();

@@ -361,6 +361,7 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
             const float yb0 = v0 ? ybar[row0] : 0.f;
             const float yb1 = v1 ? ybar[row1] : 0.f;
             mbar_wait(full_bar(s), (it / NST) & 1, &abort_flag, ctl);
+            const bool dead = abort_flag != 0;          // a wait ran out: the tile's data cannot be trusted, U is left as it is
             // one accumulator per product (hi*hi, lo*hi, hi*lo) and N tile: 3 NT independent MMA chains
             float acc[NT][4], acc1[NT][4], acc2[NT][4];
 #pragma unroll
@@ -410,8 +411,8 @@ k_pass2_mma(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ t
                     csum[nn][k & 1] += wd;
                     wn[k] = w;
                 }
-                if (v0) __stcg(reinterpret_cast<float2*>(U + row0 * R + 8 * nn + 2 * tq), make_float2(wn[0], wn[1]));
-                if (v1) __stcg(reinterpret_cast<float2*>(U + row1 * R + 8 * nn + 2 * tq), make_float2(wn[2], wn[3]));
+                if (v0 && !dead) __stcg(reinterpret_cast<float2*>(U + row0 * R + 8 * nn + 2 * tq), make_float2(wn[0], wn[1]));
+                if (v1 && !dead) __stcg(reinterpret_cast<float2*>(U + row1 * R + 8 * nn + 2 * tq), make_float2(wn[2], wn[3]));
             }
         }
     }

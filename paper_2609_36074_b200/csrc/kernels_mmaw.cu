@@ -415,6 +415,7 @@ k_pass2_mmaw(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
             const float yb0 = v0 ? ybar[row0] : 0.f;
             const float yb1 = v1 ? ybar[row1] : 0.f;
             mbar_wait(full_bar(s), (it / NST) & 1, &abort_flag, ctl);
+            const bool dead = abort_flag != 0;          // a wait ran out: the tile's data cannot be trusted, U is left as it is
             float acc[NH0][4];
 #pragma unroll
             for (int e = 0; e < NH0; ++e)
@@ -480,8 +481,8 @@ k_pass2_mmaw(const __grid_constant__ CUtensorMap tmX, const float* __restrict__ 
                     csf[e][k & 1] += w;
                     wn[k] = w;
                 }
-                if (v0 && cok) *reinterpret_cast<float2*>(U + row0 * r + c) = make_float2(wn[0], wn[1]);
-                if (v1 && cok) *reinterpret_cast<float2*>(U + row1 * r + c) = make_float2(wn[2], wn[3]);
+                if (v0 && cok && !dead) *reinterpret_cast<float2*>(U + row0 * r + c) = make_float2(wn[0], wn[1]);
+                if (v1 && cok && !dead) *reinterpret_cast<float2*>(U + row1 * r + c) = make_float2(wn[2], wn[3]);
             }
             if ((it & 3) == 3) flush_colsums();
         }

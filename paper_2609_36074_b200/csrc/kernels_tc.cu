@@ -364,7 +364,7 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                 }
                 fence_proxy_async();
                 named_bar_sync(1 + grp, GROUP_THREADS);
-                if (gt == 0) {
+                if (gt == 0 && !abort_flag) {                // after a time-out the panel cannot be trusted: U is left as it is
                     tma_store_2d(&tmU, pn * PW, (int)(t * TILE_M), pan);
                     bulk_commit();
                 }
