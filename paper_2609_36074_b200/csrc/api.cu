@@ -79,7 +79,11 @@ Layout make_layout(const gem_nlr_params& P)
     L.ytilde = take(sizeof(float) * (size_t)n);
     L.ybar = take(sizeof(float) * (size_t)n);
     // partial areas are sized for the largest user among the kernel families
-    size_t p1 = sizeof(double) * (size_t)(L.g1x > 8 || !tc_images ? L.g1x : 8) * dp * r;   // r > 256: up to 8 row ranges of the tiled tcgen05 first product
+    int p1_records = L.g1x;
+    if (tc_images && p1_records < 8) p1_records = 8;
+    if (tc_images && dp >= 256 && tiled_first_row_ranges(n, dp, r) > p1_records)
+        p1_records = tiled_first_row_ranges(n, dp, r);           // the tiled tcgen05 first product: one record per row range
+    size_t p1 = sizeof(double) * (size_t)p1_records * dp * r;
     size_t p1_fast = ((size_t)dp * r <= 16384) ? sizeof(double) * (size_t)kSMs * 2 * ((size_t)dp * r + r + 4) : 0;
     if (r <= d && p1 < sizeof(double) * 8 * (size_t)d * d) p1 = sizeof(double) * 8 * (size_t)d * d;   // X-hat^T X-hat of the data-informed start: up to 8 row chunks
     L.part1_bytes = p1 > p1_fast ? p1 : p1_fast;

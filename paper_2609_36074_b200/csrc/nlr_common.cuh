@@ -55,6 +55,22 @@ constexpr int kSMs = 148;
 constexpr int G_TM = 64, G_DT = 64, G_RT = 64;       // generic pass-1 tile
 constexpr int G2_TM = 64, G2_RT = 64, G2_DT = 32;    // generic pass-2 tile
 
+// Row ranges of the tiled tcgen05 first product (one resident CTA per 128 columns of U, 256-feature block and row
+// range): as many as fill the SMs, while every range keeps at least eight 32-row stages and the FP64 partial
+// records (one dp x r record per range) stay within 64 MB.
+inline int tiled_first_row_ranges(int64_t n, int dp, int r)
+{
+    const int tiles = ((r + 127) / 128) * ((dp + 255) / 256);
+    if (tiles > kSMs) return 0;
+    int64_t s = kSMs / tiles;
+    const int64_t rec = (int64_t)sizeof(double) * dp * r;
+    const int64_t cap = ((int64_t)64 << 20) / rec;
+    const int64_t by_rows = (n + 31) / 32 / 8;
+    if (s > cap) s = cap;
+    if (s > by_rows) s = by_rows;
+    return s < 1 ? 1 : (int)s;
+}
+
 Layout make_layout(const gem_nlr_params& P);
 
 // Host-side description of a row-sharded run (owned by the handle).
