@@ -91,6 +91,8 @@ Layout make_layout(const gem_nlr_params& P)
     L.part1v = take(sizeof(double) * (size_t)L.gv * (r + 2));
     size_t p2 = sizeof(double) * (size_t)L.g2x * L.g2y * (3 + G2_RT);
     size_t p2_fast = sizeof(double) * (size_t)kSMs * 4 * (4 + (size_t)r);
+    const size_t p2_tiled = sizeof(double) * (size_t)kSMs * (4 + 256);      // tiled tcgen05 second product: one 256-column block per CTA
+    if (p2_fast < p2_tiled) p2_fast = p2_tiled;
     L.part2 = take(p2 > p2_fast ? p2 : p2_fast);
     // generic family: nred1 block shares; fused reduction: one share per 16 entries of a record + r + 2 sums
     L.red1 = take(sizeof(double) * ((size_t)L.nred1 + ((size_t)dp * r + r + 2 + 15) / 16 + r + 2 + 8));

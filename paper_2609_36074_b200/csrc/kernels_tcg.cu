@@ -16,7 +16,14 @@
 // N = 256 an MMA runs at the tensor pipe's full rate, and the accumulator (256 TMEM columns) is
 // double-buffered, so the epilogue of one item overlaps the MMAs of the next.
 //
-//   warp 0       producer (TMA / bulk copies, 4-stage ring)
+// A CTA keeps one column block for the whole launch (CTA b: block b mod NCB, row tiles b / NCB, + lanes, ...;
+// the grid is a multiple of NCB), so only that block's p, alpha s and running column sums live in shared memory.
+// The footprint (3 x 48 KB ring + 13 KB) stays below the 164 KB carve-out step on purpose: the epilogue reads
+// and writes U straight from global memory, and the number of such requests an SM keeps in flight grows with the
+// L1 capacity the carve-out leaves (the same kernel padded to the 228 KB step is 8 % slower at d = 768 and 12 %
+// at d = 256; a fourth ring stage buys nothing).
+//
+//   warp 0       producer (TMA / bulk copies, 3-stage ring)
 //   warp 1       MMA issuer: per chunk 2 k-steps x 3 products; commits free the stage
 //   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); accumulators read in the 16x256b
 //                fragment layout and swapped between neighbouring lanes so that a thread owns 4 consecutive
@@ -41,7 +48,7 @@ constexpr int KC = 32;                        // features per chunk (64-byte fp1
 constexpr int A_BOX = TILE_M * KC * 2;        // 8 KB
 constexpr int B_BOX = NBLK * KC * 2;          // 16 KB
 constexpr int STAGE = 2 * A_BOX + 2 * B_BOX;  // 48 KB: X-hat h1, h2, Theta^T h1, h2
-constexpr int NS = 4;
+constexpr int NS = 3;                        // see the note on the shared-memory carve-out below
 constexpr int NEPI = 8;                       // epilogue warps
 constexpr int NTHREADS = (2 + NEPI) * 32;
 constexpr size_t SMEM_RING = (size_t)NS * STAGE;
@@ -172,14 +179,16 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = d / KC;
-    const int RP = NCB * NBLK;
+    const int cb = (int)(blockIdx.x % NCB);                              // this CTA's column block
+    const int lane_id = (int)(blockIdx.x / NCB), lanes = (int)(gridDim.x / NCB);
+    const int col0 = cb * NBLK;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t stage0 = smem_base;
     unsigned char* tail = smem + SMEM_RING;
-    float* sp = reinterpret_cast<float*>(tail);                         // [RP] p
-    float* sas = sp + RP;                                               // [RP] alpha s
-    double* scol = reinterpret_cast<double*>(sas + RP);                 // [RP] running column sums of W
-    float* stmp = reinterpret_cast<float*>(scol + RP);                  // [2][4][NBLK] per-quarter column sums of an item
+    float* sp = reinterpret_cast<float*>(tail);                         // [NBLK] p of the block
+    float* sas = sp + NBLK;                                             // [NBLK] alpha s
+    double* scol = reinterpret_cast<double*>(sas + NBLK);               // [NBLK] running column sums of W
+    float* stmp = reinterpret_cast<float*>(scol + NBLK);                // [2][4][NBLK] per-quarter column sums of an item
 
     const uint32_t bar0 = smem_u32(bars);
     auto xfull = [&](int s) { return bar0 + 8u * s; };
@@ -193,9 +202,9 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         abort_flag = 0;
         fence_barrier_init();
     }
-    for (int j = threadIdx.x; j < RP; j += NTHREADS) {
-        sp[j] = (j < r) ? p[j] : 0.f;
-        sas[j] = (j < r) ? alpha_s[j] : 0.f;
+    for (int j = threadIdx.x; j < NBLK; j += NTHREADS) {
+        sp[j] = (col0 + j < r) ? p[col0 + j] : 0.f;
+        sas[j] = (col0 + j < r) ? alpha_s[col0 + j] : 0.f;
         scol[j] = 0.0;
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), 512);
@@ -205,7 +214,6 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
     const uint32_t tmem_base = tmem_base_s;
 
     const int64_t n_tiles = (n + TILE_M - 1) / TILE_M;
-    const int64_t n_items = n_tiles * NCB;
     const float cf = ctl->c_f;
     // the accumulator holds (x-hat 2^15) (Theta 2^eT) sums: fold the scales into the 2 alpha factor
     const float two_alpha = 2.0f * alpha * ldexpf(1.0f, -15 - eT);
@@ -215,9 +223,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
             int64_t g = 0;
-            for (int64_t w = blockIdx.x; w < n_items && !abort_flag; w += gridDim.x) {
-                const int64_t t = w / NCB;
-                const int cb = (int)(w % NCB);
+            for (int64_t t = lane_id; t < n_tiles && !abort_flag; t += lanes) {
                 const int row0 = (int)(t * TILE_M);
                 for (int kb = 0; kb < KB; ++kb, ++g) {
                     const int s = (int)(g % NS);
@@ -245,7 +251,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
             int s = 0;
             uint32_t ph = 0;
             int i = 0;
-            for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
+            for (int64_t t = lane_id; t < n_tiles; t += lanes, ++i) {
                 const int a = i & 1;
                 // item boundary: the previous accumulator is already handed over; wait for a free one and for
                 // the first chunk
@@ -290,12 +296,11 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         // pipeline, which the tensor core's operand fetches share) as with the raw fragment's 8-byte pairs.
         const bool odd = tq & 1;
         const int cbase = 4 * (tq >> 1) + 8 * (tq & 1);
-        const int64_t my_items = (n_items > blockIdx.x) ? (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+        const int64_t my_items = (n_tiles > lane_id) ? (n_tiles - lane_id + lanes - 1) / lanes : 0;
         auto request = [&](int64_t c, float4 (&dst)[4]) {
-            const int64_t w = blockIdx.x + (c >> 3) * gridDim.x;
             const bool in = (c >> 3) < my_items;
-            const int64_t t = w / NCB;
-            const int cc = (int)(w % NCB) * NBLK + half * 128 + (int)(c & 7) * 16 + cbase;
+            const int64_t t = lane_id + (c >> 3) * lanes;
+            const int cc = col0 + half * 128 + (int)(c & 7) * 16 + cbase;
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
@@ -307,10 +312,8 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
         request(0, wq0);
         request(1, wq1);
         int i = 0;
-        for (int64_t w = blockIdx.x; w < n_items; w += gridDim.x, ++i) {
+        for (int64_t t = lane_id; t < n_tiles; t += lanes, ++i) {
             const int a = i & 1;
-            const int64_t t = w / NCB;
-            const int cb = (int)(w % NCB);
             bool valid[4];
             float nay[4];
             float* urow[4];
@@ -327,17 +330,16 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
             // chunks per item the epilogue's loads set the pace (the memory requests an SM can keep in flight
             // divided by their latency): d = 256 gains 14 %, d = 512 5 %.  With d = 768 the MMAs of an item take
             // longer than its epilogue and the extra requests cost 2 %, so long items go without.
-            if (KB <= 16 && et < TILE_M && w + gridDim.x < n_items) {
-                const int64_t wn = w + gridDim.x;
-                const int64_t rown = (wn / NCB) * TILE_M + et;
-                const int cn = (int)(wn % NCB) * NBLK;
-                if (rown < n) bulk_prefetch_l2(U + rown * (int64_t)r + cn, (uint32_t)((r - cn < NBLK ? r - cn : NBLK) * 4));
+            if (KB <= 16 && et < TILE_M && t + lanes < n_tiles) {
+                const int64_t rown = (t + lanes) * TILE_M + et;
+                if (rown < n) bulk_prefetch_l2(U + rown * (int64_t)r + col0, (uint32_t)((r - col0 < NBLK ? r - col0 : NBLK) * 4));
             }
             mbar_wait_relaxed(accfull(a), (uint32_t)(i >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
 #pragma unroll 1
             for (int jj = 0; jj < 8; ++jj) {
-                const int c = cb * NBLK + half * 128 + jj * 16 + cbase;      // this thread's four columns
+                const int lc = half * 128 + jj * 16 + cbase;                 // this thread's four columns inside the block
+                const int c = col0 + lc;
                 // acc[x2][...]: x2 = 0: rows g4, g4 + 8; x2 = 1: rows g4 + 16, g4 + 24
                 float acc[2][8];
                 const uint32_t tcol = (uint32_t)(a * NBLK + half * 128 + jj * 16);
@@ -347,8 +349,8 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
 #pragma unroll
                 for (int x = 0; x < 4; ++x) { wold[x] = wq0[x]; wq0[x] = wq1[x]; }
                 request((int64_t)i * 8 + jj + 2, wq1);
-                const float4 p4 = *reinterpret_cast<const float4*>(sp + c);
-                const float4 s4 = *reinterpret_cast<const float4*>(sas + c);
+                const float4 p4 = *reinterpret_cast<const float4*>(sp + lc);
+                const float4 s4 = *reinterpret_cast<const float4*>(sas + lc);
                 const bool cok = c < r;
                 tmem_ld_wait();
                 float cs[4] = {0.f, 0.f, 0.f, 0.f};
@@ -396,7 +398,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
             {
                 const float* t4 = stmp + (size_t)(a * 4) * NBLK + et;
                 const double v = (((double)t4[0] + (double)t4[NBLK]) + (double)t4[2 * NBLK]) + (double)t4[3 * NBLK];
-                scol[cb * NBLK + et] += v;
+                scol[et] += v;
             }
         }
     }
@@ -405,13 +407,13 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 
     // ---- CTA partial: a, b, h and the column sums of W ----
-    const int PS = 4 + r;
+    const int PS = 4 + NBLK;
     sa = block_sum<NTHREADS>(sa, sred);
     sb = block_sum<NTHREADS>(sb, sred);
     sh = block_sum<NTHREADS>(sh, sred);
     double* out = part + (size_t)blockIdx.x * PS;
     if (threadIdx.x == 0) { out[0] = sa; out[1] = sb; out[2] = sh; out[3] = 0.0; }
-    for (int j = threadIdx.x; j < r; j += NTHREADS) out[4 + j] = scol[j];
+    for (int j = threadIdx.x; j < NBLK; j += NTHREADS) out[4 + j] = scol[j];
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -440,8 +442,10 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
     __syncthreads();
     if (!sok) return;
     for (int j = threadIdx.x; j < r; j += NTHREADS) {
+        // column j belongs to the CTAs of block j / NBLK: fixed order over their row lanes
+        const int cj = j / NBLK, k = j % NBLK;
         double v = 0.0;
-        for (int i = 0; i < G; ++i) v += __ldcg(part + (size_t)i * PS + 4 + j);
+        for (int l = 0; l < lanes; ++l) v += __ldcg(part + (size_t)(l * NCB + cj) * PS + 4 + k);
         p_out[j] = (float)(sc * v);
     }
 }
@@ -676,14 +680,16 @@ bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
         frexpf(sqrtf((float)pb.P.K), &e);                  // |Theta_jk| <= ||X-hat||_2 ||U||_F = sqrt(K) <= 2^e
         pl->eT = 14 - e;
     }
-    pl->smem2 = tcg::SMEM_RING + (size_t)RP * (4 + 4 + 8) + (size_t)2 * 4 * tcg::NBLK * 4 + 1024;
+    pl->smem2 = tcg::SMEM_RING + (size_t)tcg::NBLK * (4 + 4 + 8) + (size_t)2 * 4 * tcg::NBLK * 4 + 1024;
     if (pl->smem2 > 227 * 1024 - 1024) return false;
     pl->img_h1 = img_storage;
     pl->img_h2 = reinterpret_cast<uint16_t*>(img_storage) + (size_t)d * RP;
     if (!make_tensor_map_2d_f16(&pl->tmX1, pb.ximg(0), pb.P.n, d, pb.ximg_pitch(), tcg::TILE_M, tcg::KC)) return false;
     if (!make_tensor_map_2d_f16(&pl->tmX2, pb.ximg(1), pb.P.n, d, pb.ximg_pitch(), tcg::TILE_M, tcg::KC)) return false;
-    const int64_t items = (pb.P.n + tcg::TILE_M - 1) / tcg::TILE_M * NCB;
-    pl->g2 = (int)(items < kSMs ? items : kSMs);
+    // one column block per CTA: (SMs / NCB) row lanes x NCB blocks
+    const int64_t tiles = (pb.P.n + tcg::TILE_M - 1) / tcg::TILE_M;
+    const int64_t lanes = tiles < kSMs / NCB ? tiles : kSMs / NCB;
+    pl->g2 = (int)lanes * NCB;
     if (cudaFuncSetAttribute(tcg::k_pass2_tcg, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl->smem2) != cudaSuccess)
         return false;
     return true;
