@@ -17,20 +17,24 @@
 // double-buffered, so the epilogue of one item overlaps the MMAs of the next.
 //
 // A CTA keeps one column block for the whole launch (CTA b: block b mod NCB, row tiles b / NCB, + lanes, ...;
-// the grid is a multiple of NCB), so only that block's p, alpha s and running column sums live in shared memory.
-// The footprint (3 x 48 KB ring + 13 KB) stays below the 164 KB carve-out step on purpose: the epilogue reads
-// and writes U straight from global memory, and the number of such requests an SM keeps in flight grows with the
-// L1 capacity the carve-out leaves (the same kernel padded to the 228 KB step is 8 % slower at d = 768 and 12 %
-// at d = 256; a fourth ring stage buys nothing).
+// the grid is a multiple of NCB), so only that block's p, alpha s and running column sums live in shared memory
+// and its Theta^T boxes stay hot in L2.
 //
-//   warp 0       producer (TMA / bulk copies, 3-stage ring)
+//   warp 0       producer (TMA / bulk copies, 3-stage ring; a fourth stage buys nothing)
 //   warp 1       MMA issuer: per chunk 2 k-steps x 3 products; commits free the stage
 //   warps 2-9    epilogue: warp = (TMEM lane quarter, column half); accumulators read in the 16x256b
 //                fragment layout and swapped between neighbouring lanes so that a thread owns 4 consecutive
-//                columns; old U entries straight from global memory (every 4-lane group reads and writes 64
-//                contiguous bytes of a row), requested two 16-column groups ahead; statistics in
-//                FP32 over a thread's 16 entries of a group, then FP64; column sums by warp shuffles,
-//                combined across the four quarters in fixed order
+//                columns; the old entries of U are read from, and the new ones written into, the group's
+//                panel in shared memory; statistics in FP32 over a thread's 16 entries of a group, then FP64;
+//                column sums by warp shuffles, combined across the four quarters in fixed order
+//   warp 10      U panel manager: panels of 128 rows x 32 columns (128-byte rows, 128-byte swizzle) by TMA into a
+//                ring of four slots, one panel ahead per column half, and back to U by TMA from the same slot
+// What sets the pace: everything that touches an SM's shared-memory array (TMA fills, the MMAs' operand fetches,
+// the panels) shares about 128 bytes per clock; an item moves 24 x 120 KB of operands and 512 KB of panels, i.e.
+// 26 thousand cycles against 18.6 thousand of tensor time, and that is the measured item period at d = 768.
+// An earlier epilogue read and wrote U straight from global memory; its speed depended on the L1 capacity the
+// shared-memory carve-out left (a 217 KB footprint was 8-12 % slower than a 157 KB one) and it set the pace at
+// every d; through the panels the d = 256 shapes gain 9 % and d = 768 is unchanged.
 // Every mbarrier wait is bounded (error status GEM_NLR_E_TIMEOUT, kernel runs to its end, TMEM freed).
 #include "nlr_common.cuh"
 #include "device_utils.cuh"
@@ -50,8 +54,11 @@ constexpr int B_BOX = NBLK * KC * 2;          // 16 KB
 constexpr int STAGE = 2 * A_BOX + 2 * B_BOX;  // 48 KB: X-hat h1, h2, Theta^T h1, h2
 constexpr int NS = 3;                        // see the note on the shared-memory carve-out below
 constexpr int NEPI = 8;                       // epilogue warps
-constexpr int NTHREADS = (2 + NEPI) * 32;
+constexpr int NTHREADS = (3 + NEPI) * 32;     // + producer, MMA issuer, U panel manager
 constexpr size_t SMEM_RING = (size_t)NS * STAGE;
+constexpr int NPAN = 4;                       // U panel slots
+constexpr int PAN_BYTES = TILE_M * 32 * 4;    // panel = 128 rows x 32 columns FP32 (128-byte rows, 128-byte swizzle): 16 KB
+constexpr int W_PANEL = 2 + NEPI;             // warp index of the panel manager
 
 // Theta (d x r, FP32 row-major) -> fp16 images h1, h2 of Theta^T 2^eT as K-major 64-byte-swizzled boxes:
 // box (kb, cb) = features 32 kb .. 32 kb + 31 of columns 256 cb .. 256 cb + 255 (zero beyond r).
@@ -161,7 +168,7 @@ k_ximg_build_inplace(float* X, int64_t n, int d, int64_t n_pad, int fb, __half* 
 
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
-            const __half* __restrict__ img_h1, const __half* __restrict__ img_h2, float* __restrict__ U,
+            const __grid_constant__ CUtensorMap tmU, const __half* __restrict__ img_h1, const __half* __restrict__ img_h2, float* __restrict__ U,
             const float* __restrict__ ybar, const float* __restrict__ p, const float* __restrict__ alpha_s,
             Ctl* __restrict__ ctl, int64_t n, int d, int r, int NCB, int eT, float alpha, int K, double eps_d,
             double* __restrict__ part, float* __restrict__ p_out)
@@ -169,7 +176,7 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
     if (ctl->stopped) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * NS + 4];
+    __shared__ __align__(8) uint64_t bars[2 * NS + 4 + 2 * NPAN];
     __shared__ uint32_t abort_flag;
     __shared__ uint32_t tmem_base_s;
     __shared__ double sred[32];
@@ -184,7 +191,8 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
     const int col0 = cb * NBLK;
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t stage0 = smem_base;
-    unsigned char* tail = smem + SMEM_RING;
+    const uint32_t pan0 = stage0 + (uint32_t)SMEM_RING;                 // NPAN panel slots
+    unsigned char* tail = smem + SMEM_RING + (size_t)NPAN * PAN_BYTES;
     float* sp = reinterpret_cast<float*>(tail);                         // [NBLK] p of the block
     float* sas = sp + NBLK;                                             // [NBLK] alpha s
     double* scol = reinterpret_cast<double*>(sas + NBLK);               // [NBLK] running column sums of W
@@ -195,10 +203,13 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
     auto xfree = [&](int s) { return bar0 + 8u * (NS + s); };
     auto accfull = [&](int a) { return bar0 + 8u * (2 * NS + a); };
     auto accfree = [&](int a) { return bar0 + 8u * (2 * NS + 2 + a); };
+    auto pfull = [&](int s) { return bar0 + 8u * (2 * NS + 4 + s); };            // panel landed
+    auto pdone = [&](int s) { return bar0 + 8u * (2 * NS + 4 + NPAN + s); };     // its four warps have written W into it
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(xfull(s), 1); mbar_init(xfree(s), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(accfull(a), 1); mbar_init(accfree(a), NEPI); }
+        for (int s = 0; s < NPAN; ++s) { mbar_init(pfull(s), 1); mbar_init(pdone(s), 4); }
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -276,64 +287,66 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                 umma_commit(accfull(a));
             }
         }
+    } else if (warp == W_PANEL) {
+        // ------------------------------ U panel manager ------------------------------
+        // Panels (128 rows x 32 columns of U) in the order the epilogue consumes them: item, pair of 16-column
+        // groups, column half.  A slot is loaded NPAN panels ahead, rewritten in place by the four warps of its
+        // half and stored from the same slot; it is loaded again once that store has read it.
+        if (lane == 0) {
+            const int64_t my_items = (n_tiles > lane_id) ? (n_tiles - lane_id + lanes - 1) / lanes : 0;
+            const int64_t total = my_items * 8;
+            auto px = [&](int64_t pi) { return col0 + (int)(pi & 1) * 128 + (int)((pi >> 1) & 3) * 32; };
+            auto py = [&](int64_t pi) { return (int)((lane_id + (pi >> 3) * lanes) * TILE_M); };
+            auto load = [&](int64_t pi) {
+                const int s = (int)(pi % NPAN);
+                mbar_expect_tx(pfull(s), PAN_BYTES);
+                tma_load_2d(pan0 + (uint32_t)s * PAN_BYTES, &tmU, px(pi), py(pi), pfull(s));
+            };
+            for (int64_t pi = 0; pi < NPAN && pi < total; ++pi) load(pi);
+            for (int64_t pi = 0; pi < total; ++pi) {
+                const int s = (int)(pi % NPAN);
+                mbar_wait_backoff(pdone(s), (uint32_t)(pi / NPAN) & 1, &abort_flag, ctl);
+                if (abort_flag) break;                 // after a time-out nothing more is stored
+                if (px(pi) < r) {
+                    tma_store_2d(&tmU, px(pi), py(pi), pan0 + (uint32_t)s * PAN_BYTES);
+                    bulk_commit();
+                    bulk_wait_read<0>();
+                }
+                if (pi + NPAN < total) load(pi + NPAN);
+            }
+            bulk_wait<0>();
+        }
     } else {
         // ------------------------------ epilogue (warps 2..9) ------------------------------
         // Warp = (TMEM lane quarter q, column half).  Accumulators are read in the 16x256b fragment layout:
         // a thread holds rows q*32 + g + {0, 8, 16, 24} (g = lane / 4) and, per 16-column group, the column
-        // pairs 8 b + 2 tq, + 1 (tq = lane % 4, b = 0, 1), so that the 4 lanes of a group read and write one
-        // full 32-byte sector of a row of U.
+        // pairs 8 b + 2 tq, + 1 (tq = lane % 4, b = 0, 1).  Neighbouring lanes (tq ^ 1) swap half of their
+        // fragment, so that a thread owns four consecutive columns of each of its rows: columns cbase ..
+        // cbase + 3 of the group with cbase = 0, 8, 4, 12 for tq = 0, 1, 2, 3.  The old entries of U come from
+        // the group's panel in shared memory and the new ones go back into it: one 16-byte access per row
+        // and direction, the eight row groups of a warp covering 512 contiguous bytes (no bank conflicts).
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
         const int g4 = lane >> 2, tq = lane & 3;
         const int et = (warp - 2) * 32 + lane;            // 0..255 among the epilogue threads
-        // The old entries of U do not depend on the accumulator: they are requested two 16-column groups
-        // ahead (across item boundaries too), so their DRAM latency is off the epilogue's critical path.
-        // Group index c = 8 (item ordinal) + jj.
-        // Neighbouring lanes (tq ^ 1) swap half of their accumulator fragment, so that a thread owns four
-        // consecutive columns of each of its rows: columns cbase .. cbase + 3 of the 16-column group with
-        // cbase = 0, 8, 4, 12 for tq = 0, 1, 2, 3.  A 4-lane group then reads and writes 64 contiguous bytes of
-        // a row with one 16-byte access per lane: half as many memory instructions (and passes through the L1
-        // pipeline, which the tensor core's operand fetches share) as with the raw fragment's 8-byte pairs.
         const bool odd = tq & 1;
         const int cbase = 4 * (tq >> 1) + 8 * (tq & 1);
-        const int64_t my_items = (n_tiles > lane_id) ? (n_tiles - lane_id + lanes - 1) / lanes : 0;
-        auto request = [&](int64_t c, float4 (&dst)[4]) {
-            const bool in = (c >> 3) < my_items;
-            const int64_t t = lane_id + (c >> 3) * lanes;
-            const int cc = col0 + half * 128 + (int)(c & 7) * 16 + cbase;
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-                const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
-                dst[x] = (in && row < n && cc < r) ? __ldcg(reinterpret_cast<const float4*>(U + row * (int64_t)r + cc))
-                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        };
-        float4 wq0[4], wq1[4];
-        request(0, wq0);
-        request(1, wq1);
+        // this thread's 16-byte chunk of panel row q*32 + g4 (+ 8 x: 1 KB further, same swizzle phase g4) for the
+        // even and the odd group of a panel: chunk index (0..7 along the 128-byte row) XOR row mod 8
+        const uint32_t row_off = (uint32_t)((q * 32 + g4) * 128);
+        const uint32_t ch_even = (uint32_t)((((cbase >> 2)) ^ g4) << 4), ch_odd = (uint32_t)(((4 + (cbase >> 2)) ^ g4) << 4);
         int i = 0;
         for (int64_t t = lane_id; t < n_tiles; t += lanes, ++i) {
             const int a = i & 1;
             bool valid[4];
             float nay[4];
-            float* urow[4];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int64_t row = t * TILE_M + q * 32 + g4 + 8 * x;
                 valid[x] = row < n;
                 nay[x] = valid[x] ? -alpha * ybar[row] : 0.f;
-                urow[x] = U + (valid[x] ? row : 0) * (int64_t)r;
             }
             float* my_tmp = stmp + (size_t)(a * 4 + q) * NBLK + half * 128;
-            // The next item's tile of U (128 rows x up to 1 KB) is asked into L2, one contiguous request per row, an
-            // item ahead of its 64-byte reads, which then see the latency of L2 instead of DRAM.  With few feature
-            // chunks per item the epilogue's loads set the pace (the memory requests an SM can keep in flight
-            // divided by their latency): d = 256 gains 14 %, d = 512 5 %.  With d = 768 the MMAs of an item take
-            // longer than its epilogue and the extra requests cost 2 %, so long items go without.
-            if (KB <= 16 && et < TILE_M && t + lanes < n_tiles) {
-                const int64_t rown = (t + lanes) * TILE_M + et;
-                if (rown < n) bulk_prefetch_l2(U + rown * (int64_t)r + col0, (uint32_t)((r - col0 < NBLK ? r - col0 : NBLK) * 4));
-            }
             mbar_wait_relaxed(accfull(a), (uint32_t)(i >> 1) & 1, &abort_flag, ctl);
             tc_fence_after();
 #pragma unroll 1
@@ -345,13 +358,16 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                 const uint32_t tcol = (uint32_t)(a * NBLK + half * 128 + jj * 16);
                 tmem_ld_16x256b_x2(tmem_base + ((uint32_t)(q * 32) << 16) + tcol, acc[0]);
                 tmem_ld_16x256b_x2(tmem_base + ((uint32_t)(q * 32 + 16) << 16) + tcol, acc[1]);
-                float4 wold[4];
-#pragma unroll
-                for (int x = 0; x < 4; ++x) { wold[x] = wq0[x]; wq0[x] = wq1[x]; }
-                request((int64_t)i * 8 + jj + 2, wq1);
+                const uint32_t pidx = ((uint32_t)i * 4u + (uint32_t)(jj >> 1)) * 2u + (uint32_t)half;   // this CTA's panel ordinal
+                const int slot = (int)(pidx % NPAN);
+                const uint32_t pan = pan0 + (uint32_t)slot * PAN_BYTES + row_off + ((jj & 1) ? ch_odd : ch_even);
                 const float4 p4 = *reinterpret_cast<const float4*>(sp + lc);
                 const float4 s4 = *reinterpret_cast<const float4*>(sas + lc);
                 const bool cok = c < r;
+                if (!(jj & 1)) mbar_wait_relaxed(pfull(slot), (pidx / NPAN) & 1u, &abort_flag, ctl);
+                float4 wold[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) wold[x] = lds128(pan + (uint32_t)x * 1024u);
                 tmem_ld_wait();
                 float cs[4] = {0.f, 0.f, 0.f, 0.f};
                 float fa = 0.f, fb = 0.f, fh = 0.f;     // FP32 over the thread's 16 entries of the group, then FP64
@@ -377,7 +393,13 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
                         fa = fmaf(wv[e], wv[e], fa); fb = fmaf(u, u, fb); fh = fmaf(wv[e], u, fh);
                         cs[e] += wv[e];
                     }
-                    if (live) __stcg(reinterpret_cast<float4*>(urow[x] + c), make_float4(wv[0], wv[1], wv[2], wv[3]));
+                    sts128(pan + (uint32_t)x * 1024u, make_float4(wv[0], wv[1], wv[2], wv[3]));
+                }
+                // the panel's new contents are visible to the TMA store the manager issues after the four arrivals
+                if (jj & 1) {
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(pdone(slot));
                 }
                 sa += (double)fa; sb += (double)fb; sh += (double)fh;
                 // column sums over the 32 rows of the quarter: the 8 row groups g4 of the warp
@@ -680,7 +702,8 @@ bool tcg_plan(const Problem& pb, TcgPlan* pl, float* img_storage)
         frexpf(sqrtf((float)pb.P.K), &e);                  // |Theta_jk| <= ||X-hat||_2 ||U||_F = sqrt(K) <= 2^e
         pl->eT = 14 - e;
     }
-    pl->smem2 = tcg::SMEM_RING + (size_t)tcg::NBLK * (4 + 4 + 8) + (size_t)2 * 4 * tcg::NBLK * 4 + 1024;
+    pl->smem2 = tcg::SMEM_RING + (size_t)tcg::NPAN * tcg::PAN_BYTES + (size_t)tcg::NBLK * (4 + 4 + 8) + (size_t)2 * 4 * tcg::NBLK * 4 + 1024;
+    if (!make_tensor_map_2d(&pl->tmU, pb.U, pb.P.n, r, tcg::TILE_M, 32, false, 128)) return false;     // U panels: 128-byte rows, 128-byte swizzle
     if (pl->smem2 > 227 * 1024 - 1024) return false;
     pl->img_h1 = img_storage;
     pl->img_h2 = reinterpret_cast<uint16_t*>(img_storage) + (size_t)d * RP;
@@ -749,7 +772,7 @@ void tcg_launch_second(const Problem& pb, const TcgPlan& pl)
     __half* i2 = reinterpret_cast<__half*>(pl.img_h2);
     tcg::k_theta_images64<<<kSMs * 4, 256, 0, pb.stream>>>(pb.theta(), d, r, pl.NCB, pl.eT, pb.ctl(), i1, i2);
     tcg::k_pass2_tcg<<<pl.g2, tcg::NTHREADS, pl.smem2, pb.stream>>>(
-        pl.tmX1, pl.tmX2, i1, i2, pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NCB, pl.eT,
+        pl.tmX1, pl.tmX2, pl.tmU, i1, i2, pb.U, pb.ybar(), pb.p(), pb.alpha_s(), pb.ctl(), pb.P.n, d, r, pl.NCB, pl.eT,
         pb.P.alpha, pb.P.K, pb.P.eps_d, pb.part2(), pb.p());
     pb.count(2);
 }
