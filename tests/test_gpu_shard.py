@@ -59,7 +59,7 @@ def _run_sharded(X, U0, K, hp, T, world, precision=-1):
 
 # (n, d, K, world): the general-shape kernels, the warp-level tensor-core family, the tcgen05 fp16-split pair (every
 # shard keeps n >= 4096 rows), the TMA-staged FFMA family; two and three ranks, uneven row blocks
-@pytest.mark.parametrize("n,d,K,world", [(6001, 16, 4, 2), (9001, 128, 16, 2), (12400, 64, 100, 3), (10001, 32, 8, 2)])
+@pytest.mark.parametrize("n,d,K,world", [(6001, 16, 4, 2), (9001, 128, 16, 2), (12400, 64, 100, 3), (10001, 32, 8, 2), (8801, 288, 300, 2)])
 def test_sharded_run_matches_single_gpu_and_oracle(n, d, K, world):
     spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 0)
     X, _, _ = synth.make_mixture(spec)
