@@ -204,8 +204,11 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
                     }
                 }
                 for (int pn = 0; pn < NPAN; ++pn) {
-                    const int h = i * NPAN + pn, sl = h % NUP;
-                    if (h >= NUP) mbar_wait(ufree(sl), ((h / NUP) - 1) & 1, &abort_flag, ctl);
+                    // slot and phase of the panel inside its epilogue group's own part of the ring (see the epilogue)
+                    const int eg = pn % NGROUPS, depth = NUP / NGROUPS;
+                    const int cnt = i * ((NPAN - eg + NGROUPS - 1) / NGROUPS) + pn / NGROUPS;
+                    const int sl = eg + NGROUPS * (cnt % depth);
+                    if (cnt >= depth) mbar_wait(ufree(sl), ((cnt / depth) - 1) & 1, &abort_flag, ctl);
                     mbar_expect_tx(ufull(sl), PAN_BYTES);
                     tma_load_2d(upan0 + (uint32_t)sl * PAN_BYTES, &tmU, pn * PW, row0, ufull(sl));
                 }
@@ -313,9 +316,16 @@ k_pass2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUte
             tc_fence_after();
 #pragma unroll 1
             for (int pn = grp; pn < NPAN; pn += NGROUPS) {
-                const int h = i * NPAN + pn, sl = h % NUP;
+                // The ring of NUP slots is split among the groups: group grp owns slots grp, grp + NGROUPS, ... and
+                // uses them in turn for its own panels (cnt = this group's panel count so far).  A slot therefore
+                // always belongs to the same group, which sees every phase of its barrier; a wait names a phase
+                // by its parity only, and a group that met a barrier still in another group's phase would read
+                // that parity as "landed".
+                const int depth = NUP / NGROUPS;
+                const int cnt = i * ((NPAN - grp + NGROUPS - 1) / NGROUPS) + pn / NGROUPS;
+                const int sl = grp + NGROUPS * (cnt % depth);
                 const uint32_t pan = upan0 + (uint32_t)sl * PAN_BYTES;
-                mbar_wait(ufull(sl), (h / NUP) & 1, &abort_flag, ctl);
+                mbar_wait(ufull(sl), (cnt / depth) & 1, &abort_flag, ctl);
 #pragma unroll 1
                 for (int hf = 0; hf < PW / 16; ++hf) {
                     if (pn * PW + hf * 16 >= r) break;       // columns beyond r: nothing to compute, TMA clips the store
@@ -461,11 +471,11 @@ bool tc_plan(const Problem& pb, TcPlan* pl, float* img_storage)
     // lo boxes of the TF32 split (split -> MMA -> free round trip); the X-hat box ring takes what is left.
     int NSB = 0, NUP = 0, NLO = 0;
     if (f16) {
-        for (int nup = 8; nup >= 2 && !NSB; --nup)
-            for (int nsb = 6; nsb >= 4; --nsb)
+        for (int nup = 8; nup >= 4 && !NSB; nup -= 4)              // a multiple of the four epilogue groups
+            for (int nsb = 6; nsb >= (nup == 4 ? 3 : 4); --nsb)
                 if (fixed + (size_t)nsb * tc::BOX_BYTES + (size_t)nup * pan_bytes <= limit) { NSB = nsb; NUP = nup; break; }
     } else {
-        for (int nup = 4; nup >= 2 && !NSB; --nup)
+        for (int nup = 4; nup >= 4 && !NSB; nup -= 4)
             for (int nlo = 3; nlo >= 2 && !NSB; --nlo)
                 for (int nsb = tc::MAX_RING; nsb >= (nlo == 3 ? 4 : 2); --nsb)
                     if (fixed + (size_t)(nsb + nlo) * tc::BOX_BYTES + (size_t)nup * pan_bytes <= limit) {

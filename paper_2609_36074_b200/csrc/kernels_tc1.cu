@@ -417,8 +417,12 @@ bool tc1_plan(const Problem& pb, Tc1Plan* pl)
     const size_t img = (size_t)2 * tc1::UIMG + (size_t)2 * d * 64;
     const size_t limit = 227 * 1024 - 2048;
     int NLO = 0, NSR = 0;
-    for (int nlo = 4; nlo >= 2 && !NSR; --nlo)
-        for (int nsr = 6; nsr >= 3; --nsr)
+    // A wait names a phase by its parity, so no waiter may fall two phases behind its barrier.  The raw ring is
+    // a multiple of NTEAMS deep (a raw slot then always belongs to the same team, which sees every one of its
+    // phases); the image ring needs NLO >= NTEAMS (a team that has seen the MMAs of stage g - NTEAMS - NLO finish
+    // knows those of stage g - 2 NLO have).
+    for (int nlo = 4; nlo >= tc1::NTEAMS && !NSR; --nlo)
+        for (int nsr = 2 * tc1::NTEAMS; nsr >= tc1::NTEAMS; nsr -= tc1::NTEAMS)
             if ((size_t)nsr * stage + (size_t)nlo * img + 1024 <= limit) { NSR = nsr; NLO = nlo; break; }
     if (!NSR) return false;
     pl->NSR = NSR; pl->NLO = NLO; pl->ximg = ximg;

@@ -491,7 +491,15 @@ k_pass2_tcg(const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CU
 // ================================================================================================
 constexpr int TR1 = 32;                        // data rows per stage (2 k-steps of 16)
 constexpr int NT1 = 2;                         // teams of four warps on alternate stages
-constexpr int NIM1 = 3, NRAW1 = 3;             // image stages, raw U stages
+constexpr int NIM1 = 3, NRAW1 = 4;             // image stages, raw U stages
+// Ring sizes and the two alternating teams.  A wait on an mbarrier names a phase by its parity only, so a waiter
+// must never be two phases behind the barrier it polls.  NRAW1 is a multiple of NT1: a raw slot always belongs to
+// the same team, which therefore sees each of its phases (with three slots the teams took turns on a slot, and a
+// team could find the barrier still in the other team's phase, whose parity reads as "done": on a late TMA
+// load it then converted a stale slice -- one 32-row stage of a few 32-column groups wrong, about once in
+// twenty-five launches at n = 2 x 10^6 with 147 CTAs).  The image slots may rotate through both teams (NIM1 >=
+// NT1 is enough there): a team that has seen the MMAs of stage g - 2 finish knows that those of stage g - 6
+// have, so the barrier of its slot is at most one phase away from the one it names.
 constexpr int URAW1 = TR1 * 128 * 4;           // raw U slice: 32 rows x 128 columns FP32 = 16 KB
 constexpr int UIMG1 = 128 * 64;                // fp16 image of the U operand: 128 columns x 32 data rows
 constexpr int XIMG1 = 256 * 64;                // fp16 image of the X-hat operand: 256 features x 32 data rows

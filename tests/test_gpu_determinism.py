@@ -1,0 +1,56 @@
+"""Run-to-run determinism of the CUDA path: fresh handles on the same inputs give bit-identical Theta and U.
+
+Every reduction of the path has a fixed order, so two launches may differ only through a race.  The sizes are
+large on purpose (all SMs busy, millions of rows): a hand-over race in a producer/consumer ring shows up as a
+rare difference of one 32-row stage in a few column groups, about once in twenty-five launches at these sizes.
+"""
+import pytest
+import torch
+
+import synth
+import paper_2609_36074_b200 as gem
+
+pytestmark = pytest.mark.gpu
+
+
+def _padded_d(n, d, r):
+    dp = (d + 31) // 32 * 32 if (r >= 32 and n >= 4096) else d
+    if r > 128 and 128 < dp < 256:
+        dp = 256
+    return dp
+
+
+@pytest.mark.parametrize("n,d,K,r,reps,path", [
+    (2_000_000, 200, 100, 300, 40, "f16x3.tiled"),      # tiled first product on 49 row ranges, panel epilogue
+    (1_500_000, 64, 100, 100, 25, "f16x3"),             # resident-Theta pair, three conversion teams
+    (1_000_000, 256, 64, 64, 25, "f16x3"),              # same pair with the shallow raw ring
+    (1_000_000, 128, 16, 16, 25, "mma.tf32x3"),
+])
+def test_fresh_handles_agree_bit_for_bit(n, d, K, r, reps, path):
+    spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 0)
+    X = torch.empty((n, d), dtype=torch.float32)
+    synth.make_mixture(spec, out=X.numpy())
+    U0 = torch.empty((n, r), dtype=torch.float32)
+    synth.make_u0(n, r, K, seed=0, out=U0.numpy())
+    hp = synth.default_hparams(K)
+    Xd0, U0d = X.cuda(), U0.cuda()
+    dp = _padded_d(n, d, r)
+    ref = None
+    for rep in range(reps):
+        Xd, Ud = Xd0.clone(), U0d.clone()
+        s = gem.GemNlr(Xd, Ud, K, alpha=hp["alpha"], beta=hp["beta"], eps_d=hp["eps_d"], eps_c=hp["eps_c"],
+                       T=2, T_min=2, precision=-1)
+        try:
+            assert s.path() == path, s.path()
+            s.spectral_norm()
+            s.step()
+            s.step()
+            torch.cuda.synchronize()
+            theta = s.buffer(0, dp * r).clone()
+            if ref is None:
+                ref = (theta, Ud.clone())
+            else:
+                assert torch.equal(theta, ref[0]), f"Theta differs in launch {rep}: {int((theta != ref[0]).sum())} entries"
+                assert torch.equal(Ud, ref[1]), f"U differs in launch {rep}"
+        finally:
+            s.destroy()
