@@ -48,7 +48,9 @@ Layout make_layout(const gem_nlr_params& P)
     // Wide factors (r > 128) have no resident-Theta first product; the tiled one works on 256-feature blocks.  For
     // 128 < d < 256 (the paper's d = 200 with r = 150 .. 300) the images are padded to 256 features: at most twice
     // the tensor-core work, against a first product on the FFMA fallback otherwise.
-    if (tc_images && r > 128 && dp > 128 && dp < 256) dp = 256;
+    // The same padding serves r <= 128 when d r is beyond what the resident-Theta first product takes (d r <= 16384): the
+    // pair of tiled kernels then replaces a first product on the FFMA fallback.
+    if (tc_images && dp > 128 && dp < 256 && (r > 128 || (size_t)dp * r > 16384)) dp = 256;
     L.dp = dp;
     L.has_img = tc_images ? 1 : 0;
     // x_inplace == 2: X-hat itself may be given up after setup.  Where both products read only the fp16 images (the
