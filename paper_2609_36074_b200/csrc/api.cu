@@ -50,7 +50,10 @@ Layout make_layout(const gem_nlr_params& P)
     // the tensor-core work, against a first product on the FFMA fallback otherwise.
     // The same padding serves r <= 128 when d r is beyond what the resident-Theta first product takes (d r <= 16384): the
     // pair of tiled kernels then replaces a first product on the FFMA fallback.
-    if (tc_images && dp > 128 && dp < 256 && (r > 128 || (size_t)dp * r > 16384)) dp = 256;
+    // Wide factors with fewer features (64 <= d <= 128) are padded as well: up to four times the tensor-core work and
+    // image bytes of the first product, which is still several times faster than the fallback (d = 128, r = 300:
+    // 11.6 ms on the FFMA kernels).
+    if (tc_images && dp < 256 && ((r > 128 && dp >= 64) || (dp > 128 && (size_t)dp * r > 16384))) dp = 256;
     L.dp = dp;
     L.has_img = tc_images ? 1 : 0;
     // x_inplace == 2: X-hat itself may be given up after setup.  Where both products read only the fp16 images (the

@@ -131,7 +131,7 @@ def test_tiled_tc_trajectory_on_the_embedding_shape_twin():
 # images, zero rows in Theta); includes the shapes of the paper's own scaling study (d = 50, r = 3 K) ----
 # (n, d, K, r, kernel path)
 PADDED_D_SHAPES = [(5000, 50, 60, 60, "f16x3"), (6001, 50, 20, 60, "f16x3"), (4500, 200, 100, 100, "f16x3.tiled"), (4400, 256, 128, 128, "f16x3.tiled"),
-                   (4300, 300, 400, 400, "f16x3.tiled"), (4200, 110, 300, 300, "generic+f16x3.tiled"),
+                   (4300, 300, 400, 400, "f16x3.tiled"), (4200, 110, 300, 300, "f16x3.tiled"),
                    (4300, 200, 100, 152, "f16x3.tiled"), (4200, 200, 100, 300, "f16x3.tiled")]
 
 
