@@ -25,6 +25,7 @@ def _padded_d(n, d, r):
     (1_500_000, 64, 100, 100, 25, "f16x3"),             # resident-Theta pair, three conversion teams
     (1_000_000, 256, 64, 64, 25, "f16x3"),              # same pair with the shallow raw ring
     (1_000_000, 128, 16, 16, 25, "mma.tf32x3"),
+    (4_000_000, 32, 8, 8, 25, "ffma"),
 ])
 def test_fresh_handles_agree_bit_for_bit(n, d, K, r, reps, path):
     spec = synth.MixtureSpec("t", n, d, K, "equal", 16.0, "unit", 10, 0)
