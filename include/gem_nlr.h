@@ -108,7 +108,10 @@ typedef struct {
  * optional history, when x_inplace == 0 a copy of X and, for the tensor-core shapes
  * (precision -1 or 1, r >= 32, n >= 4096), the static fp16 split images of X-hat, row-major
  * and transposed (8 n d' bytes, d' = d rounded up to a multiple of 32: the image kernels see
- * zero features beyond d, so any d is accepted).                                               */
+ * zero features beyond d, so any d is accepted; d' = 256 for wide factors, r > 128 with
+ * 64 <= d < 256, and for 128 < d < 256 with d' r > 16384, whose kernels work on 256-feature
+ * blocks), and one FP64 partial record of d' r entries per row range of the first product
+ * (up to 64 MB).                                                                               */
 size_t gem_nlr_workspace_bytes(const gem_nlr_params *params);
 
 /* Device bytes the paper's own buffer table would use for the same problem:
