@@ -53,7 +53,7 @@ namespace gemnlr {
 struct TcgPlan {
     alignas(64) CUtensorMap tmX1;  // X-hat image h1 (n x d fp16): boxes of 128 rows x 32 features, 64-byte swizzle
     alignas(64) CUtensorMap tmX2;  // X-hat image h2
-    alignas(64) CUtensorMap tmU;   // U panels of the second product: 128 rows x 16 columns FP32
+    alignas(64) CUtensorMap tmU;   // U panels of the second product: 128 rows x 32 columns FP32, 128-byte swizzle
     int NCB;                       // 256-column blocks
     int eT;                        // Theta is scaled by 2^eT before its fp16 split
     int g2;
