@@ -60,7 +60,7 @@ def test_tc_trajectory_matches_oracle_and_is_reproducible(n, d, K):
 # one and several column blocks, r not a multiple of 16, ragged last row tile, more items than CTAs
 # (4100, 1024, 48): a narrow factor whose resident Theta images do not fit in shared memory, so it takes the tiled kernels
 TCG_SHAPES = [(4200, 64, 300), (4100, 768, 1000), (5000, 64, 520), (21000, 32, 260), (4200, 288, 600), (4100, 1024, 48),
-              (19001, 288, 600)]
+              (19001, 288, 600), (40001, 64, 300)]
 
 
 @pytest.mark.parametrize("n,d,K", TCG_SHAPES)
