@@ -61,7 +61,7 @@ __device__ __forceinline__ int team_warp_index(int w)          // 0 .. 11 over t
 }
 constexpr int WARP_UPROD = 9, WARP_XPROD = 13, WARP_ISSUER = 1, WARP_EPI0 = 4;
 constexpr int MAX_RING = 8;
-constexpr int FLUSH = 32;                      // stages per accumulation period (1024 rows)
+constexpr int FLUSH = 128;                     // stages per accumulation period (4096 rows)
 constexpr int UIMG = 128 * 64;                 // one fp16 image of the U operand: 128 columns x 32 data rows
 
 // XIMG = true: the X-hat operand comes from the static transposed fp16 images (one contiguous, pre-swizzled
