@@ -70,8 +70,8 @@ NCU_TRAFFIC = {
         "first": (7.29e9, "profiles/tcgen05_64x100_config3_many_cluster.md")},
     # first phase of the tiled family: the first-product kernel alone (the separate vector pass reads U once more)
     (2_000_000, 768, 1000, "f16x3.tiled"): {
-        "second": (21.49e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md"),
-        "first": (18.95e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md")},
+        "second": (21.51e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md"),
+        "first": (16.59e9, "profiles/f16x3_tiled_768x1000_config4_embedding.md")},
     (100_000_000, 32, 8, "ffma"): {
         "second": (19.50e9, "profiles/ffma_32x8_config5_massive.md"),
         "first": (16.81e9, "profiles/ffma_32x8_config5_massive.md")},
